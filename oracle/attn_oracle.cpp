@@ -1,0 +1,294 @@
+// TEST INFRASTRUCTURE — not part of the product path.
+//
+// Plain fp64 CPU oracle for hybrid-batch attention over a paged bf16 KV cache.
+// It is the definition written out: per request, per q head, per new-token row,
+// gather the keys through the block table, materialise the mask row explicitly,
+// compute scores, softmax and the weighted sum of values in double precision.
+// No tiling, no online softmax, no page-run logic, nothing shared with the
+// CUDA library (no common header, helper, table or constant).
+//
+// Only tests, the smoke check and the bench's cpu_baseline / reference arm may
+// load this library.
+//
+// What each function follows (paper = XY-Serve, arXiv 2412.18106):
+//   * attention = QK -> Softmax -> SV per tile unit, Section 4.2.1;
+//   * K/V read block by block through the block table, valid-token count of the
+//     last block tracked, Section 4.1.1; padded positions excluded, Section 5.2;
+//   * history columns fully visible and only the specLen x specLen corner
+//     masked for verify, Section 4.1.2; causal corner for prefill, Section 4.2.2;
+//   * merge of partial results over a split of the K/V dimension = the Update
+//     stage, Section 4.2.1.
+// Readings taken where the paper is silent: kv_len counts cached tokens BEFORE
+// the new ones; tree mask = ancestor-or-self of a parent array in topological
+// order; q head a reads kv head floor(a / (Hq/Hkv)); LSE is the natural log of
+// the sum of exp(sm_scale * q.k) over allowed keys.
+//
+// Pins (tests/test_oracle_*.py): softmax rows sum to 1; chunked == unchunked
+// prefill; prefix reuse == full recompute; chain tree == causal; decode == last
+// prefill row; closed forms (Q = 0, equal keys, constant V, single key, one-hot
+// V); star tree; an independently written brute force; torch fp64 softmax /
+// logsumexp on gathered K/V; page-permutation invariance; key-shift identity;
+// merge identity over arbitrary partitions; GQA special cases.
+
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <limits>
+#include <vector>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+namespace {
+
+// bf16 -> fp64, exact: bf16 is the top 16 bits of an IEEE fp32.
+inline double widen(uint16_t b) {
+  uint32_t u = static_cast<uint32_t>(b) << 16;
+  float f;
+  std::memcpy(&f, &u, sizeof f);
+  return static_cast<double>(f);
+}
+
+struct Problem {
+  int R, Hq, Hkv, D, B;
+  const int32_t* q_len;
+  const int32_t* kv_len;
+  const int32_t* mask_kind;   // 0 causal, 1 tree
+  const int32_t* parent_off;  // into parents, tree requests only
+  const int32_t* parents;
+  const uint16_t* q;
+  int64_t q_token_stride;
+  const uint16_t* k_pool;
+  const uint16_t* v_pool;
+  int64_t page_stride, head_stride, token_stride;
+  const int32_t* block_table;
+  int32_t bt_stride;
+  double sm_scale;
+};
+
+// Step 2: one explicit mask row, M[i][0..L).  History is always visible; the
+// corner is causal (j' <= i) or ancestor-or-self of the parent array.
+void mask_row(const Problem& p, int r, int i, std::vector<uint8_t>& m) {
+  const int n = p.q_len[r], h = p.kv_len[r], L = n + h;
+  m.assign(L, 0);
+  for (int j = 0; j < h; ++j) m[j] = 1;
+  if (p.mask_kind[r] == 0) {
+    for (int jp = 0; jp <= i; ++jp) m[h + jp] = 1;
+  } else {
+    const int32_t* par = p.parents + p.parent_off[r];
+    int node = i;
+    while (node >= 0) {
+      m[h + node] = 1;
+      node = par[node];
+    }
+  }
+}
+
+// Step 1: address of cached token j of request r, kv head g (elements).
+inline int64_t kv_offset(const Problem& p, int r, int g, int j) {
+  const int64_t page = p.block_table[static_cast<int64_t>(r) * p.bt_stride + j / p.B];
+  const int slot = j % p.B;
+  return page * p.page_stride + static_cast<int64_t>(g) * p.head_stride +
+         static_cast<int64_t>(slot) * p.token_stride;
+}
+
+// Steps 1-3 for one (request, q head, row).  Outputs: o[D], lse, sum of p,
+// and optionally the probabilities p[0..L).
+// `keep` (nullable, u8[L]) restricts the allowed set further (used to form the
+// partial results the merge identity is tested on); with no allowed key the
+// row's LSE is -inf and its O is 0.
+void attend_row(const Problem& p, int r, int64_t q_start, int a, int i, double* o, double* lse,
+                double* psum, double* probs, const uint8_t* keep = nullptr) {
+  const int n = p.q_len[r], h = p.kv_len[r], L = n + h, D = p.D;
+  const int g = a / (p.Hq / p.Hkv);
+  std::vector<uint8_t> m;
+  mask_row(p, r, i, m);
+  if (keep) {
+    bool any = false;
+    for (int j = 0; j < L; ++j) {
+      m[j] = m[j] && keep[j];
+      any = any || m[j];
+    }
+    if (!any) {
+      for (int d = 0; d < D; ++d) o[d] = 0.0;
+      *lse = -std::numeric_limits<double>::infinity();
+      if (psum) *psum = 0.0;
+      if (probs) for (int j = 0; j < L; ++j) probs[j] = 0.0;
+      return;
+    }
+  }
+  const uint16_t* qrow = p.q + (q_start + i) * p.q_token_stride + static_cast<int64_t>(a) * D;
+  std::vector<double> s(L, 0.0);
+  double mx = -std::numeric_limits<double>::infinity();
+  for (int j = 0; j < L; ++j) {
+    if (!m[j]) continue;
+    const uint16_t* krow = p.k_pool + kv_offset(p, r, g, j);
+    double acc = 0.0;
+    for (int d = 0; d < D; ++d) acc += widen(qrow[d]) * widen(krow[d]);
+    s[j] = p.sm_scale * acc;
+    if (s[j] > mx) mx = s[j];
+  }
+  double Z = 0.0;
+  for (int j = 0; j < L; ++j)
+    if (m[j]) Z += std::exp(s[j] - mx);
+  const double l = mx + std::log(Z);
+  for (int d = 0; d < D; ++d) o[d] = 0.0;
+  double ps = 0.0;
+  for (int j = 0; j < L; ++j) {
+    double pj = 0.0;
+    if (m[j]) {
+      pj = std::exp(s[j] - l);
+      const uint16_t* vrow = p.v_pool + kv_offset(p, r, g, j);
+      for (int d = 0; d < D; ++d) o[d] += pj * widen(vrow[d]);
+      ps += pj;
+    }
+    if (probs) probs[j] = pj;
+  }
+  *lse = l;
+  if (psum) *psum = ps;
+}
+
+Problem make_problem(int R, int Hq, int Hkv, int D, int B, const int32_t* q_len,
+                     const int32_t* kv_len, const int32_t* mask_kind, const int32_t* parent_off,
+                     const int32_t* parents, const uint16_t* q, int64_t q_token_stride,
+                     const uint16_t* k_pool, const uint16_t* v_pool, int64_t page_stride,
+                     int64_t head_stride, int64_t token_stride, const int32_t* block_table,
+                     int32_t bt_stride, double sm_scale) {
+  Problem p;
+  p.R = R; p.Hq = Hq; p.Hkv = Hkv; p.D = D; p.B = B;
+  p.q_len = q_len; p.kv_len = kv_len; p.mask_kind = mask_kind;
+  p.parent_off = parent_off; p.parents = parents;
+  p.q = q; p.q_token_stride = q_token_stride;
+  p.k_pool = k_pool; p.v_pool = v_pool;
+  p.page_stride = page_stride; p.head_stride = head_stride; p.token_stride = token_stride;
+  p.block_table = block_table; p.bt_stride = bt_stride; p.sm_scale = sm_scale;
+  return p;
+}
+
+}  // namespace
+
+#define PROBLEM_ARGS                                                                             \
+  int R, int Hq, int Hkv, int D, int B, const int32_t *q_len, const int32_t *kv_len,             \
+      const int32_t *mask_kind, const int32_t *parent_off, const int32_t *parents,               \
+      const uint16_t *q, int64_t q_token_stride, const uint16_t *k_pool, const uint16_t *v_pool, \
+      int64_t page_stride, int64_t head_stride, int64_t token_stride,                            \
+      const int32_t *block_table, int32_t bt_stride, double sm_scale
+#define PROBLEM_PASS                                                                          \
+  R, Hq, Hkv, D, B, q_len, kv_len, mask_kind, parent_off, parents, q, q_token_stride, k_pool, \
+      v_pool, page_stride, head_stride, token_stride, block_table, bt_stride, sm_scale
+
+extern "C" {
+
+int oracle_num_threads() {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+
+// Whole batch (or the requests flagged in `only`, nullable): O fp64 [T, Hq, D],
+// LSE fp64 [T, Hq], psum fp64 [T, Hq] (nullable) = sum of each row's probabilities.
+int oracle_attention(PROBLEM_ARGS, const uint8_t* only, double* O, double* LSE, double* psum) {
+  Problem p = make_problem(PROBLEM_PASS);
+  if (Hkv <= 0 || Hq % Hkv != 0) return -1;
+  std::vector<int64_t> q_start(R + 1, 0);
+  for (int r = 0; r < R; ++r) q_start[r + 1] = q_start[r] + q_len[r];
+  for (int r = 0; r < R; ++r) {
+    if (only && !only[r]) continue;
+    const int n = q_len[r];
+    const int64_t units = static_cast<int64_t>(n) * Hq;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t u = 0; u < units; ++u) {
+      const int i = static_cast<int>(u / Hq), a = static_cast<int>(u % Hq);
+      const int64_t row = (q_start[r] + i) * Hq + a;
+      attend_row(p, r, q_start[r], a, i, O + row * D, LSE + row, psum ? psum + row : nullptr,
+                 nullptr);
+    }
+  }
+  return 0;
+}
+
+// Sampled outputs: for s in [0, S): (req[s], head[s], row[s]) -> O fp64 [S, D], LSE fp64 [S].
+int oracle_attention_rows(PROBLEM_ARGS, int S, const int32_t* req, const int32_t* head,
+                          const int32_t* row, double* O, double* LSE) {
+  Problem p = make_problem(PROBLEM_PASS);
+  if (Hkv <= 0 || Hq % Hkv != 0) return -1;
+  std::vector<int64_t> q_start(R + 1, 0);
+  for (int r = 0; r < R; ++r) q_start[r + 1] = q_start[r] + q_len[r];
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int s = 0; s < S; ++s)
+    attend_row(p, req[s], q_start[req[s]], head[s], row[s], O + static_cast<int64_t>(s) * D,
+               LSE + s, nullptr, nullptr);
+  return 0;
+}
+
+// Probabilities of one (request, q head): P fp64 [n, L]; also the mask M u8 [n, L].
+int oracle_probs(PROBLEM_ARGS, int r, int a, double* P, uint8_t* M) {
+  Problem p = make_problem(PROBLEM_PASS);
+  std::vector<int64_t> q_start(R + 1, 0);
+  for (int x = 0; x < R; ++x) q_start[x + 1] = q_start[x] + q_len[x];
+  const int n = q_len[r], L = n + kv_len[r];
+  std::vector<double> o(D);
+  for (int i = 0; i < n; ++i) {
+    double lse, ps;
+    attend_row(p, r, q_start[r], a, i, o.data(), &lse, &ps, P + static_cast<int64_t>(i) * L);
+    std::vector<uint8_t> m;
+    mask_row(p, r, i, m);
+    std::memcpy(M + static_cast<int64_t>(i) * L, m.data(), L);
+  }
+  return 0;
+}
+
+// One row restricted to the keys flagged in keep[0..L): partial (O_c, LSE_c).
+int oracle_attention_keys(PROBLEM_ARGS, int r, int a, int i, const uint8_t* keep, double* O,
+                          double* LSE) {
+  Problem p = make_problem(PROBLEM_PASS);
+  std::vector<int64_t> q_start(R + 1, 0);
+  for (int x = 0; x < R; ++x) q_start[x + 1] = q_start[x] + q_len[x];
+  attend_row(p, r, q_start[r], a, i, O, LSE, nullptr, nullptr, keep);
+  return 0;
+}
+
+// Step 5: the gathered K and V rows of (request r, kv head g), bf16 bits, [L, D] each.
+int oracle_gather(PROBLEM_ARGS, int r, int g, uint16_t* K_out, uint16_t* V_out) {
+  Problem p = make_problem(PROBLEM_PASS);
+  const int L = q_len[r] + kv_len[r];
+  for (int j = 0; j < L; ++j) {
+    const int64_t off = kv_offset(p, r, g, j);
+    std::memcpy(K_out + static_cast<int64_t>(j) * D, k_pool + off, sizeof(uint16_t) * D);
+    std::memcpy(V_out + static_cast<int64_t>(j) * D, v_pool + off, sizeof(uint16_t) * D);
+  }
+  return 0;
+}
+
+// Step 4 (Update stage): merge C partial results of `rows` rows each.
+//   LSE = ln sum_c exp(LSE_c);  O = sum_c exp(LSE_c - LSE) O_c.
+// A chunk with LSE_c = -inf (no allowed key) contributes nothing.
+// O_c fp64 [C, rows, D], LSE_c fp64 [C, rows] -> O [rows, D], LSE [rows].
+int oracle_merge(int C, int64_t rows, int D, const double* O_c, const double* LSE_c, double* O,
+                 double* LSE) {
+  for (int64_t x = 0; x < rows; ++x) {
+    double mx = -std::numeric_limits<double>::infinity();
+    for (int c = 0; c < C; ++c) mx = std::fmax(mx, LSE_c[c * rows + x]);
+    double Z = 0.0;
+    for (int c = 0; c < C; ++c) {
+      const double l = LSE_c[c * rows + x];
+      if (std::isinf(l) && l < 0) continue;
+      Z += std::exp(l - mx);
+    }
+    const double lse = mx + std::log(Z);
+    for (int d = 0; d < D; ++d) O[x * D + d] = 0.0;
+    for (int c = 0; c < C; ++c) {
+      const double l = LSE_c[c * rows + x];
+      if (std::isinf(l) && l < 0) continue;
+      const double w = std::exp(l - lse);
+      for (int d = 0; d < D; ++d) O[x * D + d] += w * O_c[(c * rows + x) * D + d];
+    }
+    LSE[x] = lse;
+  }
+  return 0;
+}
+
+}  // extern "C"
