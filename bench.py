@@ -1,0 +1,379 @@
+"""Bench of the hybrid-batch attention hot path (plan once, run K steps) on synthetic batches.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+One step = one pass of the whole hot path (attention kernel + split-KV merge) over one
+synthetic hybrid batch.  Prints ONE JSON line.  `value` is useful TFLOP/s (masked-out work
+excluded) with inputs resident in HBM; `kv_gbs` is K+V GB/s of the same runs; `e2e` repeats
+the measurement through the public API with the step's inputs (Q, block table, request
+table) coming from pinned host memory and O / LSE read back, host-side planning included.
+The KV cache itself is device-resident state, as in serving.
+
+`--impl reference` times the fp64 CPU oracle (as it stands) on a bounded sample of the same
+workload on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+SCALE = 1.0 / math.sqrt(128.0)
+NOMINAL_TFLOPS = 2250.0
+NOMINAL_GBS = 8000.0
+FALLBACK_TFLOPS = 1590.0
+FALLBACK_TFLOPS_SUSTAINED = 1400.0
+FALLBACK_GBS = 6650.0
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": FALLBACK_GBS, "bf16_tflops": FALLBACK_TFLOPS,
+            "bf16_tflops_sustained": FALLBACK_TFLOPS_SUSTAINED, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, pw, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+                pw.append(float(parts[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)),
+                "power_w_max": float(max(pw)), "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def dist_env():
+    return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+
+
+def pick_sample(batch, rng, target_pairs):
+    """Rows (request, head, row) drawn in proportion to nothing in particular: uniform over
+    all (token, head) rows, until the allowed pairs reach `target_pairs`."""
+    T, Hq = batch.total_q, batch.num_q_heads
+    q_start = batch.q_start
+    req_of_tok = np.repeat(np.arange(batch.num_requests), batch.q_len)
+    order = rng.permutation(T * Hq)
+    req, head, row, pairs = [], [], [], 0
+    for x in order:
+        t, a = divmod(int(x), Hq)
+        r = int(req_of_tok[t])
+        i = t - int(q_start[r])
+        req.append(r)
+        head.append(a)
+        row.append(i)
+        pairs += int(batch.kv_len[r]) + i + 1
+        if pairs >= target_pairs:
+            break
+    return np.array(req, np.int32), np.array(head, np.int32), np.array(row, np.int32), pairs
+
+
+def time_oracle_sample(batch, tensors, seconds_target=12.0):
+    """Times the oracle on a bounded random sample of output rows of the workload."""
+    import oracle
+    rng = np.random.default_rng(1234)
+    # calibrate on a small sample, then size the real one for about `seconds_target`
+    req, head, row, pairs = pick_sample(batch, rng, 2_000_000)
+    t0 = time.perf_counter()
+    oracle.attention_rows(batch, tensors, SCALE, req, head, row)
+    dt = max(time.perf_counter() - t0, 1e-4)
+    rate = pairs / dt
+    req, head, row, pairs = pick_sample(batch, rng, int(rate * seconds_target))
+    t0 = time.perf_counter()
+    oracle.attention_rows(batch, tensors, SCALE, req, head, row)
+    dt = time.perf_counter() - t0
+    flops = 4.0 * batch.head_dim * pairs
+    return {"tflops": flops / dt / 1e12, "seconds": dt, "rows": int(len(req)), "pairs": int(pairs),
+            "cores": oracle.num_threads()}
+
+
+def tree_pairs_note():
+    return "pairs counted as kv_len + row + 1 per sampled row (causal bound; tree rows see fewer)"
+
+
+def run_reference(args):
+    rank, local_rank, world = dist_env()
+    if rank != 0:
+        return 0
+    from paper_2412_18106_b200 import workloads as W
+    batch = W.CONFIGS[args.workload](seed=0)
+    tensors = W.make_tensors(batch)
+    # each "step" is one bounded sample; warm-up steps are shorter
+    per_step = max(2.0, min(12.0, 150.0 / max(1, args.steps + args.warmup)))
+    for _ in range(args.warmup):
+        time_oracle_sample(batch, tensors, per_step / 4)
+    vals, secs, rows = [], 0.0, 0
+    for _ in range(args.steps):
+        r = time_oracle_sample(batch, tensors, per_step)
+        vals.append(r["tflops"])
+        secs += r["seconds"]
+        rows = r["rows"]
+        cores = r["cores"]
+    v = float(np.mean(vals))
+    line = {
+        "impl": "reference", "metric": "hybrid_attention_useful_tflops", "value": v, "unit": "TFLOP/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": 1e3 * secs / max(1, args.steps), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "num_requests": batch.num_requests,
+                   "total_q_tokens": batch.total_q},
+        "cpu_baseline": {"value": v, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
+                         "sample": "%d random output rows (request, head, token) of the workload per step; %s"
+                                   % (rows, tree_pairs_note())},
+        "e2e": {"value": v, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="full_mix",
+                    choices=["decode_only", "splitfuse_mix", "verify_trees", "full_mix", "tiny_hybrid"])
+    ap.add_argument("--kernel", default="auto", choices=["auto", "reference", "mma"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import torch.distributed as dist
+
+    from paper_2412_18106_b200 import binding as xb
+    from paper_2412_18106_b200 import workloads as W
+
+    rank, local_rank, world = dist_env()
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU path)"
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    warmup = max(3, args.warmup)
+    # weak scaling: every rank serves its own batch of the same recipe (independent requests,
+    # no exchange on the data path)
+    batch = W.CONFIGS[args.workload](seed=rank)
+    tensors = W.make_tensors(batch)
+    kernel = {"auto": xb.XY_KERNEL_AUTO, "reference": xb.XY_KERNEL_REFERENCE, "mma": xb.XY_KERNEL_MMA}[args.kernel]
+    ctx = xb.XYAttn(batch.num_q_heads, batch.num_kv_heads, batch.page_size, device=local_rank,
+                    kernel=kernel, max_requests=max(256, batch.num_requests),
+                    max_q_tokens=max(1 << 15, batch.total_q),
+                    max_pages_per_req=max(1024, batch.block_table.shape[1]),
+                    max_tree_nodes=max(64, int(batch.q_len.max())))
+    t0 = time.perf_counter()
+    info = ctx.plan_batch(batch)
+    plan_us = (time.perf_counter() - t0) * 1e6
+
+    bt_host = torch.from_numpy(np.where(batch.block_table < 0, 0, batch.block_table).astype(np.int32))
+    q_host = tensors.q.contiguous().pin_memory()
+    bt_pin = bt_host.pin_memory()
+    q = q_host.to(dev)
+    k_pool = tensors.k_pool.to(dev)
+    v_pool = tensors.v_pool.to(dev)
+    bt = bt_host.to(dev)
+    T, Hq, D = batch.total_q, batch.num_q_heads, batch.head_dim
+    o = torch.empty((T, Hq, D), dtype=torch.bfloat16, device=dev)
+    lse = torch.empty((T, Hq), dtype=torch.float32, device=dev)
+    o_host = torch.empty((T, Hq, D), dtype=torch.bfloat16).pin_memory()
+    lse_host = torch.empty((T, Hq), dtype=torch.float32).pin_memory()
+
+    flops = float(info.useful_flops)
+    kvb = float(info.kv_bytes)
+    alg_bytes = float(W.algorithmic_bytes(batch))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def step():
+        ctx.run(q, k_pool, v_pool, bt, SCALE, o, lse)
+
+    for _ in range(warmup):
+        step()
+    barrier()
+    assert ctx.device_status() == 0
+
+    # ---- timed region: K steps, inputs resident in HBM; KV pools are far larger than L2
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    ctx.set_timing(True)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record()
+    for _ in range(args.steps):
+        step()
+    ev1.record()
+    barrier()
+    total_ms = ev0.elapsed_time(ev1)
+    attn_ms, merge_ms, runs = ctx.get_timing()
+    ctx.set_timing(False)
+    launches = ctx.last_launches() * args.steps
+    clocks = sampler.stop() if rank == 0 else None
+    tms = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(tms, op=dist.ReduceOp.MAX)
+    ms_per_step = float(tms.item()) / args.steps
+    # every rank processes the same recipe; whole-job units = sum over ranks
+    tot = torch.tensor([flops, kvb], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(tot, op=dist.ReduceOp.SUM)
+    job_flops, job_kvb = float(tot[0].item()), float(tot[1].item())
+    value = job_flops / (ms_per_step * 1e-3) / 1e12
+    kv_gbs = job_kvb / (ms_per_step * 1e-3) / 1e9
+
+    # ---- end to end: host planning + H2D of the step's inputs + run + D2H of O and LSE
+    e2e = None
+    if not args.no_e2e:
+        def e2e_step():
+            ctx.plan_batch(batch)
+            q.copy_(q_host, non_blocking=True)
+            bt.copy_(bt_pin, non_blocking=True)
+            ctx.run(q, k_pool, v_pool, bt, SCALE, o, lse)
+            o_host.copy_(o, non_blocking=True)
+            lse_host.copy_(lse, non_blocking=True)
+            torch.cuda.synchronize()
+        for _ in range(3):
+            e2e_step()
+        barrier()
+        n_e2e = max(3, min(args.steps, 20))
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n_e2e):
+            e2e_step()
+        e1.record()
+        barrier()
+        ems = torch.tensor([e0.elapsed_time(e1) / n_e2e], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(ems, op=dist.ReduceOp.MAX)
+        e2e_ms = float(ems.item())
+        h2d = q_host.numel() * 2 + bt_pin.numel() * 4 + info.num_tasks * 32 + batch.num_requests * 32
+        d2h = o_host.numel() * 2 + lse_host.numel() * 4
+        e2e = {"value": job_flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
+               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": n_e2e,
+               "includes": "host plan + H2D(Q, block table, task tables) + run + D2H(O, LSE); KV cache resident"}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return 0
+
+    peaks = measured_peaks()
+    attn_ms_avg = attn_ms / max(1, runs)
+    t_flop = flops / (peaks["bf16_tflops_sustained"] * 1e12)
+    t_byte = alg_bytes / (peaks["hbm_gbs"] * 1e9)
+    if t_flop >= t_byte:
+        roof = {"bound": "tensor", "achieved": flops / (attn_ms_avg * 1e-3) / 1e12,
+                "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s"}
+    else:
+        roof = {"bound": "hbm", "achieved": alg_bytes / (attn_ms_avg * 1e-3) / 1e9,
+                "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["traffic"] = None
+    roof["peak_source"] = peaks["source"] + (" (sustained bf16)" if roof["bound"] == "tensor" else " (copy)")
+    roof["kernel"] = "attention meta-kernel"
+    roof["kernel_ms"] = attn_ms_avg
+    roof["merge_ms"] = merge_ms / max(1, runs)
+    roof["algorithmic_flops"] = flops
+    roof["algorithmic_bytes"] = alg_bytes
+    roof["t_roof_us_measured"] = 1e6 * max(t_flop, t_byte)
+    roof["t_roof_us_nominal"] = 1e6 * max(flops / (NOMINAL_TFLOPS * 1e12), alg_bytes / (NOMINAL_GBS * 1e9))
+    roof["frac_of_nominal_roofline"] = roof["t_roof_us_nominal"] / (attn_ms_avg * 1e3)
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        r = time_oracle_sample(batch, tensors, 12.0)
+        cpu = {"value": r["tflops"], "unit": "TFLOP/s", "cores": r["cores"], "kind": "oracle",
+               "sample": "%d random output rows (request, head, token) of the workload, %.1f s; %s"
+                         % (r["rows"], r["seconds"], tree_pairs_note())}
+
+    line = {
+        "metric": "hybrid_attention_useful_tflops", "value": value, "unit": "TFLOP/s",
+        "kv_gbs": kv_gbs, "n_gpus": world, "steps": args.steps, "warmup": warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, "num_requests": batch.num_requests,
+                   "total_q_tokens": batch.total_q, "q_heads": batch.num_q_heads,
+                   "kv_heads": batch.num_kv_heads, "page_size": batch.page_size,
+                   "kv_tokens": int((batch.q_len + batch.kv_len).sum()), "kernel": args.kernel,
+                   "tasks": info.num_tasks, "merge_units": info.num_merge_units,
+                   "plan_us": plan_us, "l2": "KV pool (%.2f GB) exceeds L2; no flush" % (2 * k_pool.numel() * 2 / 1e9),
+                   "parallelism": "replicas x%d (requests sharded, no collective)" % world},
+        "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

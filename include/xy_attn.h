@@ -1,0 +1,211 @@
+/*
+ * xy_attn — hybrid-batch attention meta-kernel for NVIDIA B200 (sm_100a).
+ *
+ * One launch computes matmul-softmax-matmul for a mixed batch of chunked-prefill
+ * requests (optionally on a reused cached prefix), single-token decode requests
+ * and speculative-verify requests (a token tree under a tree mask), all reading
+ * a paged bf16 KV cache, and writes O (bf16) and LSE (fp32).
+ *
+ * The calls follow the problem statement of XY-Serve (arXiv 2412.18106):
+ *   - Token-Table: one entry per stage {stageID, start position, tokenNum,
+ *     historical kvLen, tileSize}                                (Section 3.2.1)
+ *   - decomposition into tile units and reordering into a Task-Table that maps
+ *     each core to its list of tiles                       (Sections 3.2.1, 3.3.1)
+ *   - Meta-Attention: QK -> Softmax -> SV per tile unit over K/V blocks read by
+ *     block table, with mask-aware skipping            (Sections 4.1.1, 4.2.1, 4.2.2)
+ *   - only the specLen x specLen corner of a verify mask is non-trivial and is
+ *     supplied from outside                                        (Section 4.1.2)
+ *   - Q is read with a stride from a fused QKV tensor and O is written as
+ *     [tokens, heads, headSize]                                     (Section 5.4)
+ *
+ * Conventions.  Every call returns an int status (XY_OK or a negative XY_ERR_*),
+ * never throws and never aborts.  "HOST" / "DEVICE" beside a pointer says where
+ * the memory lives.  The caller owns every buffer it passes in; the context owns
+ * its task tables, tree masks, split-KV workspace and status word.  No call
+ * falls back to the CPU: without a usable CUDA device `xy_attn_run` fails.
+ */
+#ifndef XY_ATTN_H_
+#define XY_ATTN_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct xy_attn_ctx xy_attn_ctx; /* opaque */
+
+enum {
+  XY_OK = 0,
+  XY_ERR_INVALID_ARG = -1,    /* null pointer, bad size, bad stride, bad head ratio */
+  XY_ERR_CAPACITY = -2,       /* batch exceeds a capacity given at create */
+  XY_ERR_BAD_TREE = -3,       /* parent[i] not in {-1} U [0, i-1] */
+  XY_ERR_NOT_PLANNED = -4,    /* run before a successful plan */
+  XY_ERR_CUDA = -5,           /* a CUDA runtime/driver call failed; see xy_attn_last_error */
+  XY_ERR_DEVICE_TIMEOUT = -6, /* a bounded wait inside a kernel gave up */
+  XY_ERR_UNSUPPORTED = -7     /* head_dim != 128, page size not a power of two in 8..128, ... */
+};
+
+enum { XY_MASK_CAUSAL = 0, XY_MASK_TREE = 1 };
+
+/* Which kernels xy_attn_run uses. */
+enum {
+  XY_KERNEL_AUTO = 0,      /* tcgen05 dense tiles + streaming decode tiles (the product path) */
+  XY_KERNEL_REFERENCE = 1, /* plain SIMT kernel for every tile: slow, kept for bisecting */
+  XY_KERNEL_MMA = 2        /* warp-level mma.sync tiles for every task (dense tasks too) */
+};
+
+/* Task-Table construction (Section 3.3.1). */
+enum {
+  XY_PLAN_BALANCED = 0, /* cost = max(tensor time, HBM time) of the visible page run; long
+                           runs are cut into KV splits; sorted + symmetric round-robin */
+  XY_PLAN_PAPER = 1     /* the paper's table literally: one task per tile unit, no KV split,
+                           load = rows x visible keys, sorted + symmetric round-robin */
+};
+
+typedef struct {
+  int32_t num_q_heads;       /* Hq */
+  int32_t num_kv_heads;      /* Hkv, divides Hq; q head a reads kv head a / (Hq/Hkv) */
+  int32_t head_dim;          /* 128 */
+  int32_t page_size;         /* B: tokens per KV page, power of two in 8..128 */
+  int32_t max_requests;      /* capacity: requests per plan */
+  int32_t max_q_tokens;      /* capacity: total new tokens per plan */
+  int32_t max_pages_per_req; /* capacity: pages a single request may reference */
+  int32_t max_tree_nodes;    /* capacity: nodes of one verify tree */
+  int32_t device;            /* CUDA device ordinal; -1 = host-only context (plan works, run fails) */
+  int32_t num_workers;       /* 0 = one worker per SM of the device (148 on B200) */
+  int32_t kernel;            /* XY_KERNEL_* */
+  int32_t plan_mode;         /* XY_PLAN_* */
+  int32_t tile_tokens;       /* XY_PLAN_PAPER only: tileSize in tokens (0 = 128 / (Hq/Hkv)) */
+  int32_t max_splits;        /* upper bound on KV splits of one tile unit (0 = 32) */
+  int64_t workspace_bytes;   /* split-KV workspace (fp32 partial O and LSE); 0 = 256 MiB */
+} xy_attn_config;
+
+/* One Token-Table entry as the caller states it (Section 3.2.1).  The start
+ * position is the prefix sum of q_len in request order, computed by plan. */
+typedef struct {
+  int32_t q_len;      /* tokenNum: new tokens this step, >= 1 */
+  int32_t kv_len;     /* historical kvLen: cached tokens BEFORE the new ones, >= 0 */
+  int32_t mask_kind;  /* XY_MASK_CAUSAL (prefill, decode) or XY_MASK_TREE (verify) */
+  int32_t parent_off; /* XY_MASK_TREE: index of this request's first node in tree_parents; else -1 */
+} xy_attn_request;
+
+/* One meta-task of the Task-Table: a packed Q tile against a run of 128-key KV
+ * tiles.  Row x of the packed tile is (token tok0 + x / G, q head kv_head*G + x % G),
+ * G = Hq/Hkv. */
+typedef struct {
+  int32_t req;     /* request index */
+  int32_t kv_head; /* kv head */
+  int32_t tok0;    /* first new token of the tile, relative to the request */
+  int32_t ntok;    /* tokens in the tile; rows = ntok * G */
+  int32_t kt_lo;   /* first 128-key tile of the run */
+  int32_t kt_hi;   /* one past the last 128-key tile of the run */
+  int32_t part;    /* -1: the task writes final O and LSE; >= 0: first row of its fp32 partial */
+  int32_t kind;    /* 0 dense (rows > 16), 1 streaming (rows <= 16: decode, tiny verify) */
+} xy_attn_task;
+
+/* A tile unit whose KV range was split: its `nsplit` partials of `rows` rows each
+ * start at partial row `part0` and are `rows` apart. */
+typedef struct {
+  int32_t req, kv_head, tok0, ntok;
+  int32_t part0, nsplit;
+} xy_attn_merge_unit;
+
+typedef struct {
+  int32_t num_tasks;
+  int32_t num_dense_tasks;
+  int32_t num_merge_units;
+  int32_t num_workers;
+  int64_t useful_flops;   /* 4 D Hq sum of allowed (row, key) pairs */
+  int64_t kv_bytes;       /* K+V bytes with each cached token of each kv head read once per request */
+  int64_t partial_rows;   /* fp32 partial rows used in the workspace */
+  float load_min, load_mean, load_max; /* per-worker summed task cost */
+  float max_task_cost;
+} xy_attn_plan_info;
+
+/* Create a context.  Allocates the device-side tables and the split workspace
+ * once (cudaMalloc); plan and run allocate nothing.  cfg->device = -1 makes a
+ * host-only context for planning without a GPU. */
+int xy_attn_create(const xy_attn_config* cfg /*HOST*/, xy_attn_ctx** out /*HOST*/);
+int xy_attn_destroy(xy_attn_ctx* ctx);
+
+/* Token-Table -> decomposition -> Task-Table (Sections 3.2.1, 3.3.1).  Host work
+ * plus asynchronous host-to-device copies of the tables on `stream` (a
+ * cudaStream_t, may be 0).  `reqs` and `tree_parents` are HOST arrays, read
+ * before return.  tree_parents holds the parent arrays of the XY_MASK_TREE
+ * requests back to back: parent[i] in {-1} U [0, i-1] (several roots allowed);
+ * anything else gives XY_ERR_BAD_TREE.  The ancestor-or-self bit matrix
+ * (ceil(n/64) 64-bit words per node, bit j' of row i set iff j' is i or one of
+ * its ancestors) is built here.  Zero requests is valid and makes run a no-op.
+ * On error the previous plan is discarded. */
+int xy_attn_plan(xy_attn_ctx* ctx, const xy_attn_request* reqs /*HOST*/, int32_t num_reqs,
+                 const int32_t* tree_parents /*HOST, nullable if no tree*/, int32_t num_parents,
+                 void* stream, xy_attn_plan_info* info /*HOST, nullable*/);
+
+/* Meta-Attention over the planned batch (Sections 4.1-4.2, 5.2, 5.4).
+ * Asynchronous on `stream`; no allocation, no host synchronisation.
+ *   q            DEVICE bf16; row of token t, head a at q + t*q_token_stride + a*D
+ *                (elements; q_token_stride >= Hq*D and a multiple of 8, so a fused
+ *                [tokens, Hq + 2 Hkv, D] tensor can be passed directly)
+ *   k_pool/v_pool DEVICE bf16 [num_pages, Hkv, B, D]; element strides page_stride,
+ *                head_stride, token_stride (multiples of 8; D contiguous); every
+ *                element of every page a request references must be finite
+ *   block_table  DEVICE int32 [num_reqs, block_table_stride]; row r holds at least
+ *                ceil((kv_len+q_len)/B) page ids in [0, num_pages)
+ *   tree_mask    DEVICE, nullable: a caller-built corner mask in plan's format
+ *                replacing the one plan built from the parent arrays
+ *   o            DEVICE bf16 [T, Hq, D] with token stride o_token_stride (elements)
+ *   lse          DEVICE fp32 [T, Hq]: natural log of sum exp(sm_scale * q.k) over allowed keys
+ * The new tokens' K/V must already be in the cache at positions kv_len .. kv_len+q_len-1. */
+int xy_attn_run(xy_attn_ctx* ctx, const void* q, int64_t q_token_stride, const void* k_pool,
+                const void* v_pool, int64_t num_pages, int64_t page_stride, int64_t head_stride,
+                int64_t token_stride, const int32_t* block_table, int32_t block_table_stride,
+                const uint64_t* tree_mask, float sm_scale, void* o, int64_t o_token_stride,
+                float* lse, void* stream);
+
+/* Split-KV LSE merge alone (the cross-core form of the Update stage, Section 4.2.1):
+ *   LSE = ln sum_c exp(LSE_c),  O = sum_c exp(LSE_c - LSE) O_c.
+ * o_part DEVICE fp32 [num_splits, rows, D], lse_part DEVICE fp32 [num_splits, rows];
+ * o DEVICE bf16 [rows, D], lse DEVICE fp32 [rows].  A partial with LSE_c = -inf is ignored.
+ * Needs no context; asynchronous on `stream`. */
+int xy_attn_merge(const float* o_part, const float* lse_part, int32_t num_splits, int64_t rows,
+                  int32_t head_dim, void* o, float* lse, void* stream);
+
+/* Debug/verification: copy the K and V rows a request sees, in logical order,
+ * through the block table: out_k/out_v DEVICE bf16 [kv_len+q_len, D] for kv head
+ * `kv_head` of planned request `req`. */
+int xy_attn_debug_gather(xy_attn_ctx* ctx, int32_t req, int32_t kv_head, const void* k_pool,
+                         const void* v_pool, int64_t page_stride, int64_t head_stride,
+                         int64_t token_stride, const int32_t* block_table,
+                         int32_t block_table_stride, void* out_k, void* out_v, void* stream);
+
+/* Introspection of the current plan (HOST outputs).  Each returns the number of
+ * items of the plan, or a negative error; at most `cap` items are written. */
+int xy_attn_get_tasks(const xy_attn_ctx* ctx, xy_attn_task* out, int32_t cap);
+int xy_attn_get_worker_offsets(const xy_attn_ctx* ctx, int32_t* out /* num_workers+1 */, int32_t cap);
+int xy_attn_get_merge_units(const xy_attn_ctx* ctx, xy_attn_merge_unit* out, int32_t cap);
+int xy_attn_get_tree_mask(const xy_attn_ctx* ctx, uint64_t* out, int32_t cap_words);
+int xy_attn_get_q_start(const xy_attn_ctx* ctx, int32_t* out /* num_reqs+1 */, int32_t cap);
+
+/* Per-kernel device timing.  With timing enabled every xy_attn_run records CUDA events on
+ * its stream around the attention launch and around the merge launch (at most 4096 runs
+ * are kept).  xy_attn_get_timing waits for the last recorded run, returns the summed
+ * durations in milliseconds and the number of runs they cover, and clears the record. */
+int xy_attn_set_timing(xy_attn_ctx* ctx, int32_t enable);
+int xy_attn_get_timing(xy_attn_ctx* ctx, float* attention_ms /*HOST*/, float* merge_ms /*HOST*/,
+                       int32_t* runs /*HOST*/);
+
+/* Number of kernel launches the last xy_attn_run enqueued. */
+int xy_attn_last_launches(const xy_attn_ctx* ctx);
+
+/* Message of the last error on this context (never null). */
+const char* xy_attn_last_error(const xy_attn_ctx* ctx);
+
+/* Synchronises the device and reads the status word the kernels write:
+ * XY_OK, or XY_ERR_DEVICE_TIMEOUT when a bounded wait inside a kernel gave up. */
+int xy_attn_device_status(xy_attn_ctx* ctx, int32_t* status_out /*HOST*/);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* XY_ATTN_H_ */

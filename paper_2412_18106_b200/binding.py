@@ -1,0 +1,273 @@
+"""Thin ctypes binding of the C-ABI library (include/xy_attn.h), same names.
+
+Argument marshalling only: every step of the path runs in the CUDA kernels.
+PyTorch is used for device memory and streams.  There is no CPU fallback: if the
+shared library is missing the import fails loudly, and `run` needs CUDA tensors.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libxy_attn.so")
+
+XY_OK = 0
+XY_ERR_INVALID_ARG = -1
+XY_ERR_CAPACITY = -2
+XY_ERR_BAD_TREE = -3
+XY_ERR_NOT_PLANNED = -4
+XY_ERR_CUDA = -5
+XY_ERR_DEVICE_TIMEOUT = -6
+XY_ERR_UNSUPPORTED = -7
+
+XY_MASK_CAUSAL = 0
+XY_MASK_TREE = 1
+
+XY_KERNEL_AUTO = 0
+XY_KERNEL_REFERENCE = 1
+XY_KERNEL_MMA = 2
+
+XY_PLAN_BALANCED = 0
+XY_PLAN_PAPER = 1
+
+
+class xy_attn_config(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in (
+        "num_q_heads", "num_kv_heads", "head_dim", "page_size", "max_requests", "max_q_tokens",
+        "max_pages_per_req", "max_tree_nodes", "device", "num_workers", "kernel", "plan_mode",
+        "tile_tokens", "max_splits")] + [("workspace_bytes", ctypes.c_int64)]
+
+
+class xy_attn_request(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("q_len", "kv_len", "mask_kind", "parent_off")]
+
+
+class xy_attn_task(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in (
+        "req", "kv_head", "tok0", "ntok", "kt_lo", "kt_hi", "part", "kind")]
+
+
+class xy_attn_merge_unit(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("req", "kv_head", "tok0", "ntok", "part0", "nsplit")]
+
+
+class xy_attn_plan_info(ctypes.Structure):
+    _fields_ = [("num_tasks", ctypes.c_int32), ("num_dense_tasks", ctypes.c_int32),
+                ("num_merge_units", ctypes.c_int32), ("num_workers", ctypes.c_int32),
+                ("useful_flops", ctypes.c_int64), ("kv_bytes", ctypes.c_int64),
+                ("partial_rows", ctypes.c_int64), ("load_min", ctypes.c_float),
+                ("load_mean", ctypes.c_float), ("load_max", ctypes.c_float),
+                ("max_task_cost", ctypes.c_float)]
+
+
+TASK_DTYPE = np.dtype([(n, np.int32) for n in ("req", "kv_head", "tok0", "ntok", "kt_lo", "kt_hi", "part", "kind")])
+MERGE_DTYPE = np.dtype([(n, np.int32) for n in ("req", "kv_head", "tok0", "ntok", "part0", "nsplit")])
+
+EXPORTS = (
+    "xy_attn_create", "xy_attn_destroy", "xy_attn_plan", "xy_attn_run", "xy_attn_merge",
+    "xy_attn_debug_gather", "xy_attn_get_tasks", "xy_attn_get_worker_offsets",
+    "xy_attn_get_merge_units", "xy_attn_get_tree_mask", "xy_attn_get_q_start",
+    "xy_attn_last_launches", "xy_attn_last_error", "xy_attn_device_status",
+    "xy_attn_set_timing", "xy_attn_get_timing",
+)
+
+_lib = None
+
+
+def load() -> ctypes.CDLL:
+    """Loads libxy_attn.so (built in-tree by `python -m paper_2412_18106_b200.build`)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            "CUDA extension missing: %s not built (run python -m paper_2412_18106_b200.build). "
+            "There is no CPU fallback." % LIB_PATH)
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+    L.xy_attn_create.argtypes = [ctypes.POINTER(xy_attn_config), ctypes.POINTER(vp)]
+    L.xy_attn_destroy.argtypes = [vp]
+    L.xy_attn_plan.argtypes = [vp, vp, i32, vp, i32, vp, ctypes.POINTER(xy_attn_plan_info)]
+    L.xy_attn_run.argtypes = [vp, vp, i64, vp, vp, i64, i64, i64, i64, vp, i32, vp, ctypes.c_float,
+                              vp, i64, vp, vp]
+    L.xy_attn_merge.argtypes = [vp, vp, i32, i64, i32, vp, vp, vp]
+    L.xy_attn_debug_gather.argtypes = [vp, i32, i32, vp, vp, i64, i64, i64, vp, i32, vp, vp, vp]
+    for name in ("xy_attn_get_tasks", "xy_attn_get_worker_offsets", "xy_attn_get_merge_units",
+                 "xy_attn_get_tree_mask", "xy_attn_get_q_start"):
+        getattr(L, name).argtypes = [vp, vp, i32]
+    L.xy_attn_set_timing.argtypes = [vp, i32]
+    L.xy_attn_get_timing.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float),
+                                     ctypes.POINTER(i32)]
+    L.xy_attn_last_launches.argtypes = [vp]
+    L.xy_attn_last_error.argtypes = [vp]
+    L.xy_attn_last_error.restype = ctypes.c_char_p
+    L.xy_attn_device_status.argtypes = [vp, ctypes.POINTER(i32)]
+    for name in EXPORTS:
+        if name != "xy_attn_last_error":
+            getattr(L, name).restype = ctypes.c_int
+    _lib = L
+    return L
+
+
+class XYAttnError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__("xy_attn error %d: %s" % (code, msg))
+        self.code = code
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> ctypes.c_void_p:
+    if stream is None:
+        if torch.cuda.is_available():
+            return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+        return ctypes.c_void_p(0)
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+class XYAttn:
+    """One xy_attn context.  Methods mirror the C entry points."""
+
+    def __init__(self, num_q_heads: int, num_kv_heads: int, page_size: int, *, head_dim: int = 128,
+                 max_requests: int = 256, max_q_tokens: int = 1 << 15, max_pages_per_req: int = 1024,
+                 max_tree_nodes: int = 64, device: int = 0, num_workers: int = 0,
+                 kernel: int = XY_KERNEL_AUTO, plan_mode: int = XY_PLAN_BALANCED, tile_tokens: int = 0,
+                 max_splits: int = 0, workspace_bytes: int = 0):
+        self.lib = load()
+        self.cfg = xy_attn_config(num_q_heads, num_kv_heads, head_dim, page_size, max_requests,
+                                  max_q_tokens, max_pages_per_req, max_tree_nodes, device, num_workers,
+                                  kernel, plan_mode, tile_tokens, max_splits, workspace_bytes)
+        self._ctx = ctypes.c_void_p(0)
+        rc = self.lib.xy_attn_create(ctypes.byref(self.cfg), ctypes.byref(self._ctx))
+        if rc != XY_OK:
+            raise XYAttnError(rc, "xy_attn_create failed")
+        self.info = xy_attn_plan_info()
+
+    def close(self):
+        if self._ctx and self._ctx.value:
+            self.lib.xy_attn_destroy(self._ctx)
+            self._ctx = ctypes.c_void_p(0)
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, rc: int):
+        if rc != XY_OK:
+            raise XYAttnError(rc, self.lib.xy_attn_last_error(self._ctx).decode())
+
+    # -- xy_attn_plan
+    def plan(self, q_len: Sequence[int], kv_len: Sequence[int], mask_kind: Sequence[int],
+             parent_off: Sequence[int], parents=None, stream=None) -> xy_attn_plan_info:
+        R = len(q_len)
+        reqs = (xy_attn_request * max(R, 1))()
+        for r in range(R):
+            reqs[r] = xy_attn_request(int(q_len[r]), int(kv_len[r]), int(mask_kind[r]), int(parent_off[r]))
+        par = np.ascontiguousarray(np.asarray(parents if parents is not None else [], dtype=np.int32))
+        par_ptr = ctypes.c_void_p(par.ctypes.data) if par.size else ctypes.c_void_p(0)
+        self._check(self.lib.xy_attn_plan(self._ctx, ctypes.cast(reqs, ctypes.c_void_p), R, par_ptr,
+                                          int(par.size), _stream_ptr(stream), ctypes.byref(self.info)))
+        return self.info
+
+    def plan_batch(self, batch, stream=None) -> xy_attn_plan_info:
+        return self.plan(batch.q_len, batch.kv_len, batch.mask_kind, batch.parent_off, batch.parents, stream)
+
+    # -- xy_attn_run
+    def run(self, q: torch.Tensor, k_pool: torch.Tensor, v_pool: torch.Tensor,
+            block_table: torch.Tensor, sm_scale: float, o: torch.Tensor, lse: torch.Tensor,
+            tree_mask: Optional[torch.Tensor] = None, stream=None) -> None:
+        for t in (q, k_pool, v_pool, block_table, o, lse):
+            if not t.is_cuda:
+                raise XYAttnError(XY_ERR_INVALID_ARG, "run needs CUDA tensors (there is no CPU path)")
+        assert q.dtype == torch.bfloat16 and k_pool.dtype == torch.bfloat16 and v_pool.dtype == torch.bfloat16
+        assert o.dtype == torch.bfloat16 and lse.dtype == torch.float32 and block_table.dtype == torch.int32
+        assert q.stride(2) == 1 and q.stride(1) == self.cfg.head_dim
+        assert o.stride(2) == 1 and o.stride(1) == self.cfg.head_dim and lse.is_contiguous()
+        assert k_pool.stride() == v_pool.stride() and k_pool.stride(3) == 1
+        assert block_table.stride(1) == 1
+        tm = ctypes.c_void_p(tree_mask.data_ptr()) if tree_mask is not None else ctypes.c_void_p(0)
+        self._check(self.lib.xy_attn_run(
+            self._ctx, q.data_ptr(), q.stride(0), k_pool.data_ptr(), v_pool.data_ptr(),
+            k_pool.shape[0], k_pool.stride(0), k_pool.stride(1), k_pool.stride(2),
+            block_table.data_ptr(), block_table.stride(0), tm, float(sm_scale), o.data_ptr(),
+            o.stride(0), lse.data_ptr(), _stream_ptr(stream)))
+
+    # -- xy_attn_debug_gather
+    def debug_gather(self, req: int, kv_head: int, k_pool, v_pool, block_table, out_k, out_v, stream=None):
+        self._check(self.lib.xy_attn_debug_gather(
+            self._ctx, req, kv_head, k_pool.data_ptr(), v_pool.data_ptr(), k_pool.stride(0),
+            k_pool.stride(1), k_pool.stride(2), block_table.data_ptr(), block_table.stride(0),
+            out_k.data_ptr(), out_v.data_ptr(), _stream_ptr(stream)))
+
+    # -- introspection
+    def _get(self, fn, dtype, count_hint=0):
+        n = fn(self._ctx, ctypes.c_void_p(0), 0)
+        if n < 0:
+            self._check(n)
+        out = np.zeros(max(n, 1), dtype=dtype)
+        fn(self._ctx, ctypes.c_void_p(out.ctypes.data), n)
+        return out[:n]
+
+    def get_tasks(self) -> np.ndarray:
+        return self._get(self.lib.xy_attn_get_tasks, TASK_DTYPE)
+
+    def get_worker_offsets(self) -> np.ndarray:
+        return self._get(self.lib.xy_attn_get_worker_offsets, np.int32)
+
+    def get_merge_units(self) -> np.ndarray:
+        return self._get(self.lib.xy_attn_get_merge_units, MERGE_DTYPE)
+
+    def get_tree_mask(self) -> np.ndarray:
+        return self._get(self.lib.xy_attn_get_tree_mask, np.uint64)
+
+    def get_q_start(self) -> np.ndarray:
+        return self._get(self.lib.xy_attn_get_q_start, np.int32)
+
+    def set_timing(self, enable: bool) -> None:
+        self._check(self.lib.xy_attn_set_timing(self._ctx, 1 if enable else 0))
+
+    def get_timing(self):
+        """(attention kernel ms, merge kernel ms, runs) summed since the last call."""
+        a, m, n = ctypes.c_float(0), ctypes.c_float(0), ctypes.c_int32(0)
+        self._check(self.lib.xy_attn_get_timing(self._ctx, ctypes.byref(a), ctypes.byref(m), ctypes.byref(n)))
+        return float(a.value), float(m.value), int(n.value)
+
+    def last_launches(self) -> int:
+        return int(self.lib.xy_attn_last_launches(self._ctx))
+
+    def last_error(self) -> str:
+        return self.lib.xy_attn_last_error(self._ctx).decode()
+
+    def device_status(self) -> int:
+        st = ctypes.c_int32(0)
+        self._check(self.lib.xy_attn_device_status(self._ctx, ctypes.byref(st)))
+        return int(st.value)
+
+
+def xy_attn_merge(o_part: torch.Tensor, lse_part: torch.Tensor, o: torch.Tensor, lse: torch.Tensor,
+                  stream=None) -> None:
+    """Split-KV LSE merge: o_part fp32 [S, rows, D], lse_part fp32 [S, rows] -> o bf16, lse fp32."""
+    L = load()
+    assert o_part.is_cuda and o_part.is_contiguous() and lse_part.is_contiguous()
+    S, rows, D = o_part.shape
+    rc = L.xy_attn_merge(o_part.data_ptr(), lse_part.data_ptr(), S, rows, D, o.data_ptr(),
+                         lse.data_ptr(), _stream_ptr(stream))
+    if rc != XY_OK:
+        raise XYAttnError(rc, "xy_attn_merge failed")
+
+
+def attention(ctx: XYAttn, batch, q, k_pool, v_pool, block_table, sm_scale, o=None, lse=None,
+              tree_mask=None, stream=None):
+    """Convenience: allocate O / LSE if needed and run the planned batch."""
+    T = q.shape[0]
+    if o is None:
+        o = torch.empty((T, ctx.cfg.num_q_heads, ctx.cfg.head_dim), dtype=torch.bfloat16, device=q.device)
+    if lse is None:
+        lse = torch.empty((T, ctx.cfg.num_q_heads), dtype=torch.float32, device=q.device)
+    ctx.run(q, k_pool, v_pool, block_table, sm_scale, o, lse, tree_mask=tree_mask, stream=stream)
+    return o, lse

@@ -1,0 +1,395 @@
+// C-ABI layer: context, plan, run, merge, introspection.  Argument checking and
+// marshalling only; every step of the path runs in the kernels.
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "xy_internal.h"
+#include "xy_kernels.h"
+
+using namespace xy;
+
+struct xy_attn_ctx {
+  xy_attn_config cfg{};
+  int num_workers = 0;
+  bool host_only = false;
+  int page_shift = 0;
+  bool planned = false;
+  PlanResult plan;
+  // capacities of the device tables
+  int64_t cap_tasks = 0, cap_merges = 0, cap_tree_words = 0, cap_partial_rows = 0;
+  ReqInfo* d_reqs = nullptr;
+  xy_attn_task* d_tasks = nullptr;
+  int32_t* d_worker_off = nullptr;
+  uint64_t* d_tree = nullptr;
+  xy_attn_merge_unit* d_merges = nullptr;
+  float* d_o_part = nullptr;
+  float* d_lse_part = nullptr;
+  int32_t* d_status = nullptr;
+  int last_launches = 0;
+  bool timing = false;
+  std::vector<cudaEvent_t> events;  // three per timed run: before attention, after it, after merge
+  int timed_runs = 0;
+  std::string err = "";
+};
+
+namespace {
+
+int set_err(xy_attn_ctx* c, int code, const std::string& msg) {
+  if (c) c->err = msg;
+  return code;
+}
+
+int cuda_fail(xy_attn_ctx* c, cudaError_t e, const char* what) {
+  return set_err(c, XY_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+}
+
+#define XY_CUDA(ctx, call)                                   \
+  do {                                                       \
+    cudaError_t e__ = (call);                                \
+    if (e__ != cudaSuccess) return cuda_fail(ctx, e__, #call); \
+  } while (0)
+
+constexpr int kMaxTimedRuns = 4096;
+
+bool pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
+
+void free_device(xy_attn_ctx* c) {
+  if (c->host_only) return;
+  for (cudaEvent_t ev : c->events) cudaEventDestroy(ev);
+  c->events.clear();
+  cudaFree(c->d_reqs);
+  cudaFree(c->d_tasks);
+  cudaFree(c->d_worker_off);
+  cudaFree(c->d_tree);
+  cudaFree(c->d_merges);
+  cudaFree(c->d_o_part);
+  cudaFree(c->d_lse_part);
+  cudaFree(c->d_status);
+}
+
+}  // namespace
+
+extern "C" {
+
+int xy_attn_create(const xy_attn_config* cfg, xy_attn_ctx** out) {
+  if (cfg == nullptr || out == nullptr) return XY_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (cfg->head_dim != kHeadDim) return XY_ERR_UNSUPPORTED;
+  if (!pow2(cfg->page_size) || cfg->page_size < 8 || cfg->page_size > 128) return XY_ERR_UNSUPPORTED;
+  if (cfg->num_q_heads < 1 || cfg->num_kv_heads < 1 || cfg->num_q_heads % cfg->num_kv_heads != 0)
+    return XY_ERR_INVALID_ARG;
+  if (cfg->num_q_heads / cfg->num_kv_heads > 128) return XY_ERR_UNSUPPORTED;
+  if (cfg->max_requests < 1 || cfg->max_q_tokens < 1 || cfg->max_pages_per_req < 1 ||
+      cfg->max_tree_nodes < 0 || cfg->num_workers < 0 || cfg->max_splits < 0 ||
+      cfg->workspace_bytes < 0 || cfg->tile_tokens < 0)
+    return XY_ERR_INVALID_ARG;
+  if (cfg->kernel < XY_KERNEL_AUTO || cfg->kernel > XY_KERNEL_MMA) return XY_ERR_INVALID_ARG;
+  if (cfg->plan_mode != XY_PLAN_BALANCED && cfg->plan_mode != XY_PLAN_PAPER) return XY_ERR_INVALID_ARG;
+
+  xy_attn_ctx* c = new (std::nothrow) xy_attn_ctx();
+  if (c == nullptr) return XY_ERR_INVALID_ARG;
+  c->cfg = *cfg;
+  c->host_only = cfg->device < 0;
+  while ((1 << c->page_shift) < cfg->page_size) ++c->page_shift;
+  c->num_workers = cfg->num_workers;
+  if (!c->host_only) {
+    cudaError_t e = cudaSetDevice(cfg->device);
+    if (e != cudaSuccess) {
+      delete c;
+      return XY_ERR_CUDA;
+    }
+    if (c->num_workers == 0) {
+      int sms = 0;
+      e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, cfg->device);
+      if (e != cudaSuccess || sms <= 0) {
+        delete c;
+        return XY_ERR_CUDA;
+      }
+      c->num_workers = sms;
+    }
+  } else if (c->num_workers == 0) {
+    c->num_workers = 148;
+  }
+
+  const int G = cfg->num_q_heads / cfg->num_kv_heads;
+  const int sub_tok = 128 / G > 0 ? 128 / G : 1;
+  const int tile_tok = cfg->plan_mode == XY_PLAN_PAPER
+                           ? (cfg->tile_tokens > 0 ? cfg->tile_tokens : sub_tok)
+                           : 2 * sub_tok;
+  const int64_t units_max = static_cast<int64_t>(cfg->num_kv_heads) *
+                            (cfg->max_requests + cfg->max_q_tokens / tile_tok + 1);
+  c->cap_tasks = 2 * units_max + 4ll * c->num_workers + 16;
+  c->cap_merges = units_max;
+  c->cap_tree_words =
+      static_cast<int64_t>(cfg->max_q_tokens) * ((cfg->max_tree_nodes + 63) / 64) + 1;
+  const int64_t ws = cfg->workspace_bytes > 0 ? cfg->workspace_bytes : (256ll << 20);
+  c->cap_partial_rows = ws / ((kHeadDim + 1) * 4);
+
+  if (!c->host_only) {
+    cudaError_t e = cudaSuccess;
+    auto alloc = [&](void** p, size_t bytes) {
+      if (e == cudaSuccess) e = cudaMalloc(p, bytes < 256 ? 256 : bytes);
+    };
+    alloc(reinterpret_cast<void**>(&c->d_reqs), sizeof(ReqInfo) * cfg->max_requests);
+    alloc(reinterpret_cast<void**>(&c->d_tasks), sizeof(xy_attn_task) * c->cap_tasks);
+    alloc(reinterpret_cast<void**>(&c->d_worker_off), sizeof(int32_t) * (c->num_workers + 1));
+    alloc(reinterpret_cast<void**>(&c->d_tree), sizeof(uint64_t) * c->cap_tree_words);
+    alloc(reinterpret_cast<void**>(&c->d_merges), sizeof(xy_attn_merge_unit) * c->cap_merges);
+    alloc(reinterpret_cast<void**>(&c->d_o_part), sizeof(float) * kHeadDim * c->cap_partial_rows);
+    alloc(reinterpret_cast<void**>(&c->d_lse_part), sizeof(float) * c->cap_partial_rows);
+    alloc(reinterpret_cast<void**>(&c->d_status), 256);
+    if (e == cudaSuccess) e = cudaMemset(c->d_status, 0, 256);
+    if (e != cudaSuccess) {
+      free_device(c);
+      delete c;
+      return XY_ERR_CUDA;
+    }
+  }
+  *out = c;
+  return XY_OK;
+}
+
+int xy_attn_destroy(xy_attn_ctx* ctx) {
+  if (ctx == nullptr) return XY_ERR_INVALID_ARG;
+  if (!ctx->host_only) {
+    cudaSetDevice(ctx->cfg.device);
+    cudaDeviceSynchronize();
+    free_device(ctx);
+  }
+  delete ctx;
+  return XY_OK;
+}
+
+int xy_attn_plan(xy_attn_ctx* ctx, const xy_attn_request* reqs, int32_t num_reqs,
+                 const int32_t* tree_parents, int32_t num_parents, void* stream,
+                 xy_attn_plan_info* info) {
+  if (ctx == nullptr) return XY_ERR_INVALID_ARG;
+  ctx->planned = false;
+  std::string err;
+  int rc = build_plan(ctx->cfg, ctx->num_workers, ctx->cap_partial_rows, reqs, num_reqs,
+                      tree_parents, num_parents, &ctx->plan, &err);
+  if (rc != XY_OK) {
+    ctx->plan = PlanResult();
+    return set_err(ctx, rc, err);
+  }
+  PlanResult& p = ctx->plan;
+  if (static_cast<int64_t>(p.tasks.size()) > ctx->cap_tasks ||
+      static_cast<int64_t>(p.merges.size()) > ctx->cap_merges ||
+      static_cast<int64_t>(p.tree_mask.size()) > ctx->cap_tree_words) {
+    ctx->plan = PlanResult();
+    return set_err(ctx, XY_ERR_CAPACITY, "plan exceeds the table capacities fixed at create");
+  }
+  if (!ctx->host_only) {
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    XY_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+    // Pageable sources: the runtime stages them before returning, so the vectors may change.
+    if (!p.reqs.empty())
+      XY_CUDA(ctx, cudaMemcpyAsync(ctx->d_reqs, p.reqs.data(), sizeof(ReqInfo) * p.reqs.size(),
+                                   cudaMemcpyHostToDevice, s));
+    if (!p.tasks.empty())
+      XY_CUDA(ctx, cudaMemcpyAsync(ctx->d_tasks, p.tasks.data(),
+                                   sizeof(xy_attn_task) * p.tasks.size(), cudaMemcpyHostToDevice, s));
+    XY_CUDA(ctx, cudaMemcpyAsync(ctx->d_worker_off, p.worker_off.data(),
+                                 sizeof(int32_t) * p.worker_off.size(), cudaMemcpyHostToDevice, s));
+    if (!p.tree_mask.empty())
+      XY_CUDA(ctx, cudaMemcpyAsync(ctx->d_tree, p.tree_mask.data(),
+                                   sizeof(uint64_t) * p.tree_mask.size(), cudaMemcpyHostToDevice, s));
+    if (!p.merges.empty())
+      XY_CUDA(ctx, cudaMemcpyAsync(ctx->d_merges, p.merges.data(),
+                                   sizeof(xy_attn_merge_unit) * p.merges.size(),
+                                   cudaMemcpyHostToDevice, s));
+  }
+  if (info) *info = p.info;
+  ctx->planned = true;
+  ctx->err = "";
+  return XY_OK;
+}
+
+int xy_attn_run(xy_attn_ctx* ctx, const void* q, int64_t q_token_stride, const void* k_pool,
+                const void* v_pool, int64_t num_pages, int64_t page_stride, int64_t head_stride,
+                int64_t token_stride, const int32_t* block_table, int32_t block_table_stride,
+                const uint64_t* tree_mask, float sm_scale, void* o, int64_t o_token_stride,
+                float* lse, void* stream) {
+  if (ctx == nullptr) return XY_ERR_INVALID_ARG;
+  ctx->last_launches = 0;
+  if (ctx->host_only) return set_err(ctx, XY_ERR_UNSUPPORTED, "host-only context cannot run");
+  if (!ctx->planned) return set_err(ctx, XY_ERR_NOT_PLANNED, "xy_attn_run before xy_attn_plan");
+  const PlanResult& p = ctx->plan;
+  if (p.tasks.empty()) return XY_OK;
+  const xy_attn_config& cfg = ctx->cfg;
+  if (!q || !k_pool || !v_pool || !block_table || !o || !lse)
+    return set_err(ctx, XY_ERR_INVALID_ARG, "null device pointer");
+  auto misaligned = [](const void* ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15u) != 0; };
+  if (misaligned(q) || misaligned(k_pool) || misaligned(v_pool) || misaligned(o))
+    return set_err(ctx, XY_ERR_INVALID_ARG, "q, k_pool, v_pool and o must be 16-byte aligned");
+  if (q_token_stride < static_cast<int64_t>(cfg.num_q_heads) * kHeadDim || q_token_stride % 8 != 0 ||
+      o_token_stride < static_cast<int64_t>(cfg.num_q_heads) * kHeadDim || o_token_stride % 8 != 0)
+    return set_err(ctx, XY_ERR_INVALID_ARG, "token stride of q / o too small or not a multiple of 8");
+  if (token_stride < kHeadDim || token_stride % 8 != 0 || head_stride % 8 != 0 || head_stride < 1 ||
+      page_stride % 8 != 0 || page_stride < 1 || num_pages < 1)
+    return set_err(ctx, XY_ERR_INVALID_ARG, "bad K/V pool strides or num_pages");
+  if (block_table_stride < 1) return set_err(ctx, XY_ERR_INVALID_ARG, "bad block_table_stride");
+
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  XY_CUDA(ctx, cudaSetDevice(cfg.device));
+  RunArgs a{};
+  a.q = static_cast<const uint16_t*>(q);
+  a.q_token_stride = q_token_stride;
+  a.k_pool = static_cast<const uint16_t*>(k_pool);
+  a.v_pool = static_cast<const uint16_t*>(v_pool);
+  a.page_stride = page_stride;
+  a.head_stride = head_stride;
+  a.token_stride = token_stride;
+  a.block_table = block_table;
+  a.bt_stride = block_table_stride;
+  a.tree_mask = tree_mask ? tree_mask : ctx->d_tree;
+  a.sm_scale = sm_scale;
+  a.o = static_cast<uint16_t*>(o);
+  a.o_token_stride = o_token_stride;
+  a.lse = lse;
+  a.reqs = ctx->d_reqs;
+  a.tasks = ctx->d_tasks;
+  a.worker_off = ctx->d_worker_off;
+  a.o_part = ctx->d_o_part;
+  a.lse_part = ctx->d_lse_part;
+  a.status = ctx->d_status;
+  a.num_q_heads = cfg.num_q_heads;
+  a.num_kv_heads = cfg.num_kv_heads;
+  a.page_size = cfg.page_size;
+  a.page_shift = ctx->page_shift;
+
+  const bool timed = ctx->timing && ctx->timed_runs < kMaxTimedRuns;
+  if (timed) {
+    while (static_cast<int>(ctx->events.size()) < 3 * (ctx->timed_runs + 1)) {
+      cudaEvent_t ev;
+      XY_CUDA(ctx, cudaEventCreate(&ev));
+      ctx->events.push_back(ev);
+    }
+    XY_CUDA(ctx, cudaEventRecord(ctx->events[3 * ctx->timed_runs], s));
+  }
+
+  XY_CUDA(ctx, launch_reference(a, ctx->num_workers, s));
+  ctx->last_launches += 1;
+  if (timed) XY_CUDA(ctx, cudaEventRecord(ctx->events[3 * ctx->timed_runs + 1], s));
+
+  if (!p.merges.empty()) {
+    MergeArgs m{};
+    m.units = ctx->d_merges;
+    m.reqs = ctx->d_reqs;
+    m.o_part = ctx->d_o_part;
+    m.lse_part = ctx->d_lse_part;
+    m.o = a.o;
+    m.o_token_stride = o_token_stride;
+    m.lse = lse;
+    m.num_q_heads = cfg.num_q_heads;
+    m.num_kv_heads = cfg.num_kv_heads;
+    XY_CUDA(ctx, launch_merge_units(m, static_cast<int>(p.merges.size()), s));
+    ctx->last_launches += 1;
+  }
+  if (timed) {
+    XY_CUDA(ctx, cudaEventRecord(ctx->events[3 * ctx->timed_runs + 2], s));
+    ctx->timed_runs += 1;
+  }
+  return XY_OK;
+}
+
+int xy_attn_set_timing(xy_attn_ctx* ctx, int32_t enable) {
+  if (ctx == nullptr) return XY_ERR_INVALID_ARG;
+  if (ctx->host_only) return set_err(ctx, XY_ERR_UNSUPPORTED, "host-only context");
+  ctx->timing = enable != 0;
+  ctx->timed_runs = 0;
+  return XY_OK;
+}
+
+int xy_attn_get_timing(xy_attn_ctx* ctx, float* attention_ms, float* merge_ms, int32_t* runs) {
+  if (ctx == nullptr || !attention_ms || !merge_ms || !runs) return XY_ERR_INVALID_ARG;
+  if (ctx->host_only) return set_err(ctx, XY_ERR_UNSUPPORTED, "host-only context");
+  float ta = 0.f, tm = 0.f;
+  if (ctx->timed_runs > 0) {
+    XY_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+    XY_CUDA(ctx, cudaEventSynchronize(ctx->events[3 * ctx->timed_runs - 1]));
+    for (int i = 0; i < ctx->timed_runs; ++i) {
+      float x = 0.f, y = 0.f;
+      XY_CUDA(ctx, cudaEventElapsedTime(&x, ctx->events[3 * i], ctx->events[3 * i + 1]));
+      XY_CUDA(ctx, cudaEventElapsedTime(&y, ctx->events[3 * i + 1], ctx->events[3 * i + 2]));
+      ta += x;
+      tm += y;
+    }
+  }
+  *attention_ms = ta;
+  *merge_ms = tm;
+  *runs = ctx->timed_runs;
+  ctx->timed_runs = 0;
+  return XY_OK;
+}
+
+int xy_attn_merge(const float* o_part, const float* lse_part, int32_t num_splits, int64_t rows,
+                  int32_t head_dim, void* o, float* lse, void* stream) {
+  if (head_dim != kHeadDim) return XY_ERR_UNSUPPORTED;
+  if (num_splits < 1 || rows < 0) return XY_ERR_INVALID_ARG;
+  if (rows == 0) return XY_OK;
+  if (!o_part || !lse_part || !o || !lse) return XY_ERR_INVALID_ARG;
+  cudaError_t e = launch_merge_plain(o_part, lse_part, num_splits, rows, static_cast<uint16_t*>(o),
+                                     lse, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? XY_OK : XY_ERR_CUDA;
+}
+
+int xy_attn_debug_gather(xy_attn_ctx* ctx, int32_t req, int32_t kv_head, const void* k_pool,
+                         const void* v_pool, int64_t page_stride, int64_t head_stride,
+                         int64_t token_stride, const int32_t* block_table,
+                         int32_t block_table_stride, void* out_k, void* out_v, void* stream) {
+  if (ctx == nullptr) return XY_ERR_INVALID_ARG;
+  if (ctx->host_only) return set_err(ctx, XY_ERR_UNSUPPORTED, "host-only context cannot run");
+  if (!ctx->planned) return set_err(ctx, XY_ERR_NOT_PLANNED, "gather before plan");
+  if (req < 0 || req >= static_cast<int32_t>(ctx->plan.reqs.size()) || kv_head < 0 ||
+      kv_head >= ctx->cfg.num_kv_heads || !k_pool || !v_pool || !block_table || !out_k || !out_v)
+    return set_err(ctx, XY_ERR_INVALID_ARG, "bad gather argument");
+  const ReqInfo& r = ctx->plan.reqs[req];
+  XY_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+  XY_CUDA(ctx, launch_gather(static_cast<const uint16_t*>(k_pool),
+                             static_cast<const uint16_t*>(v_pool), page_stride, head_stride,
+                             token_stride,
+                             block_table + static_cast<int64_t>(req) * block_table_stride,
+                             ctx->cfg.page_size, ctx->page_shift, kv_head, r.q_len + r.kv_len,
+                             static_cast<uint16_t*>(out_k), static_cast<uint16_t*>(out_v),
+                             static_cast<cudaStream_t>(stream)));
+  return XY_OK;
+}
+
+#define XY_GETTER(name, type, vec)                                              \
+  int name(const xy_attn_ctx* ctx, type* out, int32_t cap) {                    \
+    if (ctx == nullptr || (out == nullptr && cap > 0)) return XY_ERR_INVALID_ARG; \
+    if (!ctx->planned) return XY_ERR_NOT_PLANNED;                               \
+    const auto& v = ctx->plan.vec;                                              \
+    const size_t n = v.size() < static_cast<size_t>(cap < 0 ? 0 : cap) ? v.size() : (cap < 0 ? 0 : cap); \
+    if (n) std::memcpy(out, v.data(), n * sizeof(type));                        \
+    return static_cast<int>(v.size());                                          \
+  }
+
+XY_GETTER(xy_attn_get_tasks, xy_attn_task, tasks)
+XY_GETTER(xy_attn_get_worker_offsets, int32_t, worker_off)
+XY_GETTER(xy_attn_get_merge_units, xy_attn_merge_unit, merges)
+XY_GETTER(xy_attn_get_tree_mask, uint64_t, tree_mask)
+XY_GETTER(xy_attn_get_q_start, int32_t, q_start)
+
+int xy_attn_last_launches(const xy_attn_ctx* ctx) { return ctx ? ctx->last_launches : XY_ERR_INVALID_ARG; }
+
+const char* xy_attn_last_error(const xy_attn_ctx* ctx) { return ctx ? ctx->err.c_str() : "null context"; }
+
+int xy_attn_device_status(xy_attn_ctx* ctx, int32_t* status_out) {
+  if (ctx == nullptr || status_out == nullptr) return XY_ERR_INVALID_ARG;
+  if (ctx->host_only) return set_err(ctx, XY_ERR_UNSUPPORTED, "host-only context");
+  XY_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+  XY_CUDA(ctx, cudaDeviceSynchronize());
+  int32_t st = 0;
+  XY_CUDA(ctx, cudaMemcpy(&st, ctx->d_status, sizeof st, cudaMemcpyDeviceToHost));
+  *status_out = st;
+  return XY_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,210 @@
+// Reference attention kernel (plain SIMT, fp32), the split-KV LSE merge and the
+// block-table gather.  The reference kernel walks the same Task-Table as the fast
+// kernels and is kept for bisecting: one warp per packed row, one key at a time.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "xy_kernels.h"
+
+namespace xy {
+
+namespace {
+
+__device__ __forceinline__ float bf16_bits_to_float(uint16_t b) {
+  return __uint_as_float(static_cast<uint32_t>(b) << 16);
+}
+
+__device__ __forceinline__ uint16_t float_to_bf16_bits(float f) {
+  return __bfloat16_as_ushort(__float2bfloat16_rn(f));
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Section 4.2.1 (QK -> Softmax -> SV per tile unit, with the Update rescale), Section 4.1.1
+// (K/V rows found through the block table), Sections 4.1.2 / 4.2.2 (row-wise mask control).
+__global__ void __launch_bounds__(128) ref_attention_kernel(RunArgs a) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int G = a.num_q_heads / a.num_kv_heads;
+  const int t_begin = a.worker_off[blockIdx.x], t_end = a.worker_off[blockIdx.x + 1];
+  for (int ti = t_begin; ti < t_end; ++ti) {
+    const xy_attn_task t = a.tasks[ti];
+    const ReqInfo rq = a.reqs[t.req];
+    const int rows = t.ntok * G;
+    const int32_t* bt = a.block_table + static_cast<int64_t>(t.req) * a.bt_stride;
+    for (int x = warp; x < rows; x += 4) {
+      const int i = t.tok0 + x / G;
+      const int head = t.kv_head * G + x % G;
+      const uint16_t* qp =
+          a.q + static_cast<int64_t>(rq.q_start + i) * a.q_token_stride + head * kHeadDim + lane * 4;
+      float qv[4];
+#pragma unroll
+      for (int d = 0; d < 4; ++d) qv[d] = bf16_bits_to_float(qp[d]);
+      const uint64_t* mrow = nullptr;
+      if (rq.mask_kind == XY_MASK_TREE)
+        mrow = a.tree_mask + rq.tree_off + static_cast<int64_t>(i) * rq.tree_words;
+      const int j_lo = t.kt_lo * kKeyTile;
+      const int j_hi = min(t.kt_hi * kKeyTile, rq.kv_len + i + 1);
+      float m = -INFINITY, l = 0.f, o[4] = {0.f, 0.f, 0.f, 0.f};
+      for (int j = j_lo; j < j_hi; ++j) {
+        if (j >= rq.kv_len && mrow != nullptr) {
+          const int jp = j - rq.kv_len;
+          if (((mrow[jp >> 6] >> (jp & 63)) & 1ull) == 0ull) continue;
+        }
+        const int64_t page = bt[j >> a.page_shift];
+        const int64_t off = page * a.page_stride + static_cast<int64_t>(t.kv_head) * a.head_stride +
+                            static_cast<int64_t>(j & (a.page_size - 1)) * a.token_stride + lane * 4;
+        const uint16_t* kp = a.k_pool + off;
+        const uint16_t* vp = a.v_pool + off;
+        float dot = 0.f;
+#pragma unroll
+        for (int d = 0; d < 4; ++d) dot += qv[d] * bf16_bits_to_float(kp[d]);
+        const float s = warp_sum(dot) * a.sm_scale;
+        const float m_new = fmaxf(m, s);
+        const float alpha = __expf(m - m_new);  // m = -inf on the first key: alpha = 0
+        const float p = __expf(s - m_new);
+        l = l * alpha + p;
+#pragma unroll
+        for (int d = 0; d < 4; ++d) o[d] = o[d] * alpha + p * bf16_bits_to_float(vp[d]);
+        m = m_new;
+      }
+      const float inv = l > 0.f ? 1.f / l : 0.f;
+      const float lse = l > 0.f ? m + logf(l) : -INFINITY;
+      if (t.part < 0) {
+        uint16_t* op = a.o + static_cast<int64_t>(rq.q_start + i) * a.o_token_stride +
+                       head * kHeadDim + lane * 4;
+#pragma unroll
+        for (int d = 0; d < 4; ++d) op[d] = float_to_bf16_bits(o[d] * inv);
+        if (lane == 0) a.lse[static_cast<int64_t>(rq.q_start + i) * a.num_q_heads + head] = lse;
+      } else {
+        float* op = a.o_part + static_cast<int64_t>(t.part + x) * kHeadDim + lane * 4;
+#pragma unroll
+        for (int d = 0; d < 4; ++d) op[d] = o[d] * inv;
+        if (lane == 0) a.lse_part[t.part + x] = lse;
+      }
+    }
+  }
+}
+
+// Cross-task form of the Update stage (Section 4.2.1): combine the partials of every tile
+// unit whose KV range was split.  One block per merge unit, one warp per packed row.
+__global__ void __launch_bounds__(128) merge_units_kernel(MergeArgs a) {
+  const xy_attn_merge_unit u = a.units[blockIdx.x];
+  const ReqInfo rq = a.reqs[u.req];
+  const int G = a.num_q_heads / a.num_kv_heads;
+  const int rows = u.ntok * G;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int x = warp; x < rows; x += 4) {
+    float mx = -INFINITY;
+    for (int c = 0; c < u.nsplit; ++c) mx = fmaxf(mx, a.lse_part[u.part0 + c * rows + x]);
+    float z = 0.f;
+    for (int c = 0; c < u.nsplit; ++c) {
+      const float lc = a.lse_part[u.part0 + c * rows + x];
+      if (lc != -INFINITY) z += __expf(lc - mx);
+    }
+    const float lse = mx + logf(z);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int c = 0; c < u.nsplit; ++c) {
+      const float lc = a.lse_part[u.part0 + c * rows + x];
+      if (lc == -INFINITY) continue;
+      const float w = __expf(lc - lse);
+      const float4 v = *reinterpret_cast<const float4*>(
+          a.o_part + static_cast<int64_t>(u.part0 + c * rows + x) * kHeadDim + lane * 4);
+      acc.x += w * v.x;
+      acc.y += w * v.y;
+      acc.z += w * v.z;
+      acc.w += w * v.w;
+    }
+    const int i = u.tok0 + x / G;
+    const int head = u.kv_head * G + x % G;
+    uint16_t* op =
+        a.o + static_cast<int64_t>(rq.q_start + i) * a.o_token_stride + head * kHeadDim + lane * 4;
+    uint2 packed;
+    packed.x = float_to_bf16_bits(acc.x) | (static_cast<uint32_t>(float_to_bf16_bits(acc.y)) << 16);
+    packed.y = float_to_bf16_bits(acc.z) | (static_cast<uint32_t>(float_to_bf16_bits(acc.w)) << 16);
+    *reinterpret_cast<uint2*>(op) = packed;
+    if (lane == 0) a.lse[static_cast<int64_t>(rq.q_start + i) * a.num_q_heads + head] = lse;
+  }
+}
+
+// Context-free merge over plain [num_splits, rows, D] partials.
+__global__ void __launch_bounds__(128) merge_plain_kernel(const float* o_part, const float* lse_part,
+                                                         int num_splits, int64_t rows, uint16_t* o,
+                                                         float* lse_out) {
+  const int lane = threadIdx.x & 31;
+  const int64_t x = static_cast<int64_t>(blockIdx.x) * 4 + (threadIdx.x >> 5);
+  if (x >= rows) return;
+  float mx = -INFINITY;
+  for (int c = 0; c < num_splits; ++c) mx = fmaxf(mx, lse_part[c * rows + x]);
+  float z = 0.f;
+  for (int c = 0; c < num_splits; ++c) {
+    const float lc = lse_part[c * rows + x];
+    if (lc != -INFINITY) z += __expf(lc - mx);
+  }
+  const float lse = mx + logf(z);
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  for (int c = 0; c < num_splits; ++c) {
+    const float lc = lse_part[c * rows + x];
+    if (lc == -INFINITY) continue;
+    const float w = __expf(lc - lse);
+    const float* v = o_part + (c * rows + x) * kHeadDim + lane * 4;
+#pragma unroll
+    for (int d = 0; d < 4; ++d) acc[d] += w * v[d];
+  }
+#pragma unroll
+  for (int d = 0; d < 4; ++d) o[x * kHeadDim + lane * 4 + d] = float_to_bf16_bits(acc[d]);
+  if (lane == 0) lse_out[x] = lse;
+}
+
+// Step a5 in isolation: copy the rows a request sees, in logical order (Section 4.1.1).
+__global__ void gather_kernel(const uint16_t* k_pool, const uint16_t* v_pool, int64_t page_stride,
+                              int64_t head_stride, int64_t token_stride, const int32_t* bt,
+                              int page_size, int page_shift, int kv_head, int L, uint16_t* out_k,
+                              uint16_t* out_v) {
+  const int j = blockIdx.x * 4 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (j >= L) return;
+  const int64_t page = bt[j >> page_shift];
+  const int64_t off = page * page_stride + static_cast<int64_t>(kv_head) * head_stride +
+                      static_cast<int64_t>(j & (page_size - 1)) * token_stride + lane * 4;
+  *reinterpret_cast<uint2*>(out_k + static_cast<int64_t>(j) * kHeadDim + lane * 4) =
+      *reinterpret_cast<const uint2*>(k_pool + off);
+  *reinterpret_cast<uint2*>(out_v + static_cast<int64_t>(j) * kHeadDim + lane * 4) =
+      *reinterpret_cast<const uint2*>(v_pool + off);
+}
+
+}  // namespace
+
+cudaError_t launch_reference(const RunArgs& a, int num_workers, cudaStream_t s) {
+  ref_attention_kernel<<<num_workers, 128, 0, s>>>(a);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_merge_units(const MergeArgs& a, int num_units, cudaStream_t s) {
+  if (num_units == 0) return cudaSuccess;
+  merge_units_kernel<<<num_units, 128, 0, s>>>(a);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_merge_plain(const float* o_part, const float* lse_part, int num_splits,
+                               int64_t rows, uint16_t* o, float* lse, cudaStream_t s) {
+  if (rows == 0) return cudaSuccess;
+  const unsigned blocks = static_cast<unsigned>((rows + 3) / 4);
+  merge_plain_kernel<<<blocks, 128, 0, s>>>(o_part, lse_part, num_splits, rows, o, lse);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_gather(const uint16_t* k_pool, const uint16_t* v_pool, int64_t page_stride,
+                          int64_t head_stride, int64_t token_stride, const int32_t* bt,
+                          int page_size, int page_shift, int kv_head, int L, uint16_t* out_k,
+                          uint16_t* out_v, cudaStream_t s) {
+  if (L == 0) return cudaSuccess;
+  gather_kernel<<<(L + 3) / 4, 128, 0, s>>>(k_pool, v_pool, page_stride, head_stride, token_stride,
+                                            bt, page_size, page_shift, kv_head, L, out_k, out_v);
+  return cudaGetLastError();
+}
+
+}  // namespace xy

@@ -1,0 +1,277 @@
+// Host planner: Token-Table -> decomposition -> Task-Table (Sections 3.2.1 and 3.3.1).
+//
+// a1  Token-Table: per request {kind, start position = prefix sum of q_len, tokenNum,
+//     historical kvLen}; verify requests get their ancestor-or-self bit matrix.
+// a2  Decomposition: request -> q tiles -> one tile unit per kv head.  Rows of a unit are
+//     GQA-packed (token-major, the G q heads of the kv head innermost).  The unit's visible
+//     keys are cut into runs of 128-key tiles (KV splits) when a unit is too heavy for one
+//     worker.  Purely logical: no data moves.
+// a3  Reordering: cost per task, sort from largest to smallest, deal to the workers in the
+//     symmetric round-robin 0..C-1, C-1..0, ...; each worker's list is stored contiguously.
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <numeric>
+
+#include "xy_internal.h"
+
+namespace xy {
+namespace {
+
+// Per-SM time model in microseconds (free design constants; parity does not depend on them).
+constexpr float kDenseVisitUs = 0.92f;   // one 128-row sub-tile against 128 keys on the tensor pipe
+constexpr float kStreamVisitUs = 1.50f;  // 64 KiB of K+V at an even share of HBM bandwidth
+constexpr float kTaskFixedUs = 1.5f;     // Q load, pipeline fill, epilogue
+constexpr int kMinChunkTiles = 4;
+
+struct Unit {
+  int32_t req, kv_head, tok0, ntok, kind;
+  int32_t nkt;       // visible 128-key tiles
+  float visit_cost;  // per kv tile
+  float paper_load;  // rows x visible keys
+};
+
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+}  // namespace
+
+int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_capacity,
+               const xy_attn_request* reqs, int32_t num_reqs, const int32_t* tree_parents,
+               int32_t num_parents, PlanResult* out, std::string* err) {
+  *out = PlanResult();
+  char buf[256];
+  auto fail = [&](int code, const char* msg) {
+    *err = msg;
+    return code;
+  };
+  if (num_reqs < 0 || (num_reqs > 0 && reqs == nullptr)) return fail(XY_ERR_INVALID_ARG, "reqs is null");
+  if (num_reqs > cfg.max_requests) return fail(XY_ERR_CAPACITY, "num_reqs exceeds max_requests");
+  if (num_parents < 0) return fail(XY_ERR_INVALID_ARG, "num_parents < 0");
+  const int G = cfg.num_q_heads / cfg.num_kv_heads;
+  const int B = cfg.page_size;
+
+  // ---- a1: Token-Table ------------------------------------------------------------------
+  out->reqs.resize(num_reqs);
+  out->q_start.assign(num_reqs + 1, 0);
+  int64_t total_q = 0;
+  int64_t pairs = 0, kv_tokens = 0;
+  for (int r = 0; r < num_reqs; ++r) {
+    const xy_attn_request& q = reqs[r];
+    if (q.q_len < 1) {
+      snprintf(buf, sizeof buf, "request %d: q_len must be >= 1", r);
+      return fail(XY_ERR_INVALID_ARG, buf);
+    }
+    if (q.kv_len < 0) {
+      snprintf(buf, sizeof buf, "request %d: kv_len must be >= 0", r);
+      return fail(XY_ERR_INVALID_ARG, buf);
+    }
+    if (q.mask_kind != XY_MASK_CAUSAL && q.mask_kind != XY_MASK_TREE) {
+      snprintf(buf, sizeof buf, "request %d: unknown mask_kind", r);
+      return fail(XY_ERR_INVALID_ARG, buf);
+    }
+    const int64_t L = static_cast<int64_t>(q.q_len) + q.kv_len;
+    if (L > static_cast<int64_t>(cfg.max_pages_per_req) * B) {
+      snprintf(buf, sizeof buf, "request %d: kv_len+q_len exceeds max_pages_per_req pages", r);
+      return fail(XY_ERR_CAPACITY, buf);
+    }
+    total_q += q.q_len;
+    if (total_q > cfg.max_q_tokens) return fail(XY_ERR_CAPACITY, "total q tokens exceed max_q_tokens");
+    ReqInfo& ri = out->reqs[r];
+    ri.q_start = static_cast<int32_t>(total_q - q.q_len);
+    ri.q_len = q.q_len;
+    ri.kv_len = q.kv_len;
+    ri.mask_kind = q.mask_kind;
+    ri.tree_off = 0;
+    ri.tree_words = 0;
+    ri.pad0 = ri.pad1 = 0;
+    out->q_start[r + 1] = static_cast<int32_t>(total_q);
+    kv_tokens += L;
+    const int64_t n = q.q_len, h = q.kv_len;
+    if (q.mask_kind == XY_MASK_TREE) {
+      if (q.q_len > cfg.max_tree_nodes) {
+        snprintf(buf, sizeof buf, "request %d: tree has more than max_tree_nodes nodes", r);
+        return fail(XY_ERR_CAPACITY, buf);
+      }
+      if (tree_parents == nullptr || q.parent_off < 0 ||
+          static_cast<int64_t>(q.parent_off) + q.q_len > num_parents) {
+        snprintf(buf, sizeof buf, "request %d: parent_off/q_len outside tree_parents", r);
+        return fail(XY_ERR_BAD_TREE, buf);
+      }
+      const int32_t* par = tree_parents + q.parent_off;
+      const int words = ceil_div(q.q_len, 64);
+      ri.tree_off = static_cast<int32_t>(out->tree_mask.size());
+      ri.tree_words = words;
+      out->tree_mask.resize(out->tree_mask.size() + static_cast<size_t>(words) * q.q_len, 0ull);
+      uint64_t* base = out->tree_mask.data() + ri.tree_off;
+      pairs += n * h;
+      for (int i = 0; i < q.q_len; ++i) {
+        if (par[i] < -1 || par[i] >= i) {
+          snprintf(buf, sizeof buf, "request %d: parent[%d] = %d not in {-1} U [0, %d]", r, i,
+                   par[i], i - 1);
+          out->tree_mask.clear();
+          return fail(XY_ERR_BAD_TREE, buf);
+        }
+        uint64_t* row = base + static_cast<size_t>(i) * words;
+        if (par[i] >= 0) {  // ancestors of the parent are already complete (topological order)
+          const uint64_t* prow = base + static_cast<size_t>(par[i]) * words;
+          for (int w = 0; w < words; ++w) row[w] = prow[w];
+        }
+        row[i / 64] |= 1ull << (i % 64);
+        int depth = 0;
+        for (int w = 0; w < words; ++w) depth += __builtin_popcountll(row[w]);
+        pairs += depth;
+      }
+    } else {
+      pairs += n * h + n * (n + 1) / 2;
+    }
+  }
+  out->total_q = total_q;
+
+  // ---- a2: decomposition ----------------------------------------------------------------
+  const bool paper = cfg.plan_mode == XY_PLAN_PAPER;
+  const int sub_tok = std::max(1, 128 / G);  // tokens of one 128-row sub-tile
+  const int dense_tok = paper ? (cfg.tile_tokens > 0 ? cfg.tile_tokens : sub_tok) : 2 * sub_tok;
+  std::vector<Unit> units;
+  for (int r = 0; r < num_reqs; ++r) {
+    const int n = reqs[r].q_len, h = reqs[r].kv_len;
+    // q tiles of this request (same for every kv head)
+    std::vector<std::pair<int, int>> tiles;  // tok0, ntok
+    if (paper) {
+      for (int t0 = 0; t0 < n; t0 += dense_tok) tiles.push_back({t0, std::min(dense_tok, n - t0)});
+    } else if (n * G <= kStreamRowsMax) {
+      tiles.push_back({0, n});
+    } else {
+      for (int t0 = 0; t0 < n; t0 += dense_tok) tiles.push_back({t0, std::min(dense_tok, n - t0)});
+    }
+    for (int g = 0; g < cfg.num_kv_heads; ++g) {
+      for (auto& t : tiles) {
+        Unit u;
+        u.req = r;
+        u.kv_head = g;
+        u.tok0 = t.first;
+        u.ntok = t.second;
+        const int rows = u.ntok * G;
+        u.kind = rows <= kStreamRowsMax ? 1 : 0;
+        const int visible = h + u.tok0 + u.ntok;
+        u.nkt = ceil_div(visible, kKeyTile);
+        if (u.kind == 1) {
+          u.visit_cost = kStreamVisitUs;
+        } else {
+          const int subtiles = ceil_div(rows, 128);
+          const float bytes_us = kStreamVisitUs / static_cast<float>(tiles.size());
+          u.visit_cost = std::max(kDenseVisitUs * subtiles, bytes_us);
+        }
+        u.paper_load = static_cast<float>(rows) * static_cast<float>(visible);
+        units.push_back(u);
+      }
+    }
+  }
+
+  // KV splits: cap the cost of one task at a fraction of the mean per-worker load.
+  const int max_splits = cfg.max_splits > 0 ? cfg.max_splits : 32;
+  double total_cost = 0.0;
+  for (const Unit& u : units) total_cost += kTaskFixedUs + u.visit_cost * u.nkt;
+  float cap = static_cast<float>(total_cost / std::max(1, num_workers) / 4.0);
+  std::vector<int> chunk_tiles(units.size(), 0);
+  for (int attempt = 0; attempt < 64; ++attempt) {
+    int64_t prow = 0;
+    for (size_t k = 0; k < units.size(); ++k) {
+      const Unit& u = units[k];
+      int nsplit = 1;
+      if (!paper) {
+        const float cost = u.visit_cost * u.nkt;
+        nsplit = static_cast<int>(std::ceil(cost / std::max(cap, 1e-3f)));
+        nsplit = std::min(nsplit, max_splits);
+        nsplit = std::min(nsplit, std::max(1, u.nkt / kMinChunkTiles));
+        nsplit = std::max(nsplit, 1);
+      }
+      int chunk = ceil_div(std::max(u.nkt, 1), nsplit);
+      nsplit = ceil_div(std::max(u.nkt, 1), chunk);
+      chunk_tiles[k] = chunk;
+      if (nsplit > 1) prow += static_cast<int64_t>(nsplit) * u.ntok * G;
+    }
+    if (prow <= partial_row_capacity) break;
+    cap *= 1.5f;  // fewer splits until the partials fit the workspace
+    if (attempt == 63) return fail(XY_ERR_CAPACITY, "split-KV workspace too small");
+  }
+
+  struct Pending {
+    xy_attn_task t;
+    float cost;
+  };
+  std::vector<Pending> pend;
+  int64_t prow = 0;
+  for (size_t k = 0; k < units.size(); ++k) {
+    const Unit& u = units[k];
+    const int chunk = chunk_tiles[k];
+    const int nsplit = ceil_div(std::max(u.nkt, 1), chunk);
+    const int rows = u.ntok * G;
+    if (nsplit > 1) {
+      xy_attn_merge_unit mu{u.req, u.kv_head, u.tok0, u.ntok, static_cast<int32_t>(prow), nsplit};
+      out->merges.push_back(mu);
+    }
+    for (int c = 0; c < nsplit; ++c) {
+      Pending p;
+      p.t.req = u.req;
+      p.t.kv_head = u.kv_head;
+      p.t.tok0 = u.tok0;
+      p.t.ntok = u.ntok;
+      p.t.kt_lo = c * chunk;
+      p.t.kt_hi = std::min(u.nkt, (c + 1) * chunk);
+      p.t.part = nsplit > 1 ? static_cast<int32_t>(prow + static_cast<int64_t>(c) * rows) : -1;
+      p.t.kind = u.kind;
+      p.cost = paper ? u.paper_load : kTaskFixedUs + u.visit_cost * (p.t.kt_hi - p.t.kt_lo);
+      pend.push_back(p);
+    }
+    if (nsplit > 1) prow += static_cast<int64_t>(nsplit) * rows;
+  }
+  out->partial_rows = prow;
+
+  // ---- a3: reordering -> Task-Table ------------------------------------------------------
+  std::vector<int> order(pend.size());
+  std::iota(order.begin(), order.end(), 0);
+  std::stable_sort(order.begin(), order.end(),
+                   [&](int a, int b) { return pend[a].cost > pend[b].cost; });
+  const int C = std::max(1, num_workers);
+  std::vector<std::vector<int>> lists(C);
+  for (size_t pos = 0; pos < order.size(); ++pos) {
+    const size_t lap = pos / C, idx = pos % C;
+    const size_t w = (lap % 2 == 0) ? idx : C - 1 - idx;
+    lists[w].push_back(order[pos]);
+  }
+  out->worker_off.assign(C + 1, 0);
+  out->tasks.reserve(pend.size());
+  out->task_cost.reserve(pend.size());
+  float lmin = 0.f, lmax = 0.f, lsum = 0.f, tmax = 0.f;
+  int ndense = 0;
+  for (int w = 0; w < C; ++w) {
+    float load = 0.f;
+    for (int id : lists[w]) {
+      out->tasks.push_back(pend[id].t);
+      out->task_cost.push_back(pend[id].cost);
+      load += pend[id].cost;
+      tmax = std::max(tmax, pend[id].cost);
+      ndense += pend[id].t.kind == 0;
+    }
+    out->worker_off[w + 1] = static_cast<int32_t>(out->tasks.size());
+    lmin = (w == 0) ? load : std::min(lmin, load);
+    lmax = std::max(lmax, load);
+    lsum += load;
+  }
+
+  xy_attn_plan_info& info = out->info;
+  info.num_tasks = static_cast<int32_t>(out->tasks.size());
+  info.num_dense_tasks = ndense;
+  info.num_merge_units = static_cast<int32_t>(out->merges.size());
+  info.num_workers = C;
+  info.useful_flops = 4ll * kHeadDim * cfg.num_q_heads * pairs;
+  info.kv_bytes = 2ll * kv_tokens * cfg.num_kv_heads * kHeadDim * 2;
+  info.partial_rows = prow;
+  info.load_min = lmin;
+  info.load_mean = lsum / C;
+  info.load_max = lmax;
+  info.max_task_cost = tmax;
+  return XY_OK;
+}
+
+}  // namespace xy

@@ -1,0 +1,69 @@
+// Internal declarations shared by the planner, the API layer and the kernels.
+#pragma once
+
+#include <cstdint>
+#include <string>
+#include <vector>
+
+#include "xy_attn.h"
+
+namespace xy {
+
+constexpr int kHeadDim = 128;
+constexpr int kKeyTile = 128;      // keys per KV tile (one MMA N extent)
+constexpr int kStreamRowsMax = 16; // packed rows a streaming task may hold
+
+// Per-request facts the kernels need (device-visible, 32 bytes).
+struct ReqInfo {
+  int32_t q_start;    // start position: first row of the request in Q / O / LSE
+  int32_t q_len;      // tokenNum
+  int32_t kv_len;     // historical kvLen
+  int32_t mask_kind;  // XY_MASK_*
+  int32_t tree_off;   // first 64-bit word of the request's corner mask
+  int32_t tree_words; // words per corner-mask row
+  int32_t pad0, pad1;
+};
+
+struct PlanResult {
+  std::vector<ReqInfo> reqs;
+  std::vector<int32_t> q_start;            // num_reqs + 1
+  std::vector<uint64_t> tree_mask;         // all verify requests back to back
+  std::vector<xy_attn_task> tasks;         // grouped by worker
+  std::vector<float> task_cost;            // parallel to tasks
+  std::vector<int32_t> worker_off;         // num_workers + 1
+  std::vector<xy_attn_merge_unit> merges;
+  int64_t partial_rows = 0;
+  int64_t total_q = 0;
+  xy_attn_plan_info info{};
+};
+
+// Host-only planning.  Returns XY_OK or an error code and fills `err`.
+int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_capacity,
+               const xy_attn_request* reqs, int32_t num_reqs, const int32_t* tree_parents,
+               int32_t num_parents, PlanResult* out, std::string* err);
+
+// Arguments every attention kernel takes.
+struct RunArgs {
+  const uint16_t* q;
+  int64_t q_token_stride;
+  const uint16_t* k_pool;
+  const uint16_t* v_pool;
+  int64_t page_stride, head_stride, token_stride;
+  const int32_t* block_table;
+  int32_t bt_stride;
+  const uint64_t* tree_mask;
+  float sm_scale;
+  uint16_t* o;
+  int64_t o_token_stride;
+  float* lse;
+  // context-owned
+  const ReqInfo* reqs;
+  const xy_attn_task* tasks;
+  const int32_t* worker_off;
+  float* o_part;
+  float* lse_part;
+  int32_t* status;
+  int32_t num_q_heads, num_kv_heads, page_size, page_shift;
+};
+
+}  // namespace xy

@@ -1,0 +1,30 @@
+// Kernel launch entry points (host side) and their argument blocks.
+#pragma once
+
+#include <cuda_runtime.h>
+
+#include "xy_internal.h"
+
+namespace xy {
+
+struct MergeArgs {
+  const xy_attn_merge_unit* units;
+  const ReqInfo* reqs;
+  const float* o_part;
+  const float* lse_part;
+  uint16_t* o;
+  int64_t o_token_stride;
+  float* lse;
+  int32_t num_q_heads, num_kv_heads;
+};
+
+cudaError_t launch_reference(const RunArgs& a, int num_workers, cudaStream_t s);
+cudaError_t launch_merge_units(const MergeArgs& a, int num_units, cudaStream_t s);
+cudaError_t launch_merge_plain(const float* o_part, const float* lse_part, int num_splits,
+                               int64_t rows, uint16_t* o, float* lse, cudaStream_t s);
+cudaError_t launch_gather(const uint16_t* k_pool, const uint16_t* v_pool, int64_t page_stride,
+                          int64_t head_stride, int64_t token_stride, const int32_t* bt,
+                          int page_size, int page_shift, int kv_head, int L, uint16_t* out_k,
+                          uint16_t* out_v, cudaStream_t s);
+
+}  // namespace xy

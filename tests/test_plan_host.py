@@ -1,0 +1,225 @@
+"""Host logic of the C-ABI library (no GPU): symbol export, validation and error codes,
+Token-Table / decomposition / Task-Table invariants, and the paper-mode table against the
+pure-Python restatement in oracle/task_table.py and the paper's worked example."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import task_table as TT
+from paper_2412_18106_b200 import binding as xb
+from paper_2412_18106_b200 import workloads as W
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def host_ctx(hq, hkv, page, **kw):
+    kw.setdefault("device", -1)
+    kw.setdefault("max_q_tokens", 1 << 16)
+    kw.setdefault("max_pages_per_req", 4096)
+    return xb.XYAttn(hq, hkv, page, **kw)
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "xy_attn.h")).read()
+    declared = set(re.findall(r"\b(xy_attn_[a-z_]+)\s*\(", header))
+    assert declared == set(xb.EXPORTS)
+    lib = ctypes.CDLL(xb.LIB_PATH)
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+def test_struct_sizes_match_header():
+    assert ctypes.sizeof(xb.xy_attn_task) == 32
+    assert ctypes.sizeof(xb.xy_attn_request) == 16
+    assert ctypes.sizeof(xb.xy_attn_merge_unit) == 24
+    assert ctypes.sizeof(xb.xy_attn_config) == 14 * 4 + 8
+
+
+def test_create_rejects_bad_configs():
+    with pytest.raises(xb.XYAttnError) as e:
+        host_ctx(8, 2, 16, head_dim=64)
+    assert e.value.code == xb.XY_ERR_UNSUPPORTED
+    with pytest.raises(xb.XYAttnError) as e:
+        host_ctx(8, 2, 24)
+    assert e.value.code == xb.XY_ERR_UNSUPPORTED
+    with pytest.raises(xb.XYAttnError) as e:
+        host_ctx(8, 3, 16)
+    assert e.value.code == xb.XY_ERR_INVALID_ARG
+
+
+def test_plan_error_codes():
+    c = host_ctx(8, 2, 16, max_requests=4, max_q_tokens=100, max_pages_per_req=8, max_tree_nodes=4)
+    def code(*a):
+        with pytest.raises(xb.XYAttnError) as e:
+            c.plan(*a)
+        return e.value.code
+    assert code([0], [5], [0], [-1]) == xb.XY_ERR_INVALID_ARG        # q_len < 1
+    assert code([1], [-1], [0], [-1]) == xb.XY_ERR_INVALID_ARG       # kv_len < 0
+    assert code([1], [1], [7], [-1]) == xb.XY_ERR_INVALID_ARG        # mask kind
+    assert code([1] * 5, [1] * 5, [0] * 5, [-1] * 5) == xb.XY_ERR_CAPACITY  # requests
+    assert code([101], [0], [0], [-1]) == xb.XY_ERR_CAPACITY         # q tokens
+    assert code([1], [128], [0], [-1]) == xb.XY_ERR_CAPACITY         # pages per request
+    assert code([5], [0], [1], [0], [-1, 0, 1, 2, 3]) == xb.XY_ERR_CAPACITY  # tree nodes
+    assert code([3], [0], [1], [0], [-1, 1, 0]) == xb.XY_ERR_BAD_TREE   # parent >= index
+    assert code([3], [0], [1], [0], [-1, -2, 0]) == xb.XY_ERR_BAD_TREE  # parent < -1
+    assert code([3], [0], [1], [1], [-1, 0, 0]) == xb.XY_ERR_BAD_TREE   # parents array too short
+    assert code([3], [0], [1], [0], None) == xb.XY_ERR_BAD_TREE
+    # a failed plan discards the previous one
+    c.plan([2], [3], [0], [-1])
+    assert len(c.get_tasks()) > 0
+    code([0], [5], [0], [-1])
+    with pytest.raises(xb.XYAttnError) as e:
+        c.get_tasks()
+    assert e.value.code == xb.XY_ERR_NOT_PLANNED
+    # zero requests is valid
+    info = c.plan([], [], [], [])
+    assert info.num_tasks == 0
+    # host-only context cannot run
+    rc = c.lib.xy_attn_run(c._ctx, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 1.0, 0, 0, 0, 0)
+    assert rc == xb.XY_ERR_UNSUPPORTED
+
+
+def test_tree_mask_is_ancestor_or_self():
+    rng = np.random.default_rng(3)
+    trees = [W.random_tree(rng, n, 8) for n in (1, 5, 63, 64, 65, 130)]
+    trees.append(np.array([-1, -1, 0, 1, -1], dtype=np.int32))  # several roots
+    c = host_ctx(8, 2, 16, max_tree_nodes=256)
+    parents = np.concatenate(trees)
+    off = np.cumsum([0] + [len(t) for t in trees[:-1]])
+    c.plan([len(t) for t in trees], [7] * len(trees), [1] * len(trees), off, parents)
+    words = c.get_tree_mask()
+    pos = 0
+    for t in trees:
+        n = len(t)
+        W64 = (n + 63) // 64
+        for i in range(n):
+            anc = set()
+            node = i
+            while node >= 0:
+                anc.add(node)
+                node = int(t[node])
+            row = words[pos + i * W64 : pos + (i + 1) * W64]
+            got = {j for j in range(n) if (int(row[j // 64]) >> (j % 64)) & 1}
+            assert got == anc
+            assert all(int(row[j // 64]) >> (j % 64) == 0 for j in [n - 1 + 1] if j % 64)  # no bits beyond n
+        pos += n * W64
+    assert pos == len(words)
+
+
+def coverage_check(batch, ctx, info):
+    """Every (request, kv head, new token, visible 128-key tile) is covered exactly once;
+    no tile above a token's causal frontier is needed; workers partition the tasks."""
+    tasks = ctx.get_tasks()
+    off = ctx.get_worker_offsets()
+    assert off[0] == 0 and off[-1] == len(tasks) and np.all(np.diff(off) >= 0)
+    assert len(off) == info.num_workers + 1
+    G = batch.num_q_heads // batch.num_kv_heads
+    merges = ctx.get_merge_units()
+    for r in range(batch.num_requests):
+        n, h = int(batch.q_len[r]), int(batch.kv_len[r])
+        for g in range(batch.num_kv_heads):
+            sel = tasks[(tasks["req"] == r) & (tasks["kv_head"] == g)]
+            need = [-(-(h + i + 1) // 128) for i in range(n)]  # tiles row i needs
+            cover = [np.zeros(need[i], dtype=np.int32) for i in range(n)]
+            for t in sel:
+                assert t["ntok"] >= 1 and t["tok0"] >= 0 and t["tok0"] + t["ntok"] <= n
+                assert 0 <= t["kt_lo"] < t["kt_hi"]
+                # the run never goes beyond what the tile's last row can see
+                assert t["kt_hi"] <= -(-(h + t["tok0"] + t["ntok"]) // 128)
+                assert t["kind"] == (1 if t["ntok"] * G <= 16 else 0)
+                for i in range(t["tok0"], t["tok0"] + t["ntok"]):
+                    hi = min(t["kt_hi"], need[i])
+                    if hi > t["kt_lo"]:
+                        cover[i][t["kt_lo"] : hi] += 1
+            for i in range(n):
+                assert np.all(cover[i] == 1), (r, g, i)
+    # split bookkeeping: partial rows are disjoint and every split unit has a merge entry
+    used = np.zeros(max(int(info.partial_rows), 1), dtype=np.int32)
+    for t in tasks[tasks["part"] >= 0]:
+        rows = t["ntok"] * G
+        used[t["part"] : t["part"] + rows] += 1
+    assert np.all(used[: info.partial_rows] == 1)
+    for m in merges:
+        rows = m["ntok"] * G
+        sel = tasks[(tasks["req"] == m["req"]) & (tasks["kv_head"] == m["kv_head"]) & (tasks["tok0"] == m["tok0"])]
+        assert len(sel) == m["nsplit"] >= 2
+        assert sorted(sel["part"]) == [m["part0"] + c * rows for c in range(m["nsplit"])]
+        # chunks tile the visible range without gaps
+        order = np.argsort(sel["kt_lo"])
+        assert sel["kt_lo"][order][0] == 0
+        assert np.all(sel["kt_lo"][order][1:] == sel["kt_hi"][order][:-1])
+    unsplit = tasks[tasks["part"] < 0]
+    keys = {(t["req"], t["kv_head"], t["tok0"]) for t in unsplit}
+    assert len(keys) == len(unsplit)
+    assert info.num_tasks == len(tasks) and info.num_merge_units == len(merges)
+
+
+@pytest.mark.parametrize("name", ["tiny_hybrid", "decode_only", "splitfuse_mix", "verify_trees", "full_mix"])
+def test_balanced_plan_invariants_on_configs(name):
+    b = W.CONFIGS[name]()
+    c = host_ctx(b.num_q_heads, b.num_kv_heads, b.page_size)
+    info = c.plan_batch(b)
+    coverage_check(b, c, info)
+    assert info.useful_flops == W.useful_flops(b)
+    assert info.kv_bytes == W.kv_bytes(b)
+    # balance: snake dealing of a sorted list keeps every worker within one task of the mean
+    if info.num_tasks >= 4 * info.num_workers:
+        assert info.load_max <= info.load_mean + info.max_task_cost + 1e-3
+    # determinism
+    t1 = c.get_tasks().copy()
+    c.plan_batch(b)
+    assert np.array_equal(t1, c.get_tasks())
+
+
+def test_plan_edge_shapes():
+    reqs = [(n, h, 0, None) for n in (1, 15, 16, 17, 127, 128, 129) for h in (0, 5, 128, 200)]
+    b = W.custom("edges", 8, 2, 16, reqs, seed=1)
+    for workers in (1, 3, 148):
+        c = host_ctx(8, 2, 16, num_workers=workers)
+        coverage_check(b, c, c.plan_batch(b))
+    c = host_ctx(8, 2, 16, num_workers=8, workspace_bytes=(128 + 1) * 4 * 64)  # tiny workspace
+    info = c.plan_batch(b)
+    assert info.partial_rows <= 64
+    coverage_check(b, c, info)
+
+
+def test_splits_appear_for_long_decode_and_respect_max_splits():
+    b = W.custom("long", 8, 1, 128, [(1, 60000, 0, None)], seed=2)
+    c = host_ctx(8, 1, 128, max_splits=5)
+    info = c.plan_batch(b)
+    assert 2 <= info.num_tasks <= 5 and info.num_merge_units == 1
+    coverage_check(b, c, info)
+
+
+def test_paper_mode_equals_python_task_table_and_fig3b():
+    q_len, kv_len = [300, 1, 16, 1], [0, 700, 900, 350]
+    hq, hkv, C, tile = 6, 6, 4, 128
+    c = host_ctx(hq, hkv, 16, plan_mode=xb.XY_PLAN_PAPER, tile_tokens=tile, num_workers=C)
+    info = c.plan(q_len, kv_len, [0, 0, 1, 0], [-1, -1, 0, -1], W.chain_tree(16))
+    tasks, off = c.get_tasks(), c.get_worker_offsets()
+    assert info.num_merge_units == 0 and np.all(tasks["part"] == -1)
+    # Fig. 3(b): 3 + 1 + 1 + 1 tile blocks, times headNum units
+    assert len(tasks) == 6 * hkv
+    blocks = [len(set(tasks[tasks["req"] == r]["tok0"])) for r in range(4)]
+    assert blocks == [3, 1, 1, 1]
+    want = TT.reorder(TT.decompose(TT.token_table(q_len, kv_len, tile), hkv), C)
+    for w in range(C):
+        got = [(int(t["req"]), int(t["kv_head"]), int(t["tok0"]), int(t["ntok"])) for t in tasks[off[w] : off[w + 1]]]
+        exp = [(u.stage_id, u.head, u.row0, u.rows) for u in want[w]]
+        assert got == exp
+    # the first eight tiles of the sorted list went to workers 0,1,2,3,3,2,1,0
+    units = TT.decompose(TT.token_table(q_len, kv_len, tile), hkv)
+    order = sorted(range(len(units)), key=lambda k: -units[k].load)
+    first8 = [units[k] for k in order[:8]]
+    owners = []
+    for u in first8:
+        for w in range(C):
+            if any((int(t["req"]), int(t["kv_head"]), int(t["tok0"])) == (u.stage_id, u.head, u.row0)
+                   for t in tasks[off[w] : off[w + 1]]):
+                owners.append(w)
+    assert owners == [0, 1, 2, 3, 3, 2, 1, 0]
+    coverage_check(W.custom("fig3b", hq, hkv, 16, [(300, 0, 0, None), (1, 700, 0, None),
+                                                   (16, 900, 1, W.chain_tree(16)), (1, 350, 0, None)]), c, info)
