@@ -120,7 +120,7 @@ int xy_attn_create(const xy_attn_config* cfg, xy_attn_ctx** out) {
   const int sub_tok = 128 / G > 0 ? 128 / G : 1;
   const int tile_tok = cfg->plan_mode == XY_PLAN_PAPER
                            ? (cfg->tile_tokens > 0 ? cfg->tile_tokens : sub_tok)
-                           : 2 * sub_tok;
+                           : dense_subtiles(*cfg) * sub_tok;
   const int64_t units_max = static_cast<int64_t>(cfg->num_kv_heads) *
                             (cfg->max_requests + cfg->max_q_tokens / tile_tok + 1);
   c->cap_tasks = 2 * units_max + 4ll * c->num_workers + 16;
@@ -273,7 +273,11 @@ int xy_attn_run(xy_attn_ctx* ctx, const void* q, int64_t q_token_stride, const v
     XY_CUDA(ctx, cudaEventRecord(ctx->events[3 * ctx->timed_runs], s));
   }
 
-  XY_CUDA(ctx, launch_reference(a, ctx->num_workers, s));
+  if (cfg.kernel == XY_KERNEL_REFERENCE) {
+    XY_CUDA(ctx, launch_reference(a, ctx->num_workers, s));
+  } else {
+    XY_CUDA(ctx, launch_meta(a, ctx->num_workers, num_pages, s));
+  }
   ctx->last_launches += 1;
   if (timed) XY_CUDA(ctx, cudaEventRecord(ctx->events[3 * ctx->timed_runs + 1], s));
 

@@ -1,0 +1,538 @@
+// Hybrid-batch attention meta-kernel (Meta-Attention, Sections 4.1-4.2), sm_100a.
+//
+// One persistent CTA per worker walks its Task-Table list (Section 3.3.1).  Warp roles:
+//   warps 0..7  consumers: load the packed Q tile, compute QK -> softmax -> PV, write O / LSE
+//   warp  8     producer: looks page ids up in the block table and stages 128-key K and V
+//               tiles (one TMA box per page and 64-element half) into a ring of shared-memory
+//               stages; it runs ahead across task boundaries
+// Shared-memory tiles use the 128-byte TMA swizzle: element (row, d) of a tile lives at
+//   (d / 64) * 16 KiB + row * 128 B + (((d % 64) / 8) ^ (row % 8)) * 16 B + (d % 8) * 2 B,
+// which both ldmatrix and the tcgen05 shared-memory descriptors read without bank conflicts.
+//
+// Two task kinds share the ring:
+//   dense     (rows > 16): each consumer warp owns 16 packed rows against all 128 keys of a tile
+//   streaming (rows <= 16: decode, tiny verify): each consumer warp owns 16 keys of every tile
+//             against all rows; the warps' partial (m, l, O) are merged in shared memory at
+//             the end of the task.  HBM-bound: the tensor work is a 16-row warp-level MMA.
+// Online softmax runs in the log2 domain in fp32 registers with quad shuffles; P is rounded
+// to bf16 before P.V; masked scores are selected to -inf, never added.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "ptx.cuh"
+#include "xy_kernels.h"
+
+namespace xy {
+
+namespace {
+
+using namespace ptx;
+
+constexpr int kConsumerWarps = 8;
+constexpr int kConsumerThreads = kConsumerWarps * 32;
+constexpr int kThreads = kConsumerThreads + 128;  // + one warpgroup: producer, MMA issuer, 2 idle
+constexpr int kRegsConsumer = 232;               // setmaxnreg budgets: 256 x 232 + 128 x 40 <= 64 Ki
+constexpr int kRegsOther = 40;
+constexpr int kStages = 4;
+constexpr int kTileBytes = 32768;  // 2 halves x 128 rows x 128 B
+constexpr int kHalfBytes = 16384;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+struct __align__(8) SmemBarriers {
+  uint64_t full[kStages];
+  uint64_t empty[kStages];
+};
+
+constexpr int kSmemQ = 2 * kTileBytes;
+constexpr int kSmemRing = kStages * kTileBytes;
+constexpr int kSmemMl = kConsumerWarps * 16 * 2 * 4;
+constexpr int kSmemTotal = 1024 /*align slack*/ + kSmemQ + kSmemRing + kSmemMl + sizeof(SmemBarriers);
+
+__device__ __forceinline__ uint32_t swz(uint32_t row, uint32_t chunk16 /*0..15*/) {
+  return (chunk16 >> 3) * kHalfBytes + row * 128u + (((chunk16 & 7u) ^ (row & 7u)) << 4);
+}
+
+struct Pipe {
+  int stage;
+  uint32_t phase;
+  __device__ __forceinline__ void advance() {
+    if (++stage == kStages) {
+      stage = 0;
+      phase ^= 1u;
+    }
+  }
+};
+
+struct MetaParams {
+  RunArgs a;
+};
+
+// Visibility of key column `col` for new token i (Sections 4.1.2, 4.2.2, 5.2).
+__device__ __forceinline__ bool visible(const RunArgs& a, const ReqInfo& rq, int i, int col) {
+  if (col > rq.kv_len + i) return false;  // causal frontier; also excludes everything >= L
+  if (col < rq.kv_len || rq.mask_kind == XY_MASK_CAUSAL) return true;
+  const int jp = col - rq.kv_len;
+  const uint64_t w = __ldg(a.tree_mask + rq.tree_off + static_cast<int64_t>(i) * rq.tree_words + (jp >> 6));
+  return (w >> (jp & 63)) & 1ull;
+}
+
+// One consumer warp: 16 packed rows (x0 .. x0+15) against NT*8 keys (key offset koff inside
+// every 128-key tile).  Keeps m (log2 domain), l (thread-partial) and O in registers.
+// KEEPQ: Q fragments stay in registers for the whole task (streaming); otherwise they are
+// re-read from shared memory at every k-step to leave registers for the 128-key score tile.
+template <int NT, bool KEEPQ>
+struct WarpTile {
+  float o[16][4];
+  float m_lo, m_hi, l_lo, l_hi;
+  uint32_t qf[KEEPQ ? 8 : 1][4];
+  uint32_t q_addr;  // this lane's ldmatrix row address for k-step 0 (!KEEPQ)
+
+  __device__ __forceinline__ void init() {
+#pragma unroll
+    for (int n = 0; n < 16; ++n)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) o[n][e] = 0.f;
+    m_lo = m_hi = -INFINITY;
+    l_lo = l_hi = 0.f;
+  }
+
+  __device__ __forceinline__ void load_q(uint32_t q_smem, int x0, int lane) {
+    const int mi = lane >> 3;
+    const uint32_t row = x0 + (lane & 7) + (mi & 1) * 8;
+    if (KEEPQ) {
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks)
+        ldmatrix_x4(q_smem + swz(row, ks * 2 + (mi >> 1)), qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3]);
+    } else {
+      q_addr = q_smem + row * 128u;
+      q_row7 = row & 7u;
+      q_hi = mi >> 1;
+    }
+  }
+  uint32_t q_row7, q_hi;
+
+  // S = Q K^T for this warp's keys; returns scores (raw dot products) in s.
+  __device__ __forceinline__ void qk(uint32_t k_smem, int koff, int lane, float (&s)[NT][4]) {
+#pragma unroll
+    for (int n = 0; n < NT; ++n)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) s[n][e] = 0.f;
+    const int mi = lane >> 3;
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) {
+      if (!KEEPQ) {
+        const uint32_t ch = ks * 2 + q_hi;
+        ldmatrix_x4(q_addr + (ch >> 3) * kHalfBytes + (((ch & 7u) ^ q_row7) << 4), qf[0][0], qf[0][1],
+                    qf[0][2], qf[0][3]);
+      }
+      const uint32_t(&qa)[4] = qf[KEEPQ ? ks : 0];
+#pragma unroll
+      for (int np = 0; np < NT / 2; ++np) {
+        const uint32_t key = koff + np * 16 + (lane & 7) + (mi >> 1) * 8;
+        uint32_t b0, b1, b2, b3;
+        ldmatrix_x4(k_smem + swz(key, ks * 2 + (mi & 1)), b0, b1, b2, b3);
+        mma_bf16_16816(s[2 * np], qa, b0, b1);
+        mma_bf16_16816(s[2 * np + 1], qa, b2, b3);
+      }
+    }
+  }
+
+  // Mask + online softmax (Update rescale) on s; leaves P (bf16 A fragments) in p.
+  __device__ __forceinline__ void softmax(const RunArgs& a, const ReqInfo& rq, float (&s)[NT][4],
+                                          uint32_t (&p)[NT / 2][4], int col0, int i_lo, int i_hi,
+                                          bool need_mask, float scale_log2, int lane) {
+    float mx_lo = -INFINITY, mx_hi = -INFINITY;
+#pragma unroll
+    for (int n = 0; n < NT; ++n) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        float v = s[n][e] * scale_log2;
+        if (need_mask) {
+          const int col = col0 + n * 8 + 2 * (lane & 3) + (e & 1);
+          if (!visible(a, rq, (e < 2) ? i_lo : i_hi, col)) v = -INFINITY;
+        }
+        s[n][e] = v;
+        if (e < 2) mx_lo = fmaxf(mx_lo, v); else mx_hi = fmaxf(mx_hi, v);
+      }
+    }
+    mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1));
+    mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
+    mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
+    mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
+    const float mn_lo = fmaxf(m_lo, mx_lo), mn_hi = fmaxf(m_hi, mx_hi);
+    const float use_lo = (mn_lo == -INFINITY) ? 0.f : mn_lo;
+    const float use_hi = (mn_hi == -INFINITY) ? 0.f : mn_hi;
+    const float al_lo = ex2(m_lo - use_lo), al_hi = ex2(m_hi - use_hi);
+    m_lo = mn_lo;
+    m_hi = mn_hi;
+    float sum_lo = 0.f, sum_hi = 0.f;
+#pragma unroll
+    for (int n = 0; n < NT; ++n) {
+      const float p0 = ex2(s[n][0] - use_lo), p1 = ex2(s[n][1] - use_lo);
+      const float p2 = ex2(s[n][2] - use_hi), p3 = ex2(s[n][3] - use_hi);
+      sum_lo += p0 + p1;
+      sum_hi += p2 + p3;
+      // A fragment of k-step n/2: a0,a1 from the even n-tile, a2,a3 from the odd one
+      p[n >> 1][(n & 1) * 2 + 0] = pack_bf16(p0, p1);
+      p[n >> 1][(n & 1) * 2 + 1] = pack_bf16(p2, p3);
+    }
+    l_lo = l_lo * al_lo + sum_lo;
+    l_hi = l_hi * al_hi + sum_hi;
+#pragma unroll
+    for (int n = 0; n < 16; ++n) {
+      o[n][0] *= al_lo;
+      o[n][1] *= al_lo;
+      o[n][2] *= al_hi;
+      o[n][3] *= al_hi;
+    }
+  }
+
+  // O += P V for this warp's keys.
+  __device__ __forceinline__ void pv(uint32_t v_smem, int koff, int lane, const uint32_t (&p)[NT / 2][4]) {
+    const int mi = lane >> 3;
+#pragma unroll
+    for (int kk = 0; kk < NT / 2; ++kk) {
+      const uint32_t key = koff + kk * 16 + (lane & 7) + (mi & 1) * 8;
+#pragma unroll
+      for (int dp = 0; dp < 8; ++dp) {
+        uint32_t b0, b1, b2, b3;
+        ldmatrix_x4_trans(v_smem + swz(key, dp * 2 + (mi >> 1)), b0, b1, b2, b3);
+        mma_bf16_16816(o[2 * dp], p[kk], b0, b1);
+        mma_bf16_16816(o[2 * dp + 1], p[kk], b2, b3);
+      }
+    }
+  }
+
+  __device__ __forceinline__ void reduce_l() {
+    l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
+    l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
+    l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
+    l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+  }
+};
+
+struct TaskView {
+  xy_attn_task t;
+  ReqInfo rq;
+  int G, rows;
+};
+
+// Destination of packed row x: final O / LSE or the fp32 partial.
+__device__ __forceinline__ void write_row_pair(const RunArgs& a, const TaskView& tv, int x, int col,
+                                               float v0, float v1) {
+  if (tv.t.part < 0) {
+    const int i = tv.t.tok0 + x / tv.G, head = tv.t.kv_head * tv.G + x % tv.G;
+    uint32_t* dst = reinterpret_cast<uint32_t*>(
+        a.o + static_cast<int64_t>(tv.rq.q_start + i) * a.o_token_stride + head * kHeadDim + col);
+    *dst = pack_bf16(v0, v1);
+  } else {
+    float2* dst = reinterpret_cast<float2*>(a.o_part + static_cast<int64_t>(tv.t.part + x) * kHeadDim + col);
+    *dst = make_float2(v0, v1);
+  }
+}
+__device__ __forceinline__ void write_lse(const RunArgs& a, const TaskView& tv, int x, float lse) {
+  if (tv.t.part < 0) {
+    const int i = tv.t.tok0 + x / tv.G, head = tv.t.kv_head * tv.G + x % tv.G;
+    a.lse[static_cast<int64_t>(tv.rq.q_start + i) * a.num_q_heads + head] = lse;
+  } else {
+    a.lse_part[tv.t.part + x] = lse;
+  }
+}
+
+__device__ __forceinline__ void report_timeout(const RunArgs& a) {
+  atomicExch(a.status, XY_ERR_DEVICE_TIMEOUT);
+}
+
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads, 1)
+meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constant__ CUtensorMap k_map,
+                      const __grid_constant__ CUtensorMap v_map) {
+  extern __shared__ uint8_t smem_raw[];
+  const RunArgs& a = P.a;
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t q_smem = base;
+  const uint32_t ring = base + kSmemQ;
+  uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
+  float* ml = reinterpret_cast<float*>(gen_base + kSmemQ + kSmemRing);
+  SmemBarriers* bars = reinterpret_cast<SmemBarriers*>(gen_base + kSmemQ + kSmemRing + kSmemMl);
+  float* xch = reinterpret_cast<float*>(gen_base);  // streaming merge area, aliases the Q tiles
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(smem_u32(&bars->full[s]), 1);
+      mbar_init(smem_u32(&bars->empty[s]), kConsumerWarps);
+    }
+    fence_mbar_init();
+  }
+  __syncthreads();
+
+  const int t_begin = a.worker_off[blockIdx.x], t_end = a.worker_off[blockIdx.x + 1];
+  const int G = a.num_q_heads / a.num_kv_heads;
+  const float scale_log2 = a.sm_scale * kLog2e;
+
+  if (warp >= kConsumerWarps) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
+    // ================================ producer =========================================
+    if (warp == kConsumerWarps && lane == 0) {
+      prefetch_tensormap(&k_map);
+      prefetch_tensormap(&v_map);
+      Pipe pipe{0, 0};
+      bool dead = false;
+      const int ppt = kKeyTile >> a.page_shift;  // pages per 128-key tile
+      const uint32_t page_bytes = static_cast<uint32_t>(a.page_size) * 128u;
+      for (int ti = t_begin; ti < t_end && !dead; ++ti) {
+        const xy_attn_task t = a.tasks[ti];
+        const ReqInfo rq = a.reqs[t.req];
+        const int npages = (rq.kv_len + rq.q_len + a.page_size - 1) >> a.page_shift;
+        const int32_t* bt = a.block_table + static_cast<int64_t>(t.req) * a.bt_stride;
+        for (int kt = t.kt_lo; kt < t.kt_hi && !dead; ++kt) {
+          for (int op = 0; op < 2; ++op) {
+            if (!mbar_wait(smem_u32(&bars->empty[pipe.stage]), pipe.phase ^ 1u)) {
+              report_timeout(a);
+              dead = true;
+              break;
+            }
+            const uint32_t full = smem_u32(&bars->full[pipe.stage]);
+            mbar_arrive_expect_tx(full, kTileBytes);
+            const uint32_t dst = ring + pipe.stage * kTileBytes;
+            const CUtensorMap* map = op == 0 ? &k_map : &v_map;
+            for (int p = 0; p < ppt; ++p) {
+              const int pi = min(kt * ppt + p, npages - 1);  // pages past the end: reload the last
+              const int page = __ldg(bt + pi);
+              tma_load_4d(dst + p * page_bytes, map, full, 0, 0, t.kv_head, page);
+              tma_load_4d(dst + kHalfBytes + p * page_bytes, map, full, 64, 0, t.kv_head, page);
+            }
+            pipe.advance();
+          }
+        }
+      }
+    }
+  } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsConsumer));
+    // ================================ consumers ========================================
+    Pipe pipe{0, 0};
+    bool dead = false;
+    for (int ti = t_begin; ti < t_end; ++ti) {
+      TaskView tv;
+      tv.t = a.tasks[ti];
+      tv.rq = a.reqs[tv.t.req];
+      tv.G = G;
+      tv.rows = tv.t.ntok * G;
+      const int h = tv.rq.kv_len;
+      const bool tree = tv.rq.mask_kind == XY_MASK_TREE;
+      const bool stream = tv.t.kind == 1;
+
+      // ---- packed Q tile -> shared memory (rows past the tile are zero-filled)
+      {
+        const int rows_pad = stream ? 16 : 128;
+        for (int c = threadIdx.x; c < rows_pad * 16; c += kConsumerThreads) {
+          const int x = c >> 4, ch = c & 15;
+          const bool ok = x < tv.rows;
+          const int xx = ok ? x : 0;
+          const int i = tv.t.tok0 + xx / G, head = tv.t.kv_head * G + xx % G;
+          const uint16_t* src =
+              a.q + static_cast<int64_t>(tv.rq.q_start + i) * a.q_token_stride + head * kHeadDim + ch * 8;
+          cp_async_16(q_smem + swz(x, ch), src, ok);
+        }
+        cp_async_commit_wait_all();
+        named_bar_sync(1, kConsumerThreads);
+      }
+
+      if (!stream) {
+        // ---------------- dense: this warp owns rows x0 .. x0+15 -------------------------
+        const int x0 = warp * 16;
+        const bool active = x0 < tv.rows;
+        WarpTile<16, false> w;
+        w.init();
+        if (active) w.load_q(q_smem, x0, lane);
+        const int r_lo = min(x0 + (lane >> 2), tv.rows - 1), r_hi = min(x0 + (lane >> 2) + 8, tv.rows - 1);
+        const int i_lo = tv.t.tok0 + r_lo / G, i_hi = tv.t.tok0 + r_hi / G;
+        const int i_min = tv.t.tok0 + min(x0, tv.rows - 1) / G;
+        const int i_max = tv.t.tok0 + min(x0 + 15, tv.rows - 1) / G;
+        for (int kt = tv.t.kt_lo; kt < tv.t.kt_hi; ++kt) {
+          const int col0 = kt * kKeyTile;
+          const bool work = active && col0 <= h + i_max;  // mask-aware skip (Section 4.2.2)
+          float s[16][4];
+          uint32_t p[8][4];
+          if (!dead && !mbar_wait(smem_u32(&bars->full[pipe.stage]), pipe.phase)) {
+            report_timeout(a);
+            dead = true;
+          }
+          if (work) w.qk(ring + pipe.stage * kTileBytes, 0, lane, s);
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&bars->empty[pipe.stage]));
+          pipe.advance();
+          if (work) {
+            const bool need_mask = tree ? (col0 + kKeyTile > h) : (col0 + kKeyTile > h + i_min + 1);
+            w.softmax(a, tv.rq, s, p, col0, i_lo, i_hi, need_mask, scale_log2, lane);
+          }
+          if (!dead && !mbar_wait(smem_u32(&bars->full[pipe.stage]), pipe.phase)) {
+            report_timeout(a);
+            dead = true;
+          }
+          if (work) w.pv(ring + pipe.stage * kTileBytes, 0, lane, p);
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&bars->empty[pipe.stage]));
+          pipe.advance();
+        }
+        if (active) {
+          w.reduce_l();
+          const float inv_lo = w.l_lo > 0.f ? 1.f / w.l_lo : 0.f;
+          const float inv_hi = w.l_hi > 0.f ? 1.f / w.l_hi : 0.f;
+          const int xl = x0 + (lane >> 2), xh = xl + 8;
+#pragma unroll
+          for (int n = 0; n < 16; ++n) {
+            const int col = n * 8 + 2 * (lane & 3);
+            if (xl < tv.rows) write_row_pair(a, tv, xl, col, w.o[n][0] * inv_lo, w.o[n][1] * inv_lo);
+            if (xh < tv.rows) write_row_pair(a, tv, xh, col, w.o[n][2] * inv_hi, w.o[n][3] * inv_hi);
+          }
+          if ((lane & 3) == 0) {
+            if (xl < tv.rows)
+              write_lse(a, tv, xl, w.l_lo > 0.f ? (w.m_lo + log2f(w.l_lo)) * kLn2 : -INFINITY);
+            if (xh < tv.rows)
+              write_lse(a, tv, xh, w.l_hi > 0.f ? (w.m_hi + log2f(w.l_hi)) * kLn2 : -INFINITY);
+          }
+        }
+        named_bar_sync(1, kConsumerThreads);  // Q tile may be overwritten by the next task
+      } else {
+        // ---------------- streaming: this warp owns keys koff .. koff+15 of every tile ----
+        const int koff = warp * 16;
+        WarpTile<2, true> w;
+        w.init();
+        w.load_q(q_smem, 0, lane);
+        const int r_lo = min(lane >> 2, tv.rows - 1), r_hi = min((lane >> 2) + 8, tv.rows - 1);
+        const int i_lo = tv.t.tok0 + r_lo / G, i_hi = tv.t.tok0 + r_hi / G;
+        const int i_max = tv.t.tok0 + tv.t.ntok - 1;
+        for (int kt = tv.t.kt_lo; kt < tv.t.kt_hi; ++kt) {
+          const int col0 = kt * kKeyTile + koff;
+          const bool work = col0 <= h + i_max;
+          float s[2][4];
+          uint32_t p[1][4];
+          if (!dead && !mbar_wait(smem_u32(&bars->full[pipe.stage]), pipe.phase)) {
+            report_timeout(a);
+            dead = true;
+          }
+          if (work) w.qk(ring + pipe.stage * kTileBytes, koff, lane, s);
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&bars->empty[pipe.stage]));
+          pipe.advance();
+          if (work) {
+            const bool need_mask = tree ? (col0 + 16 > h) : (col0 + 16 > h + tv.t.tok0 + 1);
+            w.softmax(a, tv.rq, s, p, col0, i_lo, i_hi, need_mask, scale_log2, lane);
+          }
+          if (!dead && !mbar_wait(smem_u32(&bars->full[pipe.stage]), pipe.phase)) {
+            report_timeout(a);
+            dead = true;
+          }
+          if (work) w.pv(ring + pipe.stage * kTileBytes, koff, lane, p);
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&bars->empty[pipe.stage]));
+          pipe.advance();
+        }
+        // ---- merge the eight warps' partials (in-CTA Update stage)
+        w.reduce_l();
+        named_bar_sync(1, kConsumerThreads);  // every warp holds its Q fragments: Q smem is free
+        {
+          const int xl = lane >> 2, xh = xl + 8;
+          float* mine = xch + warp * (16 * kHeadDim);
+#pragma unroll
+          for (int n = 0; n < 16; ++n) {
+            const int col = n * 8 + 2 * (lane & 3);
+            *reinterpret_cast<float2*>(mine + xl * kHeadDim + col) = make_float2(w.o[n][0], w.o[n][1]);
+            *reinterpret_cast<float2*>(mine + xh * kHeadDim + col) = make_float2(w.o[n][2], w.o[n][3]);
+          }
+          if ((lane & 3) == 0) {
+            ml[(warp * 16 + xl) * 2 + 0] = w.m_lo;
+            ml[(warp * 16 + xl) * 2 + 1] = w.l_lo;
+            ml[(warp * 16 + xh) * 2 + 0] = w.m_hi;
+            ml[(warp * 16 + xh) * 2 + 1] = w.l_hi;
+          }
+        }
+        named_bar_sync(1, kConsumerThreads);
+        {
+          const int x = threadIdx.x >> 4, seg = threadIdx.x & 15;  // row, 8-column segment
+          if (x < tv.rows) {
+            float M = -INFINITY;
+#pragma unroll
+            for (int ww = 0; ww < kConsumerWarps; ++ww) M = fmaxf(M, ml[(ww * 16 + x) * 2]);
+            float L = 0.f, acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int ww = 0; ww < kConsumerWarps; ++ww) {
+              const float mw = ml[(ww * 16 + x) * 2], lw = ml[(ww * 16 + x) * 2 + 1];
+              if (mw == -INFINITY) continue;
+              const float f = ex2(mw - M);
+              L += f * lw;
+              const float4* src = reinterpret_cast<const float4*>(xch + ww * (16 * kHeadDim) + x * kHeadDim + seg * 8);
+              const float4 v0 = src[0], v1 = src[1];
+              acc[0] += f * v0.x; acc[1] += f * v0.y; acc[2] += f * v0.z; acc[3] += f * v0.w;
+              acc[4] += f * v1.x; acc[5] += f * v1.y; acc[6] += f * v1.z; acc[7] += f * v1.w;
+            }
+            const float inv = L > 0.f ? 1.f / L : 0.f;
+#pragma unroll
+            for (int e = 0; e < 8; e += 2)
+              write_row_pair(a, tv, x, seg * 8 + e, acc[e] * inv, acc[e + 1] * inv);
+            if (seg == 0) write_lse(a, tv, x, L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY);
+          }
+        }
+        named_bar_sync(1, kConsumerThreads);
+      }
+    }
+  }
+  __syncthreads();
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn == nullptr) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// 4-D map over a paged pool [pages, Hkv, B, D]: box = one page of one head, 64 elements wide.
+bool encode_pool_map(CUtensorMap* m, const void* pool, int64_t num_pages, int num_kv_heads, int page_size,
+                     int64_t page_stride, int64_t head_stride, int64_t token_stride) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return false;
+  cuuint64_t dims[4] = {static_cast<cuuint64_t>(kHeadDim), static_cast<cuuint64_t>(page_size),
+                        static_cast<cuuint64_t>(num_kv_heads), static_cast<cuuint64_t>(num_pages)};
+  cuuint64_t strides[3] = {static_cast<cuuint64_t>(token_stride) * 2, static_cast<cuuint64_t>(head_stride) * 2,
+                           static_cast<cuuint64_t>(page_stride) * 2};
+  cuuint32_t box[4] = {64, static_cast<cuuint32_t>(page_size), 1, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(pool), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+cudaError_t launch_meta(const RunArgs& a, int num_workers, int64_t num_pages, cudaStream_t s) {
+  cudaError_t e = cudaFuncSetAttribute(meta_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       kSmemTotal);
+  if (e != cudaSuccess) return e;
+  CUtensorMap k_map, v_map;
+  if (!encode_pool_map(&k_map, a.k_pool, num_pages, a.num_kv_heads, a.page_size, a.page_stride, a.head_stride,
+                       a.token_stride) ||
+      !encode_pool_map(&v_map, a.v_pool, num_pages, a.num_kv_heads, a.page_size, a.page_stride, a.head_stride,
+                       a.token_stride))
+    return cudaErrorInvalidValue;
+  MetaParams P{a};
+  meta_attention_kernel<<<num_workers, kThreads, kSmemTotal, s>>>(P, k_map, v_map);
+  return cudaGetLastError();
+}
+
+}  // namespace xy

@@ -130,7 +130,10 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
   // ---- a2: decomposition ----------------------------------------------------------------
   const bool paper = cfg.plan_mode == XY_PLAN_PAPER;
   const int sub_tok = std::max(1, 128 / G);  // tokens of one 128-row sub-tile
-  const int dense_tok = paper ? (cfg.tile_tokens > 0 ? cfg.tile_tokens : sub_tok) : 2 * sub_tok;
+  const int subtiles = dense_subtiles(cfg);
+  const int dense_tok = paper ? (cfg.tile_tokens > 0 ? cfg.tile_tokens : sub_tok) : subtiles * sub_tok;
+  if (paper && cfg.kernel != XY_KERNEL_REFERENCE && dense_tok * G > 128 * subtiles)
+    return fail(XY_ERR_UNSUPPORTED, "paper-mode tile_tokens x (Hq/Hkv) exceeds the rows one task may hold");
   std::vector<Unit> units;
   for (int r = 0; r < num_reqs; ++r) {
     const int n = reqs[r].q_len, h = reqs[r].kv_len;
