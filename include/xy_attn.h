@@ -152,6 +152,7 @@ int xy_attn_plan(xy_attn_ctx* ctx, const xy_attn_request* reqs /*HOST*/, int32_t
  *                element of every page a request references must be finite
  *   block_table  DEVICE int32 [num_reqs, block_table_stride]; row r holds at least
  *                ceil((kv_len+q_len)/B) page ids in [0, num_pages)
+ *   sm_scale     softmax scale, positive and finite (1/sqrt(D) in the usual case)
  *   tree_mask    DEVICE, nullable: a caller-built corner mask in plan's format
  *                replacing the one plan built from the parent arrays
  *   o            DEVICE bf16 [T, Hq, D] with token stride o_token_stride (elements)

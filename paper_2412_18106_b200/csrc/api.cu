@@ -234,6 +234,8 @@ int xy_attn_run(xy_attn_ctx* ctx, const void* q, int64_t q_token_stride, const v
       page_stride % 8 != 0 || page_stride < 1 || num_pages < 1)
     return set_err(ctx, XY_ERR_INVALID_ARG, "bad K/V pool strides or num_pages");
   if (block_table_stride < 1) return set_err(ctx, XY_ERR_INVALID_ARG, "bad block_table_stride");
+  if (!(sm_scale > 0.f) || !(sm_scale < 1e30f))
+    return set_err(ctx, XY_ERR_INVALID_ARG, "sm_scale must be positive and finite");
 
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   XY_CUDA(ctx, cudaSetDevice(cfg.device));
@@ -276,7 +278,7 @@ int xy_attn_run(xy_attn_ctx* ctx, const void* q, int64_t q_token_stride, const v
   if (cfg.kernel == XY_KERNEL_REFERENCE) {
     XY_CUDA(ctx, launch_reference(a, ctx->num_workers, s));
   } else {
-    XY_CUDA(ctx, launch_meta(a, ctx->num_workers, num_pages, s));
+    XY_CUDA(ctx, launch_meta(a, ctx->num_workers, num_pages, cfg.kernel == XY_KERNEL_AUTO, s));
   }
   ctx->last_launches += 1;
   if (timed) XY_CUDA(ctx, cudaEventRecord(ctx->events[3 * ctx->timed_runs + 1], s));

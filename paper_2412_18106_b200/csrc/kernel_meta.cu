@@ -48,7 +48,7 @@ struct __align__(8) SmemBarriers {
 constexpr int kSmemQ = 2 * kTileBytes;
 constexpr int kSmemRing = kStages * kTileBytes;
 constexpr int kSmemMl = kConsumerWarps * 16 * 2 * 4;
-constexpr int kSmemTotal = 1024 /*align slack*/ + kSmemQ + kSmemRing + kSmemMl + sizeof(SmemBarriers);
+constexpr int kSmemTotal = 1024 /*align slack*/ + kSmemQ + kSmemRing + kSmemMl + sizeof(SmemBarriers) + 128;
 
 __device__ __forceinline__ uint32_t swz(uint32_t row, uint32_t chunk16 /*0..15*/) {
   return (chunk16 >> 3) * kHalfBytes + row * 128u + (((chunk16 & 7u) ^ (row & 7u)) << 4);
@@ -246,6 +246,66 @@ __device__ __forceinline__ void report_timeout(const RunArgs& a) {
 }
 
 // ------------------------------------------------------------------------------------------
+// tcgen05 dense path.  TMEM columns: S_A [0,128) S_B [128,256) O_A [256,384) O_B [384,512);
+// P (bf16, two keys per 32-bit column) overwrites the first 64 columns of its S block.
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kTmemS = 0, kTmemO = 256;
+constexpr float kRescaleThreshold = 8.0f;  // log2 units: rescale O only when the row max grows by > 2^8
+
+// Shared-memory matrix descriptor, 128-byte swizzle, 8-row groups 1024 B apart.
+//   K-major operand (Q, K): rows are MN, 64 elements (128 B) per row; LBO unused.
+//   MN-major operand (V):   rows are K (keys), the second 64-element half of N is LBO bytes away.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((addr >> 4) & 0x3FFFu);
+  d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= static_cast<uint64_t>((1024u >> 4) & 0x3FFFu) << 32;
+  d |= 1ull << 46;  // descriptor version for sm_100
+  d |= 2ull << 61;  // SWIZZLE_128B
+  return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 128.
+constexpr uint32_t kIdescBase = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+constexpr uint32_t kIdescQK = kIdescBase;              // A, B K-major
+constexpr uint32_t kIdescPV = kIdescBase | (1u << 16);  // B (V) MN-major
+
+struct DenseShape {
+  int n[2];  // KV tiles sub-tile A / B visits in this task
+  int n_all;
+};
+__device__ __forceinline__ DenseShape dense_shape(const xy_attn_task& t, const ReqInfo& rq, int G) {
+  DenseShape d;
+  const int rows = t.ntok * G;
+#pragma unroll
+  for (int X = 0; X < 2; ++X) {
+    if (X * 128 >= rows) {
+      d.n[X] = 0;
+      continue;
+    }
+    const int last_tok = t.tok0 + (min(rows, (X + 1) * 128) - 1) / G;
+    const int frontier = (rq.kv_len + last_tok + 1 + kKeyTile - 1) / kKeyTile;
+    d.n[X] = max(0, min(t.kt_hi, frontier) - t.kt_lo);
+  }
+  d.n_all = t.kt_hi - t.kt_lo;
+  return d;
+}
+
+struct __align__(8) UmmaBarriers {
+  uint64_t q_full[2];  // consumers -> MMA: packed Q sub-tile is in shared memory
+  uint64_t s_full[2];  // MMA -> consumers: S = Q K^T of the next KV tile is in TMEM
+  uint64_t p_full[2];  // consumers -> MMA: P is in TMEM (and O rescaled if it had to be)
+  uint64_t o_done[2];  // MMA -> consumers: the task's last P V has completed
+  uint32_t tmem_base;
+  uint32_t pad;
+};
+
+// Corner-mask words of one row covering columns [jp0, jp0 + 128) of the speculative corner.
+struct TreeWords {
+  uint64_t w[3];
+  int wbase;
+};
+
+template <bool kUmma>
 __global__ void __launch_bounds__(kThreads, 1)
 meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constant__ CUtensorMap k_map,
                       const __grid_constant__ CUtensorMap v_map) {
@@ -257,6 +317,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
   uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
   float* ml = reinterpret_cast<float*>(gen_base + kSmemQ + kSmemRing);
   SmemBarriers* bars = reinterpret_cast<SmemBarriers*>(gen_base + kSmemQ + kSmemRing + kSmemMl);
+  UmmaBarriers* ub = reinterpret_cast<UmmaBarriers*>(gen_base + kSmemQ + kSmemRing + kSmemMl + sizeof(SmemBarriers));
   float* xch = reinterpret_cast<float*>(gen_base);  // streaming merge area, aliases the Q tiles
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -265,9 +326,22 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
       mbar_init(smem_u32(&bars->full[s]), 1);
       mbar_init(smem_u32(&bars->empty[s]), kConsumerWarps);
     }
+    for (int X = 0; X < 2; ++X) {
+      mbar_init(smem_u32(&ub->q_full[X]), 4);
+      mbar_init(smem_u32(&ub->s_full[X]), 1);
+      mbar_init(smem_u32(&ub->p_full[X]), 4);
+      mbar_init(smem_u32(&ub->o_done[X]), 1);
+    }
     fence_mbar_init();
   }
+  if (kUmma && warp == kConsumerWarps + 1) {
+    tmem_alloc(smem_u32(&ub->tmem_base), kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
   __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = kUmma ? ub->tmem_base : 0u;
 
   const int t_begin = a.worker_off[blockIdx.x], t_end = a.worker_off[blockIdx.x + 1];
   const int G = a.num_q_heads / a.num_kv_heads;
@@ -275,8 +349,8 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
 
   if (warp >= kConsumerWarps) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
-    // ================================ producer =========================================
     if (warp == kConsumerWarps && lane == 0) {
+      // ================================ producer =======================================
       prefetch_tensormap(&k_map);
       prefetch_tensormap(&v_map);
       Pipe pipe{0, 0};
@@ -309,12 +383,109 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
           }
         }
       }
+    } else if (kUmma && warp == kConsumerWarps + 1 && lane == 0) {
+      // ================================ tcgen05 MMA issuer ==============================
+      Pipe pipe{0, 0};
+      bool dead = false;
+      uint32_t ph_q[2] = {0, 0}, ph_p[2] = {0, 0};
+      auto wait_or_die = [&](uint32_t bar, uint32_t parity) {
+        if (!dead && !mbar_wait(bar, parity)) {
+          report_timeout(a);
+          dead = true;
+        }
+      };
+      // S_X = Q_X K^T (8 k-steps of 16 elements; the second 64-element half is 16 KiB away)
+      auto issue_qk = [&](int X, uint32_t k_tile) {
+        const uint32_t qx = q_smem + X * kTileBytes;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
+          umma_ss(tmem + kTmemS + X * 128, smem_desc(qx + off, 16), smem_desc(k_tile + off, 16), kIdescQK,
+                  ks > 0 ? 1u : 0u);
+        }
+      };
+      // O_X (+)= P_X V (8 k-steps of 16 keys; P is read from TMEM, 8 columns per k-step)
+      auto issue_pv = [&](int X, uint32_t v_tile, bool accumulate) {
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          umma_ts(tmem + kTmemO + X * 128, tmem + kTmemS + X * 128 + ks * 8,
+                  smem_desc(v_tile + ks * 2048, kHalfBytes), kIdescPV, (accumulate || ks > 0) ? 1u : 0u);
+        }
+      };
+      auto release = [&](int stage) {  // the ring's empty barriers count eight arrivals
+#pragma unroll
+        for (int c = 0; c < kConsumerWarps; ++c) umma_commit(smem_u32(&bars->empty[stage]));
+      };
+      for (int ti = t_begin; ti < t_end; ++ti) {
+        const xy_attn_task t = a.tasks[ti];
+        const int n_all = t.kt_hi - t.kt_lo;
+        if (t.kind == 1) {  // streaming tasks never touch the tensor-memory path
+          for (int c = 0; c < 2 * n_all; ++c) pipe.advance();
+          continue;
+        }
+        const ReqInfo rq = a.reqs[t.req];
+        const DenseShape ds = dense_shape(t, rq, G);
+        for (int X = 0; X < 2; ++X) {
+          if (ds.n[X] > 0) {
+            wait_or_die(smem_u32(&ub->q_full[X]), ph_q[X]);
+            ph_q[X] ^= 1u;
+          }
+        }
+        // first KV tile: S(0) for both sub-tiles
+        wait_or_die(smem_u32(&bars->full[pipe.stage]), pipe.phase);
+        tc_fence_after();
+        if (!dead) {
+          for (int X = 0; X < 2; ++X) {
+            if (ds.n[X] > 0) {
+              issue_qk(X, ring + pipe.stage * kTileBytes);
+              umma_commit(smem_u32(&ub->s_full[X]));
+            }
+          }
+          release(pipe.stage);
+        }
+        pipe.advance();
+        for (int j = 0; j < n_all; ++j) {
+          const int v_stage = pipe.stage;
+          const uint32_t v_phase = pipe.phase;
+          pipe.advance();
+          const int k_stage = pipe.stage;
+          const uint32_t k_phase = pipe.phase;
+          const bool more = j + 1 < n_all;
+          if (more) pipe.advance();
+          wait_or_die(smem_u32(&bars->full[v_stage]), v_phase);
+          bool k_ready = false;
+          for (int X = 0; X < 2; ++X) {
+            if (j < ds.n[X]) {
+              wait_or_die(smem_u32(&ub->p_full[X]), ph_p[X]);
+              ph_p[X] ^= 1u;
+              tc_fence_after();
+              if (!dead) {
+                issue_pv(X, ring + v_stage * kTileBytes, j > 0);
+                if (j == ds.n[X] - 1) umma_commit(smem_u32(&ub->o_done[X]));
+              }
+            }
+            if (X == 1 && !dead) release(v_stage);
+            if (more && !k_ready) {
+              wait_or_die(smem_u32(&bars->full[k_stage]), k_phase);
+              tc_fence_after();
+              k_ready = true;
+            }
+            if (j + 1 < ds.n[X] && !dead) {
+              issue_qk(X, ring + k_stage * kTileBytes);
+              umma_commit(smem_u32(&ub->s_full[X]));
+            }
+            if (X == 1 && more && !dead) release(k_stage);
+          }
+        }
+      }
     }
   } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsConsumer));
     // ================================ consumers ========================================
     Pipe pipe{0, 0};
     bool dead = false;
+    uint32_t ph_s = 0, ph_o = 0;  // this warpgroup's s_full / o_done parities
+    const int X = warp >> 2;       // sub-tile this warpgroup owns on the tcgen05 path
     for (int ti = t_begin; ti < t_end; ++ti) {
       TaskView tv;
       tv.t = a.tasks[ti];
@@ -324,6 +495,182 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
       const int h = tv.rq.kv_len;
       const bool tree = tv.rq.mask_kind == XY_MASK_TREE;
       const bool stream = tv.t.kind == 1;
+
+      if (kUmma && !stream) {
+        // ---------------- dense on tcgen05: this thread owns packed row x of sub-tile X ----
+        const DenseShape ds = dense_shape(tv.t, tv.rq, G);
+        for (int c = 0; c < 2 * ds.n_all; ++c) pipe.advance();  // the ring moves on without us
+        const int r = (warp & 3) * 32 + lane;
+        const int x = X * 128 + r;
+        const bool exists = X * 128 < tv.rows;
+        const bool valid = x < tv.rows;
+        if (!exists) continue;
+        const int nX = ds.n[X];
+        const int i_row = tv.t.tok0 + min(x, tv.rows - 1) / G;
+        if (nX == 0) {  // a KV split that lies wholly above this sub-tile's causal frontier
+          if (valid) {
+            for (int c = 0; c < kHeadDim; c += 2) write_row_pair(a, tv, x, c, 0.f, 0.f);
+            write_lse(a, tv, x, -INFINITY);
+          }
+          continue;
+        }
+        // packed Q sub-tile -> shared memory, then hand it to the async proxy
+        {
+          const int t128 = threadIdx.x & 127;
+          for (int c = t128; c < 128 * 16; c += 128) {
+            const int rr = c >> 4, ch = c & 15;
+            const int xr = X * 128 + rr;
+            const bool ok = xr < tv.rows;
+            const int xx = ok ? xr : 0;
+            const int i = tv.t.tok0 + xx / G, head = tv.t.kv_head * G + xx % G;
+            const uint16_t* src =
+                a.q + static_cast<int64_t>(tv.rq.q_start + i) * a.q_token_stride + head * kHeadDim + ch * 8;
+            cp_async_16(q_smem + X * kTileBytes + swz(rr, ch), src, ok);
+          }
+          cp_async_commit_wait_all();
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&ub->q_full[X]));
+        }
+        const uint32_t lane_base = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+        const uint32_t t_s = lane_base + kTmemS + X * 128, t_o = lane_base + kTmemO + X * 128;
+        const int i_min = tv.t.tok0 + (X * 128) / G;
+        float m_ref = -INFINITY, l = 0.f;
+        for (int j = 0; j < nX; ++j) {
+          const int col0 = (tv.t.kt_lo + j) * kKeyTile;
+          if (!dead && !mbar_wait(smem_u32(&ub->s_full[X]), ph_s)) {
+            report_timeout(a);
+            dead = true;
+          }
+          ph_s ^= 1u;
+          tc_fence_after();
+          uint32_t sr[128];
+          {
+            uint32_t(&c0)[32] = *reinterpret_cast<uint32_t(*)[32]>(&sr[0]);
+            uint32_t(&c1)[32] = *reinterpret_cast<uint32_t(*)[32]>(&sr[32]);
+            uint32_t(&c2)[32] = *reinterpret_cast<uint32_t(*)[32]>(&sr[64]);
+            uint32_t(&c3)[32] = *reinterpret_cast<uint32_t(*)[32]>(&sr[96]);
+            tmem_ld_32x32b_x32(t_s, c0);
+            tmem_ld_32x32b_x32(t_s + 32, c1);
+            tmem_ld_32x32b_x32(t_s + 64, c2);
+            tmem_ld_32x32b_x32(t_s + 96, c3);
+            tmem_wait_ld();
+          }
+          const bool need_mask = tree ? (col0 + kKeyTile > h) : (col0 + kKeyTile > h + i_min + 1);
+          if (need_mask) {
+            const int frontier = h + i_row;  // last visible column of this row
+            TreeWords tw;
+            tw.wbase = 0;
+            tw.w[0] = tw.w[1] = tw.w[2] = 0ull;
+            if (tree) {
+              const int jp0 = max(col0 - h, 0);
+              tw.wbase = jp0 >> 6;
+              const uint64_t* mrow = a.tree_mask + tv.rq.tree_off + static_cast<int64_t>(i_row) * tv.rq.tree_words;
+#pragma unroll
+              for (int q = 0; q < 3; ++q)
+                if (tw.wbase + q < tv.rq.tree_words) tw.w[q] = __ldg(mrow + tw.wbase + q);
+            }
+#pragma unroll
+            for (int k = 0; k < 128; ++k) {
+              const int col = col0 + k;
+              bool vis = col <= frontier;
+              if (tree && col >= h) {
+                const int jp = col - h;
+                const int wi = (jp >> 6) - tw.wbase;
+                const uint64_t word = wi == 0 ? tw.w[0] : (wi == 1 ? tw.w[1] : tw.w[2]);
+                vis = vis && ((word >> (jp & 63)) & 1ull);
+              }
+              if (!vis) sr[k] = 0xff800000u;  // -inf, selected (never added)
+            }
+          }
+          float mx = -INFINITY;
+#pragma unroll
+          for (int k = 0; k < 128; ++k) mx = fmaxf(mx, __uint_as_float(sr[k]));
+          const float m_cand = fmaxf(m_ref, mx * scale_log2);
+          bool need = false;
+          if (j == 0 || m_ref == -INFINITY) {
+            m_ref = m_cand;  // nothing accumulated yet for this row: adopt the max, no rescale
+          } else {
+            need = m_cand - m_ref > kRescaleThreshold;
+          }
+          if (__any_sync(0xffffffffu, need)) {
+            // Update stage: O *= 2^(m_old - m_new).  The previous P V has completed, because
+            // this tile's S was issued behind it on the in-order tensor pipe.
+            const float alpha = (m_cand == -INFINITY) ? 1.f : ex2(m_ref - m_cand);
+            l *= alpha;
+            m_ref = m_cand;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              uint32_t orow[32];
+              tmem_ld_32x32b_x32(t_o + c * 32, orow);
+              tmem_wait_ld();
+#pragma unroll
+              for (int k = 0; k < 32; ++k) orow[k] = __float_as_uint(__uint_as_float(orow[k]) * alpha);
+              tmem_st_32x32b_x32(t_o + c * 32, orow);
+            }
+          }
+          const float neg_off = (m_ref == -INFINITY) ? 0.f : -m_ref;
+          float sum = 0.f;
+          uint32_t pk[64];
+#pragma unroll
+          for (int k = 0; k < 64; ++k) {
+            const float p0 = ex2(fmaf(__uint_as_float(sr[2 * k]), scale_log2, neg_off));
+            const float p1 = ex2(fmaf(__uint_as_float(sr[2 * k + 1]), scale_log2, neg_off));
+            sum += p0 + p1;
+            pk[k] = pack_bf16(p0, p1);
+          }
+          l += sum;
+          {
+            uint32_t(&h0)[32] = *reinterpret_cast<uint32_t(*)[32]>(&pk[0]);
+            uint32_t(&h1)[32] = *reinterpret_cast<uint32_t(*)[32]>(&pk[32]);
+            tmem_st_32x32b_x32(t_s, h0);
+            tmem_st_32x32b_x32(t_s + 32, h1);
+            tmem_wait_st();
+          }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&ub->p_full[X]));
+        }
+        // ---- epilogue: O / l -> global
+        if (!dead && !mbar_wait(smem_u32(&ub->o_done[X]), ph_o)) {
+          report_timeout(a);
+          dead = true;
+        }
+        ph_o ^= 1u;
+        tc_fence_after();
+        const float inv = l > 0.f ? 1.f / l : 0.f;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint32_t orow[32];
+          tmem_ld_32x32b_x32(t_o + c * 32, orow);
+          tmem_wait_ld();
+          if (valid) {
+            if (tv.t.part < 0) {
+              const int head = tv.t.kv_head * G + x % G;
+              uint4* dst = reinterpret_cast<uint4*>(a.o + static_cast<int64_t>(tv.rq.q_start + i_row) * a.o_token_stride +
+                                                    head * kHeadDim + c * 32);
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                uint4 v;
+                v.x = pack_bf16(__uint_as_float(orow[q * 8 + 0]) * inv, __uint_as_float(orow[q * 8 + 1]) * inv);
+                v.y = pack_bf16(__uint_as_float(orow[q * 8 + 2]) * inv, __uint_as_float(orow[q * 8 + 3]) * inv);
+                v.z = pack_bf16(__uint_as_float(orow[q * 8 + 4]) * inv, __uint_as_float(orow[q * 8 + 5]) * inv);
+                v.w = pack_bf16(__uint_as_float(orow[q * 8 + 6]) * inv, __uint_as_float(orow[q * 8 + 7]) * inv);
+                dst[q] = v;
+              }
+            } else {
+              float4* dst = reinterpret_cast<float4*>(a.o_part + static_cast<int64_t>(tv.t.part + x) * kHeadDim + c * 32);
+#pragma unroll
+              for (int q = 0; q < 8; ++q)
+                dst[q] = make_float4(__uint_as_float(orow[q * 4 + 0]) * inv, __uint_as_float(orow[q * 4 + 1]) * inv,
+                                     __uint_as_float(orow[q * 4 + 2]) * inv, __uint_as_float(orow[q * 4 + 3]) * inv);
+            }
+          }
+        }
+        if (valid) write_lse(a, tv, x, l > 0.f ? (m_ref + log2f(l)) * kLn2 : -INFINITY);
+        tc_fence_before();  // order this task's TMEM reads before the next task's MMAs
+        continue;
+      }
 
       // ---- packed Q tile -> shared memory (rows past the tile are zero-filled)
       {
@@ -481,7 +828,12 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
       }
     }
   }
+  tc_fence_before();
   __syncthreads();
+  if (kUmma && warp == kConsumerWarps + 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, kTmemCols);
+  }
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -520,9 +872,9 @@ bool encode_pool_map(CUtensorMap* m, const void* pool, int64_t num_pages, int nu
 
 }  // namespace
 
-cudaError_t launch_meta(const RunArgs& a, int num_workers, int64_t num_pages, cudaStream_t s) {
-  cudaError_t e = cudaFuncSetAttribute(meta_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       kSmemTotal);
+cudaError_t launch_meta(const RunArgs& a, int num_workers, int64_t num_pages, bool umma, cudaStream_t s) {
+  auto kernel = umma ? meta_attention_kernel<true> : meta_attention_kernel<false>;
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTotal);
   if (e != cudaSuccess) return e;
   CUtensorMap k_map, v_map;
   if (!encode_pool_map(&k_map, a.k_pool, num_pages, a.num_kv_heads, a.page_size, a.page_stride, a.head_stride,
@@ -531,7 +883,7 @@ cudaError_t launch_meta(const RunArgs& a, int num_workers, int64_t num_pages, cu
                        a.token_stride))
     return cudaErrorInvalidValue;
   MetaParams P{a};
-  meta_attention_kernel<<<num_workers, kThreads, kSmemTotal, s>>>(P, k_map, v_map);
+  kernel<<<num_workers, kThreads, kSmemTotal, s>>>(P, k_map, v_map);
   return cudaGetLastError();
 }
 

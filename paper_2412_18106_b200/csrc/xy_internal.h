@@ -38,7 +38,7 @@ struct PlanResult {
 };
 
 // 128-row sub-tiles one dense task may hold (the tcgen05 path ping-pongs two; the others one).
-inline int dense_subtiles(const xy_attn_config& cfg) { (void)cfg; return 1; }
+inline int dense_subtiles(const xy_attn_config& cfg) { return cfg.kernel == XY_KERNEL_AUTO ? 2 : 1; }
 
 // Host-only planning.  Returns XY_OK or an error code and fills `err`.
 int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_capacity,
