@@ -194,7 +194,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="full_mix",
-                    choices=["decode_only", "splitfuse_mix", "verify_trees", "full_mix", "tiny_hybrid"])
+                    choices=["decode_only", "splitfuse_mix", "verify_trees", "full_mix", "tiny_hybrid",
+                             "prefill_prefix"])
     ap.add_argument("--kernel", default="auto", choices=["auto", "reference", "mma"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")

@@ -180,6 +180,13 @@ int xy_attn_debug_gather(xy_attn_ctx* ctx, int32_t req, int32_t kv_head, const v
                          int64_t token_stride, const int32_t* block_table,
                          int32_t block_table_stride, void* out_k, void* out_v, void* stream);
 
+/* Debug tracing.  When the environment variable XY_ATTN_TRACE=1 is set at create time, the
+ * roles of worker 0 (sub-tile A, sub-tile B, MMA issuer, producer) stamp (tag << 48 | SM cycle
+ * counter) records into a context-owned buffer of 4 x 2048 entries per run.  This call
+ * synchronises the device and copies them to `out` (HOST); it returns the number of entries
+ * (0 when tracing is off) and copies only if `cap` is large enough. */
+int xy_attn_debug_trace(xy_attn_ctx* ctx, uint64_t* out, int32_t cap);
+
 /* Introspection of the current plan (HOST outputs).  Each returns the number of
  * items of the plan, or a negative error; at most `cap` items are written. */
 int xy_attn_get_tasks(const xy_attn_ctx* ctx, xy_attn_task* out, int32_t cap);

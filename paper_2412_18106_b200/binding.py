@@ -73,7 +73,7 @@ EXPORTS = (
     "xy_attn_debug_gather", "xy_attn_get_tasks", "xy_attn_get_worker_offsets",
     "xy_attn_get_merge_units", "xy_attn_get_tree_mask", "xy_attn_get_q_start",
     "xy_attn_last_launches", "xy_attn_last_error", "xy_attn_device_status",
-    "xy_attn_set_timing", "xy_attn_get_timing",
+    "xy_attn_set_timing", "xy_attn_get_timing", "xy_attn_debug_trace",
 )
 
 _lib = None
@@ -103,6 +103,7 @@ def load() -> ctypes.CDLL:
     L.xy_attn_set_timing.argtypes = [vp, i32]
     L.xy_attn_get_timing.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float),
                                      ctypes.POINTER(i32)]
+    L.xy_attn_debug_trace.argtypes = [vp, vp, i32]
     L.xy_attn_last_launches.argtypes = [vp]
     L.xy_attn_last_error.argtypes = [vp]
     L.xy_attn_last_error.restype = ctypes.c_char_p
@@ -236,6 +237,15 @@ class XYAttn:
         a, m, n = ctypes.c_float(0), ctypes.c_float(0), ctypes.c_int32(0)
         self._check(self.lib.xy_attn_get_timing(self._ctx, ctypes.byref(a), ctypes.byref(m), ctypes.byref(n)))
         return float(a.value), float(m.value), int(n.value)
+
+    def debug_trace(self) -> np.ndarray:
+        """uint64 [4, 2048] trace records of worker 0 (empty unless XY_ATTN_TRACE=1 at create)."""
+        n = self.lib.xy_attn_debug_trace(self._ctx, ctypes.c_void_p(0), 0)
+        if n <= 0:
+            return np.zeros((0,), dtype=np.uint64)
+        out = np.zeros(n, dtype=np.uint64)
+        self.lib.xy_attn_debug_trace(self._ctx, ctypes.c_void_p(out.ctypes.data), n)
+        return out.reshape(4, -1)
 
     def last_launches(self) -> int:
         return int(self.lib.xy_attn_last_launches(self._ctx))

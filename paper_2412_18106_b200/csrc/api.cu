@@ -3,6 +3,7 @@
 #include <cuda_runtime.h>
 
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <string>
@@ -30,6 +31,7 @@ struct xy_attn_ctx {
   float* d_o_part = nullptr;
   float* d_lse_part = nullptr;
   int32_t* d_status = nullptr;
+  unsigned long long* d_trace = nullptr;
   int last_launches = 0;
   bool timing = false;
   std::vector<cudaEvent_t> events;  // three per timed run: before attention, after it, after merge
@@ -70,6 +72,7 @@ void free_device(xy_attn_ctx* c) {
   cudaFree(c->d_o_part);
   cudaFree(c->d_lse_part);
   cudaFree(c->d_status);
+  cudaFree(c->d_trace);
 }
 
 }  // namespace
@@ -144,6 +147,11 @@ int xy_attn_create(const xy_attn_config* cfg, xy_attn_ctx** out) {
     alloc(reinterpret_cast<void**>(&c->d_lse_part), sizeof(float) * c->cap_partial_rows);
     alloc(reinterpret_cast<void**>(&c->d_status), 256);
     if (e == cudaSuccess) e = cudaMemset(c->d_status, 0, 256);
+    const char* tr = getenv("XY_ATTN_TRACE");
+    if (tr != nullptr && tr[0] == '1') {
+      alloc(reinterpret_cast<void**>(&c->d_trace), sizeof(unsigned long long) * kTraceRoles * kTraceLen);
+      if (e == cudaSuccess) e = cudaMemset(c->d_trace, 0, sizeof(unsigned long long) * kTraceRoles * kTraceLen);
+    }
     if (e != cudaSuccess) {
       free_device(c);
       delete c;
@@ -260,6 +268,7 @@ int xy_attn_run(xy_attn_ctx* ctx, const void* q, int64_t q_token_stride, const v
   a.o_part = ctx->d_o_part;
   a.lse_part = ctx->d_lse_part;
   a.status = ctx->d_status;
+  a.trace = ctx->d_trace;
   a.num_q_heads = cfg.num_q_heads;
   a.num_kv_heads = cfg.num_kv_heads;
   a.page_size = cfg.page_size;
@@ -382,6 +391,16 @@ XY_GETTER(xy_attn_get_worker_offsets, int32_t, worker_off)
 XY_GETTER(xy_attn_get_merge_units, xy_attn_merge_unit, merges)
 XY_GETTER(xy_attn_get_tree_mask, uint64_t, tree_mask)
 XY_GETTER(xy_attn_get_q_start, int32_t, q_start)
+
+int xy_attn_debug_trace(xy_attn_ctx* ctx, uint64_t* out, int32_t cap) {
+  if (ctx == nullptr || (out == nullptr && cap > 0)) return XY_ERR_INVALID_ARG;
+  if (ctx->host_only || ctx->d_trace == nullptr) return 0;
+  const int n = kTraceRoles * kTraceLen;
+  XY_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+  XY_CUDA(ctx, cudaDeviceSynchronize());
+  if (cap >= n) XY_CUDA(ctx, cudaMemcpy(out, ctx->d_trace, sizeof(uint64_t) * n, cudaMemcpyDeviceToHost));
+  return n;
+}
 
 int xy_attn_last_launches(const xy_attn_ctx* ctx) { return ctx ? ctx->last_launches : XY_ERR_INVALID_ARG; }
 

@@ -32,8 +32,8 @@ using namespace ptx;
 constexpr int kConsumerWarps = 8;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
 constexpr int kThreads = kConsumerThreads + 128;  // + one warpgroup: producer, MMA issuer, 2 idle
-constexpr int kRegsConsumer = 232;               // setmaxnreg budgets: 256 x 232 + 128 x 40 <= 64 Ki
-constexpr int kRegsOther = 40;
+constexpr int kRegsConsumer = 216;  // setmaxnreg budgets: 256 x 216 + 128 x 72 = 168 x 384, the launch allocation
+constexpr int kRegsOther = 72;
 constexpr int kStages = 4;
 constexpr int kTileBytes = 32768;  // 2 halves x 128 rows x 128 B
 constexpr int kHalfBytes = 16384;
@@ -42,7 +42,8 @@ constexpr float kLn2 = 0.6931471805599453f;
 
 struct __align__(8) SmemBarriers {
   uint64_t full[kStages];
-  uint64_t empty[kStages];
+  uint64_t empty[kStages];      // released by the eight consumer warps (warp-level MMA paths)
+  uint64_t empty_umma[kStages];  // released by two tcgen05.commit arrivals (tensor-memory path)
 };
 
 constexpr int kSmemQ = 2 * kTileBytes;
@@ -241,6 +242,19 @@ __device__ __forceinline__ void write_lse(const RunArgs& a, const TaskView& tv, 
   }
 }
 
+// Debug trace of worker 0: one record per call, (tag << 48) | SM cycle counter.
+struct Tracer {
+  unsigned long long* p;
+  int n;
+  __device__ __forceinline__ void init(const RunArgs& a, int role, bool on) {
+    p = (a.trace != nullptr && blockIdx.x == 0 && on) ? a.trace + role * kTraceLen : nullptr;
+    n = 0;
+  }
+  __device__ __forceinline__ void operator()(unsigned tag) {
+    if (p != nullptr && n < kTraceLen) p[n++] = (static_cast<unsigned long long>(tag) << 48) | (clock64() & 0xFFFFFFFFFFFFull);
+  }
+};
+
 __device__ __forceinline__ void report_timeout(const RunArgs& a) {
   atomicExch(a.status, XY_ERR_DEVICE_TIMEOUT);
 }
@@ -293,10 +307,10 @@ __device__ __forceinline__ DenseShape dense_shape(const xy_attn_task& t, const R
 struct __align__(8) UmmaBarriers {
   uint64_t q_full[2];  // consumers -> MMA: packed Q sub-tile is in shared memory
   uint64_t s_full[2];  // MMA -> consumers: S = Q K^T of the next KV tile is in TMEM
-  uint64_t p_full[2];  // consumers -> MMA: P is in TMEM (and O rescaled if it had to be)
+  uint64_t p_full[2][2];  // consumers -> MMA: [sub-tile][half] 64 keys of P are in TMEM (O rescaled if need be)
   uint64_t o_done[2];  // MMA -> consumers: the task's last P V has completed
   uint32_t tmem_base;
-  uint32_t pad;
+  volatile uint32_t turn;  // index of the next MMA group allowed onto the tensor pipe
 };
 
 // Corner-mask words of one row covering columns [jp0, jp0 + 128) of the speculative corner.
@@ -325,11 +339,14 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
     for (int s = 0; s < kStages; ++s) {
       mbar_init(smem_u32(&bars->full[s]), 1);
       mbar_init(smem_u32(&bars->empty[s]), kConsumerWarps);
+      mbar_init(smem_u32(&bars->empty_umma[s]), 2);
     }
+    ub->turn = 0;
     for (int X = 0; X < 2; ++X) {
       mbar_init(smem_u32(&ub->q_full[X]), 4);
       mbar_init(smem_u32(&ub->s_full[X]), 1);
-      mbar_init(smem_u32(&ub->p_full[X]), 4);
+      mbar_init(smem_u32(&ub->p_full[X][0]), 4);
+      mbar_init(smem_u32(&ub->p_full[X][1]), 4);
       mbar_init(smem_u32(&ub->o_done[X]), 1);
     }
     fence_mbar_init();
@@ -355,6 +372,11 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
       prefetch_tensormap(&v_map);
       Pipe pipe{0, 0};
       bool dead = false;
+      // Who read each stage last (bit set: the tcgen05 path) and the parity to wait for on each
+      // of the two empty barriers of a stage; a stage that was never filled needs no wait.
+      uint32_t used = 0, last_umma = 0, ph_cons = 0, ph_umma = 0;
+      Tracer tr;
+      tr.init(a, 3, true);
       const int ppt = kKeyTile >> a.page_shift;  // pages per 128-key tile
       const uint32_t page_bytes = static_cast<uint32_t>(a.page_size) * 128u;
       for (int ti = t_begin; ti < t_end && !dead; ++ti) {
@@ -362,13 +384,28 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
         const ReqInfo rq = a.reqs[t.req];
         const int npages = (rq.kv_len + rq.q_len + a.page_size - 1) >> a.page_shift;
         const int32_t* bt = a.block_table + static_cast<int64_t>(t.req) * a.bt_stride;
+        const bool by_umma = kUmma && t.kind == 0;
         for (int kt = t.kt_lo; kt < t.kt_hi && !dead; ++kt) {
           for (int op = 0; op < 2; ++op) {
-            if (!mbar_wait(smem_u32(&bars->empty[pipe.stage]), pipe.phase ^ 1u)) {
-              report_timeout(a);
-              dead = true;
-              break;
+            const uint32_t bit = 1u << pipe.stage;
+            if (used & bit) {
+              bool ok;
+              if (last_umma & bit) {
+                ok = mbar_wait(smem_u32(&bars->empty_umma[pipe.stage]), (ph_umma >> pipe.stage) & 1u, a.status);
+                ph_umma ^= bit;
+              } else {
+                ok = mbar_wait(smem_u32(&bars->empty[pipe.stage]), (ph_cons >> pipe.stage) & 1u, a.status);
+                ph_cons ^= bit;
+              }
+              if (!ok) {
+                report_timeout(a);
+                dead = true;
+                break;
+              }
             }
+            used |= bit;
+            last_umma = by_umma ? (last_umma | bit) : (last_umma & ~bit);
+            tr(1 + op);
             const uint32_t full = smem_u32(&bars->full[pipe.stage]);
             mbar_arrive_expect_tx(full, kTileBytes);
             const uint32_t dst = ring + pipe.stage * kTileBytes;
@@ -383,99 +420,150 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
           }
         }
       }
-    } else if (kUmma && warp == kConsumerWarps + 1 && lane == 0) {
-      // ================================ tcgen05 MMA issuer ==============================
-      Pipe pipe{0, 0};
+    } else if (kUmma && (warp == kConsumerWarps + 1 || warp == kConsumerWarps + 2) && lane == 0) {
+      // ================================ tcgen05 MMA issuers =============================
+      // One issuing thread per sub-tile (on different schedulers), each walking its own chain
+      //   S_X(0);  for j: [P_X(j) ready] O_X += P_X(j) V(j);  S_X(j+1) = Q_X K(j+1)^T.
+      // The MMAs of one thread execute in order, which is what lets P overwrite S in place.
+      const int X = warp - (kConsumerWarps + 1);
+      uint32_t pos = 0;  // ring position: stage = pos % kStages, parity = (pos / kStages) & 1
       bool dead = false;
-      uint32_t ph_q[2] = {0, 0}, ph_p[2] = {0, 0};
+      uint32_t ph_q = 0, ph_p = 0;
+      Tracer tr;
+      tr.init(a, 2, X == 0);
       auto wait_or_die = [&](uint32_t bar, uint32_t parity) {
-        if (!dead && !mbar_wait(bar, parity)) {
+        if (!dead && !mbar_wait(bar, parity, a.status)) {
           report_timeout(a);
           dead = true;
         }
       };
-      // S_X = Q_X K^T (8 k-steps of 16 elements; the second 64-element half is 16 KiB away)
-      auto issue_qk = [&](int X, uint32_t k_tile) {
-        const uint32_t qx = q_smem + X * kTileBytes;
+      auto wait_full = [&](uint32_t p) {
+        wait_or_die(smem_u32(&bars->full[p % kStages]), (p / kStages) & 1u);
+        tc_fence_after();
+      };
+      // Descriptor halves.  High word (same for every operand here): 8-row groups 1024 B apart,
+      // sm_100 descriptor version, 128-byte swizzle.  Low word: start address >> 4 in bits 0-13,
+      // leading byte offset >> 4 in bits 16-29 (16 B for the K-major Q / K tiles; 16 KiB, the
+      // distance to the second 64-element half, for the MN-major V tile).
+      constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+      constexpr uint64_t kDescHi64 = static_cast<uint64_t>(kDescHi) << 32;
+      const uint32_t ring_lo = (ring >> 4) & 0x3FFFu;
+      const uint32_t t_s = tmem + kTmemS + X * 128, t_o = tmem + kTmemO + X * 128;
+      // The issuing thread gets few issue slots next to the softmax warps, so everything an MMA
+      // needs is computed ahead of the turn: Q descriptors once, K / V descriptors per tile.
+      uint64_t qd[8];
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-          const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
-          umma_ss(tmem + kTmemS + X * 128, smem_desc(qx + off, 16), smem_desc(k_tile + off, 16), kIdescQK,
-                  ks > 0 ? 1u : 0u);
+      for (int ks = 0; ks < 8; ++ks) {
+        const uint32_t off = (ks >> 2) * (kHalfBytes >> 4) + (ks & 3) * 2;
+        qd[ks] = kDescHi64 | (((((q_smem + X * kTileBytes) >> 4) & 0x3FFFu) + off) | (1u << 16));
+      }
+      // K tile (K-major): 8 k-steps of 16 elements, 32 B apart, the second half 16 KiB away
+      auto k_descs = [&](uint32_t p, uint64_t (&kd)[8]) {
+        const uint32_t b0 = (ring_lo + (p % kStages) * (kTileBytes >> 4)) | (1u << 16);
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks)
+          kd[ks] = kDescHi64 | (b0 + (ks >> 2) * (kHalfBytes >> 4) + (ks & 3) * 2);
+      };
+      // V tile (MN-major): 8 k-steps of 16 keys, 2 KiB apart; LBO = 16 KiB to the second half
+      auto v_descs = [&](uint32_t p, uint64_t (&vd)[8]) {
+        const uint32_t b0 = (ring_lo + (p % kStages) * (kTileBytes >> 4)) | ((kHalfBytes >> 4) << 16);
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) vd[ks] = kDescHi64 | (b0 + ks * 128);
+      };
+      auto issue_qk = [&](const uint64_t (&kd)[8]) {  // S_X = Q_X K^T
+        umma_ss64(t_s, qd[0], kd[0], kIdescQK, 0u);
+#pragma unroll
+        for (int ks = 1; ks < 8; ++ks) umma_ss64(t_s, qd[ks], kd[ks], kIdescQK, 1u);
+        umma_commit(smem_u32(&ub->s_full[X]));
+      };
+      // O_X (+)= P_X V with P in TMEM, in two halves of 64 keys: the first half is issued while
+      // the softmax warps are still exponentiating the second.
+      auto issue_pv_lo = [&](const uint64_t (&vd)[8], bool accumulate) {
+        umma_ts64(t_o, t_s, vd[0], kIdescPV, accumulate ? 1u : 0u);
+#pragma unroll
+        for (int ks = 1; ks < 4; ++ks) umma_ts64(t_o, t_s + ks * 8, vd[ks], kIdescPV, 1u);
+      };
+      auto issue_pv_hi = [&](const uint64_t (&vd)[8]) {
+#pragma unroll
+        for (int ks = 4; ks < 8; ++ks) umma_ts64(t_o, t_s + ks * 8, vd[ks], kIdescPV, 1u);
+      };
+      // A stage's empty barrier counts two arrivals: one per sub-tile that reads it, or both
+      // from the only reader.
+      auto release = [&](uint32_t p, bool alone) {
+        umma_commit(smem_u32(&bars->empty_umma[p % kStages]));
+        if (alone) umma_commit(smem_u32(&bars->empty_umma[p % kStages]));
+      };
+      // The two issuers take strict turns on the tensor pipe (A, B, A, B, ... skipping a sub-tile
+      // that has nothing left), so that one sub-tile's softmax always overlaps the other's MMAs
+      // instead of both falling into lockstep.  `turn` counts the groups issued so far.
+      uint32_t g_base = 0;
+      auto take_turn = [&](uint32_t g) {
+        if (dead) return;
+        for (uint32_t spin = 0; ub->turn != g; ++spin) {
+          if (spin > (1u << 22) || ((spin & 4095u) == 4095u && *reinterpret_cast<const volatile int32_t*>(a.status) != 0)) {
+            report_timeout(a);
+            dead = true;
+            return;
+          }
         }
       };
-      // O_X (+)= P_X V (8 k-steps of 16 keys; P is read from TMEM, 8 columns per k-step)
-      auto issue_pv = [&](int X, uint32_t v_tile, bool accumulate) {
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-          umma_ts(tmem + kTmemO + X * 128, tmem + kTmemS + X * 128 + ks * 8,
-                  smem_desc(v_tile + ks * 2048, kHalfBytes), kIdescPV, (accumulate || ks > 0) ? 1u : 0u);
-        }
-      };
-      auto release = [&](int stage) {  // the ring's empty barriers count eight arrivals
-#pragma unroll
-        for (int c = 0; c < kConsumerWarps; ++c) umma_commit(smem_u32(&bars->empty[stage]));
-      };
+      auto pass_turn = [&](uint32_t g) { ub->turn = g + 1; };
       for (int ti = t_begin; ti < t_end; ++ti) {
         const xy_attn_task t = a.tasks[ti];
-        const int n_all = t.kt_hi - t.kt_lo;
-        if (t.kind == 1) {  // streaming tasks never touch the tensor-memory path
-          for (int c = 0; c < 2 * n_all; ++c) pipe.advance();
-          continue;
-        }
+        const uint32_t n_all = t.kt_hi - t.kt_lo;
+        const uint32_t pos0 = pos;
+        pos += 2 * n_all;
+        if (t.kind == 1) continue;  // streaming tasks never touch the tensor-memory path
         const ReqInfo rq = a.reqs[t.req];
         const DenseShape ds = dense_shape(t, rq, G);
-        for (int X = 0; X < 2; ++X) {
-          if (ds.n[X] > 0) {
-            wait_or_die(smem_u32(&ub->q_full[X]), ph_q[X]);
-            ph_q[X] ^= 1u;
+        const int nX = ds.n[X], nY = ds.n[1 - X];
+        const int nA = ds.n[0], nB = ds.n[1];
+        const uint32_t g0 = g_base;                                  // first group of this task
+        const uint32_t g1 = g0 + (nA > 0 ? 1u : 0u) + (nB > 0 ? 1u : 0u);  // first group of the j loop
+        g_base = g1 + nA + nB;
+        if (nX == 0) continue;
+        wait_or_die(smem_u32(&ub->q_full[X]), ph_q);
+        ph_q ^= 1u;
+        uint64_t kd[8], vd[8];
+        k_descs(pos0, kd);
+        wait_full(pos0);
+        {
+          const uint32_t g = g0 + ((X == 1 && nA > 0) ? 1u : 0u);
+          take_turn(g);
+          if (!dead) {
+            issue_qk(kd);
+            release(pos0, nY == 0);
           }
+          pass_turn(g);
         }
-        // first KV tile: S(0) for both sub-tiles
-        wait_or_die(smem_u32(&bars->full[pipe.stage]), pipe.phase);
-        tc_fence_after();
-        if (!dead) {
-          for (int X = 0; X < 2; ++X) {
-            if (ds.n[X] > 0) {
-              issue_qk(X, ring + pipe.stage * kTileBytes);
-              umma_commit(smem_u32(&ub->s_full[X]));
+        for (int j = 0; j < nX; ++j) {
+          const uint32_t pv = pos0 + 2 * j + 1, pk = pv + 1;
+          const bool more = j + 1 < nX;
+          const uint32_t g = g1 + min(j, nA) + min(j, nB) + ((X == 1 && j < nA) ? 1u : 0u);
+          v_descs(pv, vd);
+          k_descs(pk, kd);
+          wait_full(pv);
+          if (more) wait_full(pk);
+          wait_or_die(smem_u32(&ub->p_full[X][0]), ph_p);
+          tc_fence_after();
+          tr(12);
+          take_turn(g);
+          tr(19);
+          if (!dead) issue_pv_lo(vd, j > 0);
+          wait_or_die(smem_u32(&ub->p_full[X][1]), ph_p);  // second half of P
+          ph_p ^= 1u;
+          tc_fence_after();
+          if (!dead) {
+            issue_pv_hi(vd);
+            if (j == nX - 1) umma_commit(smem_u32(&ub->o_done[X]));
+            release(pv, j >= nY);
+            if (more) {
+              issue_qk(kd);
+              release(pk, j + 1 >= nY);
             }
           }
-          release(pipe.stage);
-        }
-        pipe.advance();
-        for (int j = 0; j < n_all; ++j) {
-          const int v_stage = pipe.stage;
-          const uint32_t v_phase = pipe.phase;
-          pipe.advance();
-          const int k_stage = pipe.stage;
-          const uint32_t k_phase = pipe.phase;
-          const bool more = j + 1 < n_all;
-          if (more) pipe.advance();
-          wait_or_die(smem_u32(&bars->full[v_stage]), v_phase);
-          bool k_ready = false;
-          for (int X = 0; X < 2; ++X) {
-            if (j < ds.n[X]) {
-              wait_or_die(smem_u32(&ub->p_full[X]), ph_p[X]);
-              ph_p[X] ^= 1u;
-              tc_fence_after();
-              if (!dead) {
-                issue_pv(X, ring + v_stage * kTileBytes, j > 0);
-                if (j == ds.n[X] - 1) umma_commit(smem_u32(&ub->o_done[X]));
-              }
-            }
-            if (X == 1 && !dead) release(v_stage);
-            if (more && !k_ready) {
-              wait_or_die(smem_u32(&bars->full[k_stage]), k_phase);
-              tc_fence_after();
-              k_ready = true;
-            }
-            if (j + 1 < ds.n[X] && !dead) {
-              issue_qk(X, ring + k_stage * kTileBytes);
-              umma_commit(smem_u32(&ub->s_full[X]));
-            }
-            if (X == 1 && more && !dead) release(k_stage);
-          }
+          pass_turn(g);
+          tr(16);
         }
       }
     }
@@ -485,6 +573,8 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
     Pipe pipe{0, 0};
     bool dead = false;
     uint32_t ph_s = 0, ph_o = 0;  // this warpgroup's s_full / o_done parities
+    Tracer tr;
+    tr.init(a, warp >> 2, (threadIdx.x & 127) == 0);
     const int X = warp >> 2;       // sub-tile this warpgroup owns on the tcgen05 path
     for (int ti = t_begin; ti < t_end; ++ti) {
       TaskView tv;
@@ -538,24 +628,21 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
         float m_ref = -INFINITY, l = 0.f;
         for (int j = 0; j < nX; ++j) {
           const int col0 = (tv.t.kt_lo + j) * kKeyTile;
-          if (!dead && !mbar_wait(smem_u32(&ub->s_full[X]), ph_s)) {
+          tr(20);
+          if (!dead && !mbar_wait(smem_u32(&ub->s_full[X]), ph_s, a.status)) {
             report_timeout(a);
             dead = true;
           }
           ph_s ^= 1u;
           tc_fence_after();
           uint32_t sr[128];
-          {
-            uint32_t(&c0)[32] = *reinterpret_cast<uint32_t(*)[32]>(&sr[0]);
-            uint32_t(&c1)[32] = *reinterpret_cast<uint32_t(*)[32]>(&sr[32]);
-            uint32_t(&c2)[32] = *reinterpret_cast<uint32_t(*)[32]>(&sr[64]);
-            uint32_t(&c3)[32] = *reinterpret_cast<uint32_t(*)[32]>(&sr[96]);
-            tmem_ld_32x32b_x32(t_s, c0);
-            tmem_ld_32x32b_x32(t_s + 32, c1);
-            tmem_ld_32x32b_x32(t_s + 64, c2);
-            tmem_ld_32x32b_x32(t_s + 96, c3);
-            tmem_wait_ld();
-          }
+          tmem_ld_32x32b_x32(t_s, &sr[0]);
+          tmem_ld_32x32b_x32(t_s + 32, &sr[32]);
+          tmem_ld_32x32b_x32(t_s + 64, &sr[64]);
+          tmem_ld_32x32b_x32(t_s + 96, &sr[96]);
+          tr(21);
+          tmem_wait_ld();
+          tr(22);
           const bool need_mask = tree ? (col0 + kKeyTile > h) : (col0 + kKeyTile > h + i_min + 1);
           if (need_mask) {
             const int frontier = h + i_row;  // last visible column of this row
@@ -583,9 +670,20 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
               if (!vis) sr[k] = 0xff800000u;  // -inf, selected (never added)
             }
           }
-          float mx = -INFINITY;
+          float mx;
+          {  // eight independent chains of three-input max, then a short tree
+            float m8[8];
 #pragma unroll
-          for (int k = 0; k < 128; ++k) mx = fmaxf(mx, __uint_as_float(sr[k]));
+            for (int q = 0; q < 8; ++q) m8[q] = fmaxf(__uint_as_float(sr[q]), __uint_as_float(sr[q + 8]));
+#pragma unroll
+            for (int k = 16; k < 128; k += 16) {
+#pragma unroll
+              for (int q = 0; q < 8; ++q)
+                m8[q] = max3(m8[q], __uint_as_float(sr[k + q]), __uint_as_float(sr[k + q + 8]));
+            }
+            mx = max3(max3(m8[0], m8[1], m8[2]), max3(m8[3], m8[4], m8[5]), fmaxf(m8[6], m8[7]));
+          }
+          tr(23);
           const float m_cand = fmaxf(m_ref, mx * scale_log2);
           bool need = false;
           if (j == 0 || m_ref == -INFINITY) {
@@ -609,30 +707,41 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
               tmem_st_32x32b_x32(t_o + c * 32, orow);
             }
           }
+          tr(24);
           const float neg_off = (m_ref == -INFINITY) ? 0.f : -m_ref;
-          float sum = 0.f;
-          uint32_t pk[64];
+          // P = 2^(s * scale - m), two keys packed per 32-bit column, written over sr in place.
+          // The scale-and-subtract and the row sum run as packed f32x2 instructions.
+          const uint64_t scale2 = pack_f32x2(scale_log2, scale_log2), off2 = pack_f32x2(neg_off, neg_off);
+          uint64_t sum2[4] = {0ull, 0ull, 0ull, 0ull};
 #pragma unroll
-          for (int k = 0; k < 64; ++k) {
-            const float p0 = ex2(fmaf(__uint_as_float(sr[2 * k]), scale_log2, neg_off));
-            const float p1 = ex2(fmaf(__uint_as_float(sr[2 * k + 1]), scale_log2, neg_off));
-            sum += p0 + p1;
-            pk[k] = pack_bf16(p0, p1);
-          }
-          l += sum;
-          {
-            uint32_t(&h0)[32] = *reinterpret_cast<uint32_t(*)[32]>(&pk[0]);
-            uint32_t(&h1)[32] = *reinterpret_cast<uint32_t(*)[32]>(&pk[32]);
-            tmem_st_32x32b_x32(t_s, h0);
-            tmem_st_32x32b_x32(t_s + 32, h1);
+          for (int half = 0; half < 2; ++half) {
+#pragma unroll
+            for (int k = half * 32; k < half * 32 + 32; ++k) {
+              float x0, x1;
+              unpack_f32x2(
+                  fma_f32x2(pack_f32x2(__uint_as_float(sr[2 * k]), __uint_as_float(sr[2 * k + 1])), scale2, off2), x0,
+                  x1);
+              const float p0 = ex2(x0), p1 = ex2(x1);
+              sum2[k & 3] = add_f32x2(sum2[k & 3], pack_f32x2(p0, p1));
+              sr[k] = pack_bf16(p0, p1);
+            }
+            // hand this half of P (64 keys, 32 columns) to the MMA issuer
+            tmem_st_32x32b_x32(t_s + half * 32, &sr[half * 32]);
             tmem_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ub->p_full[X][half]));
+            if (half == 0) tr(25);
           }
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&ub->p_full[X]));
+          {
+            float a0, a1;
+            unpack_f32x2(add_f32x2(add_f32x2(sum2[0], sum2[1]), add_f32x2(sum2[2], sum2[3])), a0, a1);
+            l += a0 + a1;
+          }
+          tr(26);
         }
         // ---- epilogue: O / l -> global
-        if (!dead && !mbar_wait(smem_u32(&ub->o_done[X]), ph_o)) {
+        if (!dead && !mbar_wait(smem_u32(&ub->o_done[X]), ph_o, a.status)) {
           report_timeout(a);
           dead = true;
         }
@@ -704,7 +813,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
           const bool work = active && col0 <= h + i_max;  // mask-aware skip (Section 4.2.2)
           float s[16][4];
           uint32_t p[8][4];
-          if (!dead && !mbar_wait(smem_u32(&bars->full[pipe.stage]), pipe.phase)) {
+          if (!dead && !mbar_wait(smem_u32(&bars->full[pipe.stage]), pipe.phase, a.status)) {
             report_timeout(a);
             dead = true;
           }
@@ -716,7 +825,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
             const bool need_mask = tree ? (col0 + kKeyTile > h) : (col0 + kKeyTile > h + i_min + 1);
             w.softmax(a, tv.rq, s, p, col0, i_lo, i_hi, need_mask, scale_log2, lane);
           }
-          if (!dead && !mbar_wait(smem_u32(&bars->full[pipe.stage]), pipe.phase)) {
+          if (!dead && !mbar_wait(smem_u32(&bars->full[pipe.stage]), pipe.phase, a.status)) {
             report_timeout(a);
             dead = true;
           }
@@ -758,7 +867,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
           const bool work = col0 <= h + i_max;
           float s[2][4];
           uint32_t p[1][4];
-          if (!dead && !mbar_wait(smem_u32(&bars->full[pipe.stage]), pipe.phase)) {
+          if (!dead && !mbar_wait(smem_u32(&bars->full[pipe.stage]), pipe.phase, a.status)) {
             report_timeout(a);
             dead = true;
           }
@@ -770,7 +879,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
             const bool need_mask = tree ? (col0 + 16 > h) : (col0 + 16 > h + tv.t.tok0 + 1);
             w.softmax(a, tv.rq, s, p, col0, i_lo, i_hi, need_mask, scale_log2, lane);
           }
-          if (!dead && !mbar_wait(smem_u32(&bars->full[pipe.stage]), pipe.phase)) {
+          if (!dead && !mbar_wait(smem_u32(&bars->full[pipe.stage]), pipe.phase, a.status)) {
             report_timeout(a);
             dead = true;
           }

@@ -11,7 +11,9 @@ namespace xy {
 
 constexpr int kHeadDim = 128;
 constexpr int kKeyTile = 128;      // keys per KV tile (one MMA N extent)
-constexpr int kStreamRowsMax = 16; // packed rows a streaming task may hold
+constexpr int kStreamRowsMax = 16;
+constexpr int kTraceRoles = 4;      // sub-tile A, sub-tile B, MMA issuer, producer (worker 0 only)
+constexpr int kTraceLen = 2048; // packed rows a streaming task may hold
 
 // Per-request facts the kernels need (device-visible, 32 bytes).
 struct ReqInfo {
@@ -66,6 +68,7 @@ struct RunArgs {
   float* o_part;
   float* lse_part;
   int32_t* status;
+  unsigned long long* trace;  // null unless tracing: kTraceRoles x kTraceLen (tag << 48 | cycle) records
   int32_t num_q_heads, num_kv_heads, page_size, page_shift;
 };
 

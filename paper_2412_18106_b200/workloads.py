@@ -229,12 +229,23 @@ def config5_full_mix(seed: int = 0, num_requests: int = 96) -> Batch:
     return assemble("full_mix", 64, 8, 128, q_len, kv_len, kind, trees, rng, seed)
 
 
+def prefill_prefix(seed: int = 0, num_requests: int = 4, q_tokens: int = 4096) -> Batch:
+    """Prefill on a reused prefix (shape of the paper's Section 6.2.1 sweep): prompts of
+    `q_tokens` new tokens on cached prefixes drawn token by token from [0, 4096].  32/8 heads,
+    page 128.  Not one of the five benchmark configurations; used to tune the dense path."""
+    rng = np.random.default_rng(seed)
+    kv = [int(x) for x in rng.integers(0, 4097, size=num_requests)]
+    R = num_requests
+    return assemble("prefill_prefix", 32, 8, 128, [q_tokens] * R, kv, [MASK_CAUSAL] * R, [None] * R, rng, seed)
+
+
 CONFIGS = {
     "tiny_hybrid": config1_tiny,
     "decode_only": config2_decode,
     "splitfuse_mix": config3_splitfuse,
     "verify_trees": config4_verify,
     "full_mix": config5_full_mix,
+    "prefill_prefix": prefill_prefix,
 }
 
 
