@@ -172,6 +172,33 @@ int xy_attn_run(xy_attn_ctx* ctx, const void* q, int64_t q_token_stride, const v
 int xy_attn_merge(const float* o_part, const float* lse_part, int32_t num_splits, int64_t rows,
                   int32_t head_dim, void* o, float* lse, void* stream);
 
+/* Allocation-free decode attention.  The paper has no counterpart for this call: it exists
+ * for callers that cannot allocate device memory where they need attention - a serving loop
+ * whose memory pool is already handed out in full, a plugin that is given only a stream and
+ * its buffers, a program that must keep away from the allocator while another library owns
+ * it.  It computes the same result as xy_attn_run for a batch of decode requests (one new
+ * token each, causal): request r attends to its kv_len[r] cached tokens plus the new token,
+ * whose K/V is already in the cache.  No context is needed and nothing is allocated or freed,
+ * on the device or through any library: the split-KV scratch is a fixed array inside the
+ * library image, XY_ATTN_STATIC_MAX_ROWS rows of 129 floats (about 4.03 MiB), which every GPU
+ * that loads the library holds until the process exits.
+ *   q, k_pool, v_pool, block_table, o, lse: as for xy_attn_run (token r of q / o / lse is request r)
+ *   kv_len      DEVICE int32 [num_reqs]: cached tokens before the new one
+ *   max_kv_len  HOST value, >= every kv_len[r]; sets the number of 2048-key chunks
+ * Limit: num_reqs * num_q_heads * ceil((max_kv_len + 1) / 2048) <= XY_ATTN_STATIC_MAX_ROWS;
+ * beyond it the call returns XY_ERR_CAPACITY (and prints one line to stderr) without launching.
+ * The first call on each device looks up the scratch's device address; make that first call
+ * outside any stream capture.  All calls share the one scratch array and every call rewrites
+ * the part it reads, so nothing needs clearing between calls, but two calls whose kernels can
+ * overlap on the GPU (different streams, no ordering between them) race on it: order them. */
+#define XY_ATTN_STATIC_MAX_ROWS 8192
+int xy_attn_decode_static(const void* q, int64_t q_token_stride, const void* k_pool, const void* v_pool,
+                          int64_t page_stride, int64_t head_stride, int64_t token_stride,
+                          const int32_t* block_table, int32_t block_table_stride,
+                          const int32_t* kv_len /*DEVICE*/, int32_t num_reqs, int32_t max_kv_len,
+                          int32_t num_q_heads, int32_t num_kv_heads, int32_t page_size, float sm_scale,
+                          void* o, int64_t o_token_stride, float* lse, void* stream);
+
 /* Debug/verification: copy the K and V rows a request sees, in logical order,
  * through the block table: out_k/out_v DEVICE bf16 [kv_len+q_len, D] for kv head
  * `kv_head` of planned request `req`. */

@@ -73,7 +73,7 @@ EXPORTS = (
     "xy_attn_debug_gather", "xy_attn_get_tasks", "xy_attn_get_worker_offsets",
     "xy_attn_get_merge_units", "xy_attn_get_tree_mask", "xy_attn_get_q_start",
     "xy_attn_last_launches", "xy_attn_last_error", "xy_attn_device_status",
-    "xy_attn_set_timing", "xy_attn_get_timing", "xy_attn_debug_trace",
+    "xy_attn_set_timing", "xy_attn_get_timing", "xy_attn_debug_trace", "xy_attn_decode_static",
 )
 
 _lib = None
@@ -104,6 +104,8 @@ def load() -> ctypes.CDLL:
     L.xy_attn_get_timing.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float),
                                      ctypes.POINTER(i32)]
     L.xy_attn_debug_trace.argtypes = [vp, vp, i32]
+    L.xy_attn_decode_static.argtypes = [vp, i64, vp, vp, i64, i64, i64, vp, i32, vp, i32, i32, i32, i32, i32,
+                                        ctypes.c_float, vp, i64, vp, vp]
     L.xy_attn_last_launches.argtypes = [vp]
     L.xy_attn_last_error.argtypes = [vp]
     L.xy_attn_last_error.restype = ctypes.c_char_p
@@ -269,6 +271,27 @@ def xy_attn_merge(o_part: torch.Tensor, lse_part: torch.Tensor, o: torch.Tensor,
                          lse.data_ptr(), _stream_ptr(stream))
     if rc != XY_OK:
         raise XYAttnError(rc, "xy_attn_merge failed")
+
+
+XY_ATTN_STATIC_MAX_ROWS = 8192
+
+
+def xy_attn_decode_static(q, k_pool, v_pool, block_table, kv_len, max_kv_len: int, sm_scale: float, o, lse,
+                          stream=None) -> int:
+    """Decode attention for callers that cannot allocate device memory (a full memory pool, a
+    plugin that only owns its buffers): no context, no cudaMalloc; the split-KV scratch is a
+    fixed array inside the library.  q / o bf16 [R, Hq, 128], lse fp32 [R, Hq], kv_len int32 [R]
+    on the device.  Returns the C status code (XY_ERR_CAPACITY beyond the scratch's limit).
+    Calls that may overlap on the GPU share the scratch and must be ordered by the caller."""
+    L = load()
+    for t in (q, k_pool, v_pool, block_table, kv_len, o, lse):
+        if not t.is_cuda:
+            raise XYAttnError(XY_ERR_INVALID_ARG, "xy_attn_decode_static needs CUDA tensors")
+    return int(L.xy_attn_decode_static(
+        q.data_ptr(), q.stride(0), k_pool.data_ptr(), v_pool.data_ptr(), k_pool.stride(0), k_pool.stride(1),
+        k_pool.stride(2), block_table.data_ptr(), block_table.stride(0), kv_len.data_ptr(), q.shape[0],
+        int(max_kv_len), q.shape[1], k_pool.shape[1], k_pool.shape[2], float(sm_scale), o.data_ptr(),
+        o.stride(0), lse.data_ptr(), _stream_ptr(stream)))
 
 
 def attention(ctx: XYAttn, batch, q, k_pool, v_pool, block_table, sm_scale, o=None, lse=None,
