@@ -287,7 +287,7 @@ int xy_attn_run(xy_attn_ctx* ctx, const void* q, int64_t q_token_stride, const v
   if (cfg.kernel == XY_KERNEL_REFERENCE) {
     XY_CUDA(ctx, launch_reference(a, ctx->num_workers, s));
   } else {
-    XY_CUDA(ctx, launch_meta(a, ctx->num_workers, num_pages, cfg.kernel == XY_KERNEL_AUTO, s));
+    XY_CUDA(ctx, launch_meta(a, ctx->num_workers, num_pages, cfg.kernel == XY_KERNEL_AUTO && p.info.num_dense_tasks > 0, s));
   }
   ctx->last_launches += 1;
   if (timed) XY_CUDA(ctx, cudaEventRecord(ctx->events[3 * ctx->timed_runs + 1], s));

@@ -90,14 +90,15 @@ __global__ void __launch_bounds__(128) ref_attention_kernel(RunArgs a) {
 }
 
 // Cross-task form of the Update stage (Section 4.2.1): combine the partials of every tile
-// unit whose KV range was split.  One block per merge unit, one warp per packed row.
+// unit whose KV range was split.  kMergeSlices blocks per merge unit, one warp per packed row.
+constexpr int kMergeSlices = 8;
 __global__ void __launch_bounds__(128) merge_units_kernel(MergeArgs a) {
   const xy_attn_merge_unit u = a.units[blockIdx.x];
   const ReqInfo rq = a.reqs[u.req];
   const int G = a.num_q_heads / a.num_kv_heads;
   const int rows = u.ntok * G;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (int x = warp; x < rows; x += 4) {
+  for (int x = blockIdx.y * 4 + warp; x < rows; x += 4 * kMergeSlices) {
     float mx = -INFINITY;
     for (int c = 0; c < u.nsplit; ++c) mx = fmaxf(mx, a.lse_part[u.part0 + c * rows + x]);
     float z = 0.f;
@@ -185,7 +186,7 @@ cudaError_t launch_reference(const RunArgs& a, int num_workers, cudaStream_t s) 
 
 cudaError_t launch_merge_units(const MergeArgs& a, int num_units, cudaStream_t s) {
   if (num_units == 0) return cudaSuccess;
-  merge_units_kernel<<<num_units, 128, 0, s>>>(a);
+  merge_units_kernel<<<dim3(num_units, kMergeSlices), 128, 0, s>>>(a);
   return cudaGetLastError();
 }
 

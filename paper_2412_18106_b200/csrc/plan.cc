@@ -23,6 +23,10 @@ constexpr float kDenseVisitUs = 0.92f;   // one 128-row sub-tile against 128 key
 constexpr float kStreamVisitUs = 1.50f;  // 64 KiB of K+V at an even share of HBM bandwidth
 constexpr float kTaskFixedUs = 1.5f;     // Q load, pipeline fill, epilogue
 constexpr int kMinChunkTiles = 4;
+// A task may cost at most this fraction of the mean per-worker load before its KV range is
+// split (measured on the five benchmark batches: finer splits lose more to per-task overhead
+// and partial traffic than they gain in balance).
+constexpr float kTaskCapFraction = 0.77f;
 
 struct Unit {
   int32_t req, kv_head, tok0, ntok, kind;
@@ -174,7 +178,7 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
   const int max_splits = cfg.max_splits > 0 ? cfg.max_splits : 32;
   double total_cost = 0.0;
   for (const Unit& u : units) total_cost += kTaskFixedUs + u.visit_cost * u.nkt;
-  float cap = static_cast<float>(total_cost / std::max(1, num_workers) / 4.0);
+  float cap = static_cast<float>(total_cost / std::max(1, num_workers) * kTaskCapFraction);
   std::vector<int> chunk_tiles(units.size(), 0);
   for (int attempt = 0; attempt < 64; ++attempt) {
     int64_t prow = 0;
