@@ -207,7 +207,9 @@ int xy_attn_debug_gather(xy_attn_ctx* ctx, int32_t req, int32_t kv_head, const v
                          int64_t token_stride, const int32_t* block_table,
                          int32_t block_table_stride, void* out_k, void* out_v, void* stream);
 
-/* Debug tracing.  When the environment variable XY_ATTN_TRACE=1 is set at create time, the
+/* Debug tracing (only in a library built with -DXY_ENABLE_TRACE, i.e. XY_BUILD_TRACE=1 for
+ * paper_2412_18106_b200.build; otherwise no records are written and 0 entries are meaningful).
+ * When the environment variable XY_ATTN_TRACE=1 is set at create time, the
  * roles of worker 0 (sub-tile A, sub-tile B, MMA issuer, producer) stamp (tag << 48 | SM cycle
  * counter) records into a context-owned buffer of 4 x 2048 entries per run.  This call
  * synchronises the device and copies them to `out` (HOST); it returns the number of entries

@@ -242,8 +242,10 @@ __device__ __forceinline__ void write_lse(const RunArgs& a, const TaskView& tv, 
   }
 }
 
-// Debug trace of worker 0: one record per call, (tag << 48) | SM cycle counter.
+// Debug trace of worker 0: one record per call, (tag << 48) | SM cycle counter.  Compiled in
+// only with -DXY_ENABLE_TRACE (the stamps cost issue slots on the critical path).
 struct Tracer {
+#ifdef XY_ENABLE_TRACE
   unsigned long long* p;
   int n;
   __device__ __forceinline__ void init(const RunArgs& a, int role, bool on) {
@@ -253,6 +255,10 @@ struct Tracer {
   __device__ __forceinline__ void operator()(unsigned tag) {
     if (p != nullptr && n < kTraceLen) p[n++] = (static_cast<unsigned long long>(tag) << 48) | (clock64() & 0xFFFFFFFFFFFFull);
   }
+#else
+  __device__ __forceinline__ void init(const RunArgs&, int, bool) {}
+  __device__ __forceinline__ void operator()(unsigned) {}
+#endif
 };
 
 __device__ __forceinline__ void report_timeout(const RunArgs& a) {
