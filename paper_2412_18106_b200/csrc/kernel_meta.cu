@@ -38,6 +38,7 @@ constexpr int kStages = 4;
 constexpr int kTileBytes = 32768;  // 2 halves x 128 rows x 128 B
 constexpr int kHalfBytes = 16384;
 constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kRescaleThresholdWarp = 8.0f;  // log2 units, warp-level MMA paths
 constexpr float kLn2 = 0.6931471805599453f;
 
 struct __align__(8) SmemBarriers {
@@ -116,6 +117,34 @@ struct WarpTile {
 
   // S = Q K^T for this warp's keys; returns scores (raw dot products) in s.
   __device__ __forceinline__ void qk(uint32_t k_smem, int koff, int lane, float (&s)[NT][4]) {
+    if constexpr (NT == 2 && KEEPQ) {
+      // Streaming tile: all eight K fragments are fetched first (one shared-memory latency
+      // instead of eight), and even / odd k-steps accumulate separately so that the MMAs form
+      // four chains of four instead of two chains of eight.
+      const int mi = lane >> 3;
+      const uint32_t key = koff + (lane & 7) + (mi >> 1) * 8;
+      uint32_t kb[8][4];
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks)
+        ldmatrix_x4(k_smem + swz(key, ks * 2 + (mi & 1)), kb[ks][0], kb[ks][1], kb[ks][2], kb[ks][3]);
+      float t[2][4];
+#pragma unroll
+      for (int n = 0; n < 2; ++n)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) s[n][e] = t[n][e] = 0.f;
+#pragma unroll
+      for (int ks = 0; ks < 8; ks += 2) {
+        mma_bf16_16816(s[0], qf[ks], kb[ks][0], kb[ks][1]);
+        mma_bf16_16816(s[1], qf[ks], kb[ks][2], kb[ks][3]);
+        mma_bf16_16816(t[0], qf[ks + 1], kb[ks + 1][0], kb[ks + 1][1]);
+        mma_bf16_16816(t[1], qf[ks + 1], kb[ks + 1][2], kb[ks + 1][3]);
+      }
+#pragma unroll
+      for (int n = 0; n < 2; ++n)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) s[n][e] += t[n][e];
+      return;
+    }
 #pragma unroll
     for (int n = 0; n < NT; ++n)
 #pragma unroll
@@ -163,11 +192,27 @@ struct WarpTile {
     mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
     mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
     const float mn_lo = fmaxf(m_lo, mx_lo), mn_hi = fmaxf(m_hi, mx_hi);
-    const float use_lo = (mn_lo == -INFINITY) ? 0.f : mn_lo;
-    const float use_hi = (mn_hi == -INFINITY) ? 0.f : mn_hi;
-    const float al_lo = ex2(m_lo - use_lo), al_hi = ex2(m_hi - use_hi);
-    m_lo = mn_lo;
-    m_hi = mn_hi;
+    // Lazy Update: the reference moves (and O, l are rescaled) only when some row of the warp
+    // would otherwise exceed it by more than 2^kRescaleThresholdWarp, or has no reference yet.
+    const bool grow = (mn_lo - m_lo > kRescaleThresholdWarp) || (mn_hi - m_hi > kRescaleThresholdWarp) ||
+                      (m_lo == -INFINITY && mn_lo != -INFINITY) || (m_hi == -INFINITY && mn_hi != -INFINITY);
+    if (__any_sync(0xffffffffu, grow)) {
+      const float u_lo = (mn_lo == -INFINITY) ? 0.f : mn_lo, u_hi = (mn_hi == -INFINITY) ? 0.f : mn_hi;
+      const float al_lo = ex2(m_lo - u_lo), al_hi = ex2(m_hi - u_hi);
+      m_lo = mn_lo;
+      m_hi = mn_hi;
+      l_lo *= al_lo;
+      l_hi *= al_hi;
+#pragma unroll
+      for (int n = 0; n < 16; ++n) {
+        o[n][0] *= al_lo;
+        o[n][1] *= al_lo;
+        o[n][2] *= al_hi;
+        o[n][3] *= al_hi;
+      }
+    }
+    const float use_lo = (m_lo == -INFINITY) ? 0.f : m_lo;
+    const float use_hi = (m_hi == -INFINITY) ? 0.f : m_hi;
     float sum_lo = 0.f, sum_hi = 0.f;
 #pragma unroll
     for (int n = 0; n < NT; ++n) {
@@ -179,20 +224,26 @@ struct WarpTile {
       p[n >> 1][(n & 1) * 2 + 0] = pack_bf16(p0, p1);
       p[n >> 1][(n & 1) * 2 + 1] = pack_bf16(p2, p3);
     }
-    l_lo = l_lo * al_lo + sum_lo;
-    l_hi = l_hi * al_hi + sum_hi;
-#pragma unroll
-    for (int n = 0; n < 16; ++n) {
-      o[n][0] *= al_lo;
-      o[n][1] *= al_lo;
-      o[n][2] *= al_hi;
-      o[n][3] *= al_hi;
-    }
+    l_lo += sum_lo;
+    l_hi += sum_hi;
   }
 
   // O += P V for this warp's keys.
   __device__ __forceinline__ void pv(uint32_t v_smem, int koff, int lane, const uint32_t (&p)[NT / 2][4]) {
     const int mi = lane >> 3;
+    if constexpr (NT == 2 && KEEPQ) {  // streaming tile: fetch the eight V fragments, then 16 MMAs
+      const uint32_t key = koff + (lane & 7) + (mi & 1) * 8;
+      uint32_t vb[8][4];
+#pragma unroll
+      for (int dp = 0; dp < 8; ++dp)
+        ldmatrix_x4_trans(v_smem + swz(key, dp * 2 + (mi >> 1)), vb[dp][0], vb[dp][1], vb[dp][2], vb[dp][3]);
+#pragma unroll
+      for (int dp = 0; dp < 8; ++dp) {
+        mma_bf16_16816(o[2 * dp], p[0], vb[dp][0], vb[dp][1]);
+        mma_bf16_16816(o[2 * dp + 1], p[0], vb[dp][2], vb[dp][3]);
+      }
+      return;
+    }
 #pragma unroll
     for (int kk = 0; kk < NT / 2; ++kk) {
       const uint32_t key = koff + kk * 16 + (lane & 7) + (mi & 1) * 8;
