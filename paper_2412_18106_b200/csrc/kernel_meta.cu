@@ -117,7 +117,7 @@ struct WarpTile {
 
   // S = Q K^T for this warp's keys; returns scores (raw dot products) in s.
   __device__ __forceinline__ void qk(uint32_t k_smem, int koff, int lane, float (&s)[NT][4]) {
-    if constexpr (NT == 2 && KEEPQ) {
+    if constexpr (NT == 2) {
       // Streaming tile: all eight K fragments are fetched first (one shared-memory latency
       // instead of eight), and even / odd k-steps accumulate separately so that the MMAs form
       // four chains of four instead of two chains of eight.
@@ -127,6 +127,15 @@ struct WarpTile {
 #pragma unroll
       for (int ks = 0; ks < 8; ++ks)
         ldmatrix_x4(k_smem + swz(key, ks * 2 + (mi & 1)), kb[ks][0], kb[ks][1], kb[ks][2], kb[ks][3]);
+      uint32_t qq[8][4];
+      if constexpr (!KEEPQ) {
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          const uint32_t ch = ks * 2 + q_hi;
+          ldmatrix_x4(q_addr + (ch >> 3) * kHalfBytes + (((ch & 7u) ^ q_row7) << 4), qq[ks][0], qq[ks][1],
+                      qq[ks][2], qq[ks][3]);
+        }
+      }
       float t[2][4];
 #pragma unroll
       for (int n = 0; n < 2; ++n)
@@ -134,10 +143,12 @@ struct WarpTile {
         for (int e = 0; e < 4; ++e) s[n][e] = t[n][e] = 0.f;
 #pragma unroll
       for (int ks = 0; ks < 8; ks += 2) {
-        mma_bf16_16816(s[0], qf[ks], kb[ks][0], kb[ks][1]);
-        mma_bf16_16816(s[1], qf[ks], kb[ks][2], kb[ks][3]);
-        mma_bf16_16816(t[0], qf[ks + 1], kb[ks + 1][0], kb[ks + 1][1]);
-        mma_bf16_16816(t[1], qf[ks + 1], kb[ks + 1][2], kb[ks + 1][3]);
+        const uint32_t(&qa)[4] = KEEPQ ? qf[KEEPQ ? ks : 0] : qq[ks];
+        const uint32_t(&qb)[4] = KEEPQ ? qf[KEEPQ ? ks + 1 : 0] : qq[ks + 1];
+        mma_bf16_16816(s[0], qa, kb[ks][0], kb[ks][1]);
+        mma_bf16_16816(s[1], qa, kb[ks][2], kb[ks][3]);
+        mma_bf16_16816(t[0], qb, kb[ks + 1][0], kb[ks + 1][1]);
+        mma_bf16_16816(t[1], qb, kb[ks + 1][2], kb[ks + 1][3]);
       }
 #pragma unroll
       for (int n = 0; n < 2; ++n)
@@ -231,7 +242,7 @@ struct WarpTile {
   // O += P V for this warp's keys.
   __device__ __forceinline__ void pv(uint32_t v_smem, int koff, int lane, const uint32_t (&p)[NT / 2][4]) {
     const int mi = lane >> 3;
-    if constexpr (NT == 2 && KEEPQ) {  // streaming tile: fetch the eight V fragments, then 16 MMAs
+    if constexpr (NT == 2) {  // streaming tile: fetch the eight V fragments, then 16 MMAs
       const uint32_t key = koff + (lane & 7) + (mi & 1) * 8;
       uint32_t vb[8][4];
 #pragma unroll
@@ -913,7 +924,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
       } else {
         // ---------------- streaming: this warp owns keys koff .. koff+15 of every tile ----
         const int koff = warp * 16;
-        WarpTile<2, true> w;
+        WarpTile<2, false> w;
         w.init();
         w.load_q(q_smem, 0, lane);
         const int r_lo = min(lane >> 2, tv.rows - 1), r_hi = min((lane >> 2) + 8, tv.rows - 1);
