@@ -447,46 +447,94 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
       tr.init(a, 3, true);
       const int ppt = kKeyTile >> a.page_shift;  // pages per 128-key tile
       const uint32_t page_bytes = static_cast<uint32_t>(a.page_size) * 128u;
-      for (int ti = t_begin; ti < t_end && !dead; ++ti) {
-        const xy_attn_task t = a.tasks[ti];
-        const ReqInfo rq = a.reqs[t.req];
-        const int npages = (rq.kv_len + rq.q_len + a.page_size - 1) >> a.page_shift;
-        const int32_t* bt = a.block_table + static_cast<int64_t>(t.req) * a.bt_stride;
-        const bool by_umma = kUmma && t.kind == 0;
-        for (int kt = t.kt_lo; kt < t.kt_hi && !dead; ++kt) {
-          for (int op = 0; op < 2; ++op) {
-            const uint32_t bit = 1u << pipe.stage;
-            if (used & bit) {
-              bool ok;
-              if (last_umma & bit) {
-                ok = mbar_wait(smem_u32(&bars->empty_umma[pipe.stage]), (ph_umma >> pipe.stage) & 1u, a.status);
-                ph_umma ^= bit;
-              } else {
-                ok = mbar_wait(smem_u32(&bars->empty[pipe.stage]), (ph_cons >> pipe.stage) & 1u, a.status);
-                ph_cons ^= bit;
-              }
-              if (!ok) {
-                report_timeout(a);
-                dead = true;
-                break;
-              }
-            }
-            used |= bit;
-            last_umma = by_umma ? (last_umma | bit) : (last_umma & ~bit);
-            tr(1 + op);
-            const uint32_t full = smem_u32(&bars->full[pipe.stage]);
-            mbar_arrive_expect_tx(full, kTileBytes);
-            const uint32_t dst = ring + pipe.stage * kTileBytes;
-            const CUtensorMap* map = op == 0 ? &k_map : &v_map;
-            for (int p = 0; p < ppt; ++p) {
-              const int pi = min(kt * ppt + p, npages - 1);  // pages past the end: reload the last
-              const int page = __ldg(bt + pi);
-              tma_load_4d(dst + p * page_bytes, map, full, 0, 0, t.kv_head, page);
-              tma_load_4d(dst + kHalfBytes + p * page_bytes, map, full, 64, 0, t.kv_head, page);
-            }
-            pipe.advance();
+      // Fill one stage (the K or the V tile) once its previous reader has released it.
+      auto fill = [&](int op, bool by_umma, int kv_head, int kt, const int32_t* bt, int npages, int page0) {
+        const uint32_t bit = 1u << pipe.stage;
+        if (used & bit) {
+          bool ok;
+          if (last_umma & bit) {
+            ok = mbar_wait(smem_u32(&bars->empty_umma[pipe.stage]), (ph_umma >> pipe.stage) & 1u, a.status);
+            ph_umma ^= bit;
+          } else {
+            ok = mbar_wait(smem_u32(&bars->empty[pipe.stage]), (ph_cons >> pipe.stage) & 1u, a.status);
+            ph_cons ^= bit;
+          }
+          if (!ok) {
+            report_timeout(a);
+            dead = true;
+            return;
           }
         }
+        used |= bit;
+        last_umma = by_umma ? (last_umma | bit) : (last_umma & ~bit);
+        tr(1 + op);
+        const uint32_t full = smem_u32(&bars->full[pipe.stage]);
+        mbar_arrive_expect_tx(full, kTileBytes);
+        const uint32_t dst = ring + pipe.stage * kTileBytes;
+        const CUtensorMap* map = op == 0 ? &k_map : &v_map;
+        if (ppt == 1) {
+          tma_load_4d(dst, map, full, 0, 0, kv_head, page0);
+          tma_load_4d(dst + kHalfBytes, map, full, 64, 0, kv_head, page0);
+        } else {
+          for (int p = 0; p < ppt; ++p) {
+            const int pi = min(kt * ppt + p, npages - 1);  // pages past the end: reload the last
+            const int page = __ldg(bt + pi);
+            tma_load_4d(dst + p * page_bytes, map, full, 0, 0, kv_head, page);
+            tma_load_4d(dst + kHalfBytes + p * page_bytes, map, full, 64, 0, kv_head, page);
+          }
+        }
+        pipe.advance();
+      };
+      // A cursor over the worker's (task, key tile) sequence.  The block-table entry of a tile is
+      // requested three tiles before the tile is issued, so its global-memory latency (and the
+      // task / request loads at a task boundary) never sits between a stage's release and its
+      // TMA: that latency would otherwise add to every refill of the ring.
+      struct Tile {
+        const int32_t* bt;
+        int kv_head, kt, npages, page;
+        bool by_umma, valid;
+      };
+      int f_ti = t_begin, f_kt = 0, f_hi = 0, f_head = 0, f_npages = 1;
+      const int32_t* f_bt = a.block_table;
+      bool f_umma = false, f_open = false;
+      auto next_tile = [&]() {
+        Tile x;
+        x.valid = false;
+        x.bt = f_bt;
+        x.kv_head = x.kt = x.page = 0;
+        x.npages = 1;
+        x.by_umma = false;
+        while (!f_open || f_kt >= f_hi) {
+          if (f_open) ++f_ti;
+          if (f_ti >= t_end) return x;
+          const xy_attn_task t = a.tasks[f_ti];
+          const ReqInfo rq = a.reqs[t.req];
+          f_kt = t.kt_lo;
+          f_hi = t.kt_hi;
+          f_head = t.kv_head;
+          f_npages = (rq.kv_len + rq.q_len + a.page_size - 1) >> a.page_shift;
+          f_bt = a.block_table + static_cast<int64_t>(t.req) * a.bt_stride;
+          f_umma = kUmma && t.kind == 0;
+          f_open = true;
+        }
+        x.valid = true;
+        x.bt = f_bt;
+        x.kv_head = f_head;
+        x.kt = f_kt;
+        x.npages = f_npages;
+        x.by_umma = f_umma;
+        x.page = __ldg(f_bt + min(f_kt * ppt, f_npages - 1));  // consumed three tiles later
+        ++f_kt;
+        return x;
+      };
+      Tile q0 = next_tile(), q1 = next_tile(), q2 = next_tile();
+      while (q0.valid && !dead) {
+        const Tile cur = q0;
+        q0 = q1;
+        q1 = q2;
+        q2 = next_tile();
+        fill(0, cur.by_umma, cur.kv_head, cur.kt, cur.bt, cur.npages, cur.page);
+        if (!dead) fill(1, cur.by_umma, cur.kv_head, cur.kt, cur.bt, cur.npages, cur.page);
       }
     } else if (kUmma && (warp == kConsumerWarps + 1 || warp == kConsumerWarps + 2) && lane == 0) {
       // ================================ tcgen05 MMA issuers =============================
