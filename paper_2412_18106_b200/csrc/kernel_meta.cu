@@ -447,6 +447,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
       tr.init(a, 3, true);
       const int ppt = kKeyTile >> a.page_shift;  // pages per 128-key tile
       const uint32_t page_bytes = static_cast<uint32_t>(a.page_size) * 128u;
+      const uint64_t pol_stream = make_l2_policy_evict_first(), pol_keep = make_l2_policy_evict_last();
       // Fill one stage (the K or the V tile) once its previous reader has released it.
       auto fill = [&](int op, bool by_umma, int kv_head, int kt, const int32_t* bt, int npages, int page0) {
         const uint32_t bit = 1u << pipe.stage;
@@ -473,8 +474,11 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
         const uint32_t dst = ring + pipe.stage * kTileBytes;
         const CUtensorMap* map = op == 0 ? &k_map : &v_map;
         if (ppt == 1) {
-          tma_load_4d(dst, map, full, 0, 0, kv_head, page0);
-          tma_load_4d(dst + kHalfBytes, map, full, 64, 0, kv_head, page0);
+          // K/V of streaming tasks is read once: mark it evict-first in L2 so that it does not
+          // push out the K/V that the q tiles of a prefill share through L2 (kept evict-last).
+          const uint64_t pol = by_umma ? pol_keep : pol_stream;
+          tma_load_4d_hint(dst, map, full, 0, 0, kv_head, page0, pol);
+          tma_load_4d_hint(dst + kHalfBytes, map, full, 64, 0, kv_head, page0, pol);
         } else {
           for (int p = 0; p < ppt; ++p) {
             const int pi = min(kt * ppt + p, npages - 1);  // pages past the end: reload the last

@@ -19,9 +19,13 @@ namespace xy {
 namespace {
 
 // Per-SM time model in microseconds (free design constants; parity does not depend on them).
-constexpr float kDenseVisitUs = 0.92f;   // one 128-row sub-tile against 128 keys on the tensor pipe
-constexpr float kStreamVisitUs = 1.50f;  // 64 KiB of K+V at an even share of HBM bandwidth
-constexpr float kTaskFixedUs = 1.5f;     // Q load, pipeline fill, epilogue
+// Measured on B200 with the cycle-stamp trace: a dense task advances one key tile per ~3400
+// cycles whether one or both of its 128-row sub-tiles are in use (the softmax -> MMA chain of a
+// sub-tile sets the pace and the two sub-tiles overlap each other); a streaming task one key tile
+// per ~2700 cycles; a task boundary costs ~6000 cycles (Q load, pipeline refill, epilogue).
+constexpr float kDenseVisitUs = 1.80f;
+constexpr float kStreamVisitUs = 1.40f;
+constexpr float kTaskFixedUs = 3.0f;
 constexpr int kMinChunkTiles = 4;
 // A task may cost at most this fraction of the mean per-worker load before its KV range is
 // split (measured on the five benchmark batches: finer splits lose more to per-task overhead
@@ -164,9 +168,7 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
         if (u.kind == 1) {
           u.visit_cost = kStreamVisitUs;
         } else {
-          const int subtiles = ceil_div(rows, 128);
-          const float bytes_us = kStreamVisitUs / static_cast<float>(tiles.size());
-          u.visit_cost = std::max(kDenseVisitUs * subtiles, bytes_us);
+          u.visit_cost = kDenseVisitUs * static_cast<float>(std::max(1, ceil_div(rows, 256)));
         }
         u.paper_load = static_cast<float>(rows) * static_cast<float>(visible);
         units.push_back(u);
