@@ -5,9 +5,10 @@
 One step = one pass of the whole hot path (attention kernel + split-KV merge) over one
 synthetic hybrid batch.  Prints ONE JSON line.  `value` is useful TFLOP/s (masked-out work
 excluded) with inputs resident in HBM; `kv_gbs` is K+V GB/s of the same runs; `e2e` repeats
-the measurement through the public API with the step's inputs (Q, block table, request
-table) coming from pinned host memory and O / LSE read back, host-side planning included.
-The KV cache itself is device-resident state, as in serving.
+the measurement through the public API with the step's inputs (the fused QKV of the new
+tokens, block table, request table) coming from pinned host memory, the new K/V appended to
+the paged cache, and O / LSE read back, host-side planning included.  The cached history is
+device-resident state, as in serving.
 
 `--impl reference` times the fp64 CPU oracle (as it stands) on a bounded sample of the same
 workload on the host cores.
@@ -272,7 +273,7 @@ def main():
     # weak scaling: every rank serves its own batch of the same recipe (independent requests,
     # no exchange on the data path)
     batch = W.CONFIGS[args.workload](seed=rank)
-    tensors = W.make_tensors(batch)
+    tensors = W.make_tensors(batch, fused_qkv=True)  # Q is read with a stride from [T, Hq + 2 Hkv, D]
     kernel = {"auto": xb.XY_KERNEL_AUTO, "reference": xb.XY_KERNEL_REFERENCE, "mma": xb.XY_KERNEL_MMA}[args.kernel]
     ctx = xb.XYAttn(batch.num_q_heads, batch.num_kv_heads, batch.page_size, device=local_rank,
                     kernel=kernel, max_requests=max(256, batch.num_requests),
@@ -284,9 +285,10 @@ def main():
     plan_us = (time.perf_counter() - t0) * 1e6
 
     bt_host = torch.from_numpy(np.where(batch.block_table < 0, 0, batch.block_table).astype(np.int32))
-    q_host = tensors.q.contiguous().pin_memory()
+    qkv_host = tensors.qkv.contiguous().pin_memory()
     bt_pin = bt_host.pin_memory()
-    q = q_host.to(dev)
+    qkv = qkv_host.to(dev)
+    q = qkv[:, : batch.num_q_heads, :]
     k_pool = tensors.k_pool.to(dev)
     v_pool = tensors.v_pool.to(dev)
     bt = bt_host.to(dev)
@@ -348,8 +350,9 @@ def main():
     if not args.no_e2e:
         def e2e_step():
             ctx.plan_batch(batch)
-            q.copy_(q_host, non_blocking=True)
+            qkv.copy_(qkv_host, non_blocking=True)
             bt.copy_(bt_pin, non_blocking=True)
+            ctx.append_kv(qkv, k_pool, v_pool, bt)  # the step's new K/V go into the paged cache
             ctx.run(q, k_pool, v_pool, bt, SCALE, o, lse)
             o_host.copy_(o, non_blocking=True)
             lse_host.copy_(lse, non_blocking=True)
@@ -368,11 +371,12 @@ def main():
         if world > 1:
             dist.all_reduce(ems, op=dist.ReduceOp.MAX)
         e2e_ms = float(ems.item())
-        h2d = q_host.numel() * 2 + bt_pin.numel() * 4 + info.num_tasks * 32 + batch.num_requests * 32
+        h2d = qkv_host.numel() * 2 + bt_pin.numel() * 4 + info.num_tasks * 32 + batch.num_requests * 32
         d2h = o_host.numel() * 2 + lse_host.numel() * 4
         e2e = {"value": job_flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": n_e2e,
-               "includes": "host plan + H2D(Q, block table, task tables) + run + D2H(O, LSE); KV cache resident"}
+               "includes": "host plan + H2D(fused QKV of the new tokens, block table, task tables) + KV-cache "
+                           "append + run + D2H(O, LSE); the cached history is device-resident state"}
 
     if rank != 0:
         if world > 1:
@@ -412,7 +416,7 @@ def main():
     others = None
     if not args.no_others and world == 1:
         others = {}
-        del q, k_pool, v_pool, o, lse, tensors
+        del q, qkv, k_pool, v_pool, o, lse, tensors
         torch.cuda.empty_cache()
         for name in ("decode_only", "splitfuse_mix", "verify_trees", "full_mix"):
             if name == args.workload:

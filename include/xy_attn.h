@@ -164,6 +164,18 @@ int xy_attn_run(xy_attn_ctx* ctx, const void* q, int64_t q_token_stride, const v
                 const uint64_t* tree_mask, float sm_scale, void* o, int64_t o_token_stride,
                 float* lse, void* stream);
 
+/* KV-cache append with fused QKV split (the step before attention: Sections 4.1.1 and 5.4).
+ * For every planned request r and new token i the K and V head rows of the fused tensor
+ *   qkv DEVICE bf16 [T, Hq + 2 Hkv, D] (token stride qkv_token_stride elements; K heads follow
+ *   the Hq query heads, V heads follow the K heads)
+ * are copied into the paged cache at logical position kv_len[r] + i, found through the block
+ * table, with no intermediate split / permute tensors.  Uses the current plan's Token-Table;
+ * asynchronous on `stream`; run it before xy_attn_run of the same step (stream order suffices).
+ * The pools are written, everything else is read-only. */
+int xy_attn_append_kv(xy_attn_ctx* ctx, const void* qkv, int64_t qkv_token_stride, void* k_pool, void* v_pool,
+                      int64_t num_pages, int64_t page_stride, int64_t head_stride, int64_t token_stride,
+                      const int32_t* block_table, int32_t block_table_stride, void* stream);
+
 /* Split-KV LSE merge alone (the cross-core form of the Update stage, Section 4.2.1):
  *   LSE = ln sum_c exp(LSE_c),  O = sum_c exp(LSE_c - LSE) O_c.
  * o_part DEVICE fp32 [num_splits, rows, D], lse_part DEVICE fp32 [num_splits, rows];

@@ -163,3 +163,16 @@ def merge(O_c: np.ndarray, LSE_c: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
                             _ptr(LSE_c), _ptr(O), _ptr(LSE))
     assert rc == 0
     return O, LSE
+
+
+def append_kv(batch, qkv: torch.Tensor, k_pool: torch.Tensor, v_pool: torch.Tensor) -> None:
+    """Writes the K / V head rows of the fused QKV tensor (bf16 [T, Hq + 2 Hkv, D]) into the paged
+    cache at positions kv_len .. kv_len + q_len - 1 of every request (in place, bit copy)."""
+    assert qkv.dtype == torch.bfloat16 and qkv.stride(2) == 1 and qkv.stride(1) == batch.head_dim
+    ql, kl, bt = _i32(batch.q_len), _i32(batch.kv_len), _i32(batch.block_table)
+    rc = lib().oracle_append_kv(
+        ctypes.c_int(batch.num_requests), ctypes.c_int(batch.num_q_heads), ctypes.c_int(batch.num_kv_heads),
+        ctypes.c_int(batch.head_dim), ctypes.c_int(batch.page_size), _ptr(ql), _ptr(kl), _ptr(_u16(qkv)),
+        ctypes.c_int64(qkv.stride(0)), _ptr(_u16(k_pool)), _ptr(_u16(v_pool)), ctypes.c_int64(k_pool.stride(0)),
+        ctypes.c_int64(k_pool.stride(1)), ctypes.c_int64(k_pool.stride(2)), _ptr(bt), ctypes.c_int32(bt.shape[1]))
+    assert rc == 0

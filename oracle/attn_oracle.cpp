@@ -28,7 +28,7 @@
 // prefill row; closed forms (Q = 0, equal keys, constant V, single key, one-hot
 // V); star tree; an independently written brute force; torch fp64 softmax /
 // logsumexp on gathered K/V; page-permutation invariance; key-shift identity;
-// merge identity over arbitrary partitions; GQA special cases.
+// merge identity over arbitrary partitions; GQA special cases; append-then-gather round trip.
 
 #include <cmath>
 #include <cstdint>
@@ -259,6 +259,32 @@ int oracle_gather(PROBLEM_ARGS, int r, int g, uint16_t* K_out, uint16_t* V_out) 
     const int64_t off = kv_offset(p, r, g, j);
     std::memcpy(K_out + static_cast<int64_t>(j) * D, k_pool + off, sizeof(uint16_t) * D);
     std::memcpy(V_out + static_cast<int64_t>(j) * D, v_pool + off, sizeof(uint16_t) * D);
+  }
+  return 0;
+}
+
+// KV-cache append (the step before attention; Sections 4.1.1 and 5.4): for every request r and
+// new token i, the K and V head rows of the fused QKV tensor [T, Hq + 2 Hkv, D] are written to
+// the cache slot of logical position kv_len[r] + i, found through the block table.  Plain copy
+// of bf16 bits; K heads follow the Hq query heads, V heads follow the K heads.
+int oracle_append_kv(int R, int Hq, int Hkv, int D, int B, const int32_t* q_len, const int32_t* kv_len,
+                     const uint16_t* qkv, int64_t qkv_token_stride, uint16_t* k_pool, uint16_t* v_pool,
+                     int64_t page_stride, int64_t head_stride, int64_t token_stride,
+                     const int32_t* block_table, int32_t bt_stride) {
+  int64_t t = 0;
+  for (int r = 0; r < R; ++r) {
+    for (int i = 0; i < q_len[r]; ++i, ++t) {
+      const int j = kv_len[r] + i;
+      const int64_t page = block_table[static_cast<int64_t>(r) * bt_stride + j / B];
+      const int slot = j % B;
+      for (int g = 0; g < Hkv; ++g) {
+        const int64_t dst = page * page_stride + g * head_stride + static_cast<int64_t>(slot) * token_stride;
+        const uint16_t* ksrc = qkv + t * qkv_token_stride + static_cast<int64_t>(Hq + g) * D;
+        const uint16_t* vsrc = qkv + t * qkv_token_stride + static_cast<int64_t>(Hq + Hkv + g) * D;
+        std::memcpy(k_pool + dst, ksrc, sizeof(uint16_t) * D);
+        std::memcpy(v_pool + dst, vsrc, sizeof(uint16_t) * D);
+      }
+    }
   }
   return 0;
 }

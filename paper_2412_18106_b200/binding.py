@@ -74,6 +74,7 @@ EXPORTS = (
     "xy_attn_get_merge_units", "xy_attn_get_tree_mask", "xy_attn_get_q_start",
     "xy_attn_last_launches", "xy_attn_last_error", "xy_attn_device_status",
     "xy_attn_set_timing", "xy_attn_get_timing", "xy_attn_debug_trace", "xy_attn_decode_static",
+    "xy_attn_append_kv",
 )
 
 _lib = None
@@ -96,6 +97,7 @@ def load() -> ctypes.CDLL:
     L.xy_attn_run.argtypes = [vp, vp, i64, vp, vp, i64, i64, i64, i64, vp, i32, vp, ctypes.c_float,
                               vp, i64, vp, vp]
     L.xy_attn_merge.argtypes = [vp, vp, i32, i64, i32, vp, vp, vp]
+    L.xy_attn_append_kv.argtypes = [vp, vp, i64, vp, vp, i64, i64, i64, i64, vp, i32, vp]
     L.xy_attn_debug_gather.argtypes = [vp, i32, i32, vp, vp, i64, i64, i64, vp, i32, vp, vp, vp]
     for name in ("xy_attn_get_tasks", "xy_attn_get_worker_offsets", "xy_attn_get_merge_units",
                  "xy_attn_get_tree_mask", "xy_attn_get_q_start"):
@@ -199,6 +201,20 @@ class XYAttn:
             k_pool.shape[0], k_pool.stride(0), k_pool.stride(1), k_pool.stride(2),
             block_table.data_ptr(), block_table.stride(0), tm, float(sm_scale), o.data_ptr(),
             o.stride(0), lse.data_ptr(), _stream_ptr(stream)))
+
+    # -- xy_attn_append_kv
+    def append_kv(self, qkv: torch.Tensor, k_pool: torch.Tensor, v_pool: torch.Tensor, block_table: torch.Tensor,
+                  stream=None) -> None:
+        """Copies the K / V heads of the fused bf16 [T, Hq + 2 Hkv, D] tensor into the paged cache."""
+        for t in (qkv, k_pool, v_pool, block_table):
+            if not t.is_cuda:
+                raise XYAttnError(XY_ERR_INVALID_ARG, "append_kv needs CUDA tensors (there is no CPU path)")
+        assert qkv.dtype == torch.bfloat16 and qkv.stride(2) == 1 and qkv.stride(1) == self.cfg.head_dim
+        assert k_pool.stride() == v_pool.stride() and k_pool.stride(3) == 1
+        self._check(self.lib.xy_attn_append_kv(
+            self._ctx, qkv.data_ptr(), qkv.stride(0), k_pool.data_ptr(), v_pool.data_ptr(), k_pool.shape[0],
+            k_pool.stride(0), k_pool.stride(1), k_pool.stride(2), block_table.data_ptr(), block_table.stride(0),
+            _stream_ptr(stream)))
 
     # -- xy_attn_debug_gather
     def debug_gather(self, req: int, kv_head: int, k_pool, v_pool, block_table, out_k, out_v, stream=None):

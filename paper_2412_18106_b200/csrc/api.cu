@@ -343,6 +343,34 @@ int xy_attn_get_timing(xy_attn_ctx* ctx, float* attention_ms, float* merge_ms, i
   return XY_OK;
 }
 
+int xy_attn_append_kv(xy_attn_ctx* ctx, const void* qkv, int64_t qkv_token_stride, void* k_pool, void* v_pool,
+                      int64_t num_pages, int64_t page_stride, int64_t head_stride, int64_t token_stride,
+                      const int32_t* block_table, int32_t block_table_stride, void* stream) {
+  if (ctx == nullptr) return XY_ERR_INVALID_ARG;
+  if (ctx->host_only) return set_err(ctx, XY_ERR_UNSUPPORTED, "host-only context cannot run");
+  if (!ctx->planned) return set_err(ctx, XY_ERR_NOT_PLANNED, "xy_attn_append_kv before xy_attn_plan");
+  const PlanResult& p = ctx->plan;
+  if (p.total_q == 0) return XY_OK;
+  const xy_attn_config& cfg = ctx->cfg;
+  if (!qkv || !k_pool || !v_pool || !block_table) return set_err(ctx, XY_ERR_INVALID_ARG, "null device pointer");
+  auto misaligned = [](const void* ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15u) != 0; };
+  if (misaligned(qkv) || misaligned(k_pool) || misaligned(v_pool))
+    return set_err(ctx, XY_ERR_INVALID_ARG, "qkv, k_pool and v_pool must be 16-byte aligned");
+  if (qkv_token_stride < static_cast<int64_t>(cfg.num_q_heads + 2 * cfg.num_kv_heads) * kHeadDim ||
+      qkv_token_stride % 8 != 0)
+    return set_err(ctx, XY_ERR_INVALID_ARG, "qkv token stride too small or not a multiple of 8");
+  if (token_stride < kHeadDim || token_stride % 8 != 0 || head_stride % 8 != 0 || head_stride < 1 ||
+      page_stride % 8 != 0 || page_stride < 1 || num_pages < 1 || block_table_stride < 1)
+    return set_err(ctx, XY_ERR_INVALID_ARG, "bad K/V pool strides, num_pages or block_table_stride");
+  XY_CUDA(ctx, cudaSetDevice(cfg.device));
+  XY_CUDA(ctx, launch_append_kv(static_cast<const uint16_t*>(qkv), qkv_token_stride, static_cast<uint16_t*>(k_pool),
+                                static_cast<uint16_t*>(v_pool), page_stride, head_stride, token_stride, block_table,
+                                block_table_stride, ctx->d_reqs, static_cast<int>(p.reqs.size()),
+                                static_cast<int>(p.total_q), cfg.num_q_heads, cfg.num_kv_heads, cfg.page_size,
+                                ctx->page_shift, static_cast<cudaStream_t>(stream)));
+  return XY_OK;
+}
+
 int xy_attn_merge(const float* o_part, const float* lse_part, int32_t num_splits, int64_t rows,
                   int32_t head_dim, void* o, float* lse, void* stream) {
   if (head_dim != kHeadDim) return XY_ERR_UNSUPPORTED;

@@ -177,7 +177,48 @@ __global__ void gather_kernel(const uint16_t* k_pool, const uint16_t* v_pool, in
       *reinterpret_cast<const uint2*>(v_pool + off);
 }
 
+// KV-cache append with fused QKV split (Sections 4.1.1, 5.4): one block per new token; the
+// request is found by bisection over the start positions; every thread moves 16 bytes at a time.
+__global__ void __launch_bounds__(128) append_kv_kernel(const uint16_t* qkv, int64_t qkv_token_stride,
+                                                        uint16_t* k_pool, uint16_t* v_pool, int64_t page_stride,
+                                                        int64_t head_stride, int64_t token_stride,
+                                                        const int32_t* block_table, int bt_stride,
+                                                        const ReqInfo* reqs, int num_reqs, int Hq, int Hkv,
+                                                        int page_size, int page_shift) {
+  const int t = blockIdx.x;
+  int lo = 0, hi = num_reqs - 1;  // last request whose start position is <= t
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (reqs[mid].q_start <= t) lo = mid; else hi = mid - 1;
+  }
+  const ReqInfo rq = reqs[lo];
+  const int j = rq.kv_len + (t - rq.q_start);
+  const int64_t page = block_table[static_cast<int64_t>(lo) * bt_stride + (j >> page_shift)];
+  const int64_t slot_off = page * page_stride + static_cast<int64_t>(j & (page_size - 1)) * token_stride;
+  const uint16_t* src = qkv + static_cast<int64_t>(t) * qkv_token_stride + static_cast<int64_t>(Hq) * kHeadDim;
+  const int chunks = 2 * Hkv * (kHeadDim / 8);  // 16-byte chunks of this token's K then V heads
+  for (int c = threadIdx.x; c < chunks; c += blockDim.x) {
+    const int hv = c / (kHeadDim / 8), d8 = c % (kHeadDim / 8);  // head index within [K heads | V heads]
+    const bool is_v = hv >= Hkv;
+    const int g = is_v ? hv - Hkv : hv;
+    const uint4 val = *reinterpret_cast<const uint4*>(src + static_cast<int64_t>(hv) * kHeadDim + d8 * 8);
+    uint16_t* pool = is_v ? v_pool : k_pool;
+    *reinterpret_cast<uint4*>(pool + slot_off + static_cast<int64_t>(g) * head_stride + d8 * 8) = val;
+  }
+}
+
 }  // namespace
+
+cudaError_t launch_append_kv(const uint16_t* qkv, int64_t qkv_token_stride, uint16_t* k_pool, uint16_t* v_pool,
+                             int64_t page_stride, int64_t head_stride, int64_t token_stride,
+                             const int32_t* block_table, int bt_stride, const ReqInfo* reqs, int num_reqs,
+                             int total_q, int Hq, int Hkv, int page_size, int page_shift, cudaStream_t s) {
+  if (total_q == 0) return cudaSuccess;
+  append_kv_kernel<<<total_q, 128, 0, s>>>(qkv, qkv_token_stride, k_pool, v_pool, page_stride, head_stride,
+                                           token_stride, block_table, bt_stride, reqs, num_reqs, Hq, Hkv,
+                                           page_size, page_shift);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_reference(const RunArgs& a, int num_workers, cudaStream_t s) {
   ref_attention_kernel<<<num_workers, 128, 0, s>>>(a);

@@ -490,3 +490,30 @@ def test_tail_poison_does_not_change_the_result():
     O1, L1 = oracle.attention(b, t, SCALE)
     O2, L2 = oracle.attention(b, tp, SCALE)
     assert np.array_equal(O1, O2) and np.array_equal(L1, L2)
+
+
+# ---------------------------------------------------------------- KV-cache append (next-row N1)
+def test_append_kv_round_trip_and_untouched_slots():
+    """Oracle append pinned by direct indexing: after the append, the cache slot of logical
+    position kv_len + i of every request holds exactly the K / V heads of token i of the fused
+    tensor, and no other slot changed."""
+    rng = np.random.default_rng(41)
+    b = W.custom("append", 6, 2, 4, [(5, 3, 0, None), (1, 9, 0, None), (7, 0, 1, W.random_tree(rng, 7, 3))], seed=41)
+    t = W.make_tensors(b, fused_qkv=True)
+    k0, v0 = t.k_pool.clone(), t.v_pool.clone()
+    oracle.append_kv(b, t.qkv, t.k_pool, t.v_pool)
+    touched = torch.zeros(t.k_pool.shape[:3], dtype=torch.bool)
+    B, Hq, Hkv = b.page_size, b.num_q_heads, b.num_kv_heads
+    for r in range(b.num_requests):
+        for i in range(int(b.q_len[r])):
+            tok = int(b.q_start[r]) + i
+            j = int(b.kv_len[r]) + i
+            page, slot = int(b.block_table[r, j // B]), j % B
+            for g in range(Hkv):
+                assert torch.equal(t.k_pool[page, g, slot], t.qkv[tok, Hq + g])
+                assert torch.equal(t.v_pool[page, g, slot], t.qkv[tok, Hq + Hkv + g])
+                touched[page, g, slot] = True
+    assert torch.equal(t.k_pool[~touched], k0[~touched]) and torch.equal(t.v_pool[~touched], v0[~touched])
+    # the gather of the oracle sees the appended rows at the end of each request
+    K, V = oracle.gather(b, t, 0, 1)
+    assert torch.equal(K[3:], t.qkv[0:5, Hq + 1]) and torch.equal(V[3:], t.qkv[0:5, Hq + Hkv + 1])
