@@ -219,6 +219,12 @@ int xy_attn_debug_gather(xy_attn_ctx* ctx, int32_t req, int32_t kv_head, const v
                          int64_t token_stride, const int32_t* block_table,
                          int32_t block_table_stride, void* out_k, void* out_v, void* stream);
 
+/* Per-worker wall time of the last xy_attn_run (load-balance metric): synchronises the device
+ * and copies 2 x num_workers nanosecond time stamps (entry, exit of each persistent worker, from
+ * the GPU's global timer) to `out` (HOST).  Returns the number of entries; copies only if `cap`
+ * is large enough.  Only the attention meta-kernel records them (not XY_KERNEL_REFERENCE). */
+int xy_attn_worker_times(xy_attn_ctx* ctx, uint64_t* out, int32_t cap);
+
 /* Debug tracing (only in a library built with -DXY_ENABLE_TRACE, i.e. XY_BUILD_TRACE=1 for
  * paper_2412_18106_b200.build; otherwise no records are written and 0 entries are meaningful).
  * When the environment variable XY_ATTN_TRACE=1 is set at create time, the

@@ -74,7 +74,7 @@ EXPORTS = (
     "xy_attn_get_merge_units", "xy_attn_get_tree_mask", "xy_attn_get_q_start",
     "xy_attn_last_launches", "xy_attn_last_error", "xy_attn_device_status",
     "xy_attn_set_timing", "xy_attn_get_timing", "xy_attn_debug_trace", "xy_attn_decode_static",
-    "xy_attn_append_kv",
+    "xy_attn_append_kv", "xy_attn_worker_times",
 )
 
 _lib = None
@@ -106,6 +106,7 @@ def load() -> ctypes.CDLL:
     L.xy_attn_get_timing.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float),
                                      ctypes.POINTER(i32)]
     L.xy_attn_debug_trace.argtypes = [vp, vp, i32]
+    L.xy_attn_worker_times.argtypes = [vp, vp, i32]
     L.xy_attn_decode_static.argtypes = [vp, i64, vp, vp, i64, i64, i64, vp, i32, vp, i32, i32, i32, i32, i32,
                                         ctypes.c_float, vp, i64, vp, vp]
     L.xy_attn_last_launches.argtypes = [vp]
@@ -255,6 +256,15 @@ class XYAttn:
         a, m, n = ctypes.c_float(0), ctypes.c_float(0), ctypes.c_int32(0)
         self._check(self.lib.xy_attn_get_timing(self._ctx, ctypes.byref(a), ctypes.byref(m), ctypes.byref(n)))
         return float(a.value), float(m.value), int(n.value)
+
+    def worker_times(self) -> np.ndarray:
+        """uint64 [num_workers, 2]: (entry, exit) nanosecond stamps of each worker in the last run."""
+        n = self.lib.xy_attn_worker_times(self._ctx, ctypes.c_void_p(0), 0)
+        if n <= 0:
+            self._check(n)
+        out = np.zeros(n, dtype=np.uint64)
+        self.lib.xy_attn_worker_times(self._ctx, ctypes.c_void_p(out.ctypes.data), n)
+        return out.reshape(-1, 2)
 
     def debug_trace(self) -> np.ndarray:
         """uint64 [4, 2048] trace records of worker 0 (empty unless XY_ATTN_TRACE=1 at create)."""

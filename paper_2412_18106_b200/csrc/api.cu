@@ -26,12 +26,14 @@ struct xy_attn_ctx {
   ReqInfo* d_reqs = nullptr;
   xy_attn_task* d_tasks = nullptr;
   int32_t* d_worker_off = nullptr;
+  int32_t* d_queue = nullptr;
   uint64_t* d_tree = nullptr;
   xy_attn_merge_unit* d_merges = nullptr;
   float* d_o_part = nullptr;
   float* d_lse_part = nullptr;
   int32_t* d_status = nullptr;
   unsigned long long* d_trace = nullptr;
+  unsigned long long* d_worker_times = nullptr;
   int last_launches = 0;
   bool timing = false;
   std::vector<cudaEvent_t> events;  // three per timed run: before attention, after it, after merge
@@ -67,12 +69,14 @@ void free_device(xy_attn_ctx* c) {
   cudaFree(c->d_reqs);
   cudaFree(c->d_tasks);
   cudaFree(c->d_worker_off);
+  cudaFree(c->d_queue);
   cudaFree(c->d_tree);
   cudaFree(c->d_merges);
   cudaFree(c->d_o_part);
   cudaFree(c->d_lse_part);
   cudaFree(c->d_status);
   cudaFree(c->d_trace);
+  cudaFree(c->d_worker_times);
 }
 
 }  // namespace
@@ -141,11 +145,13 @@ int xy_attn_create(const xy_attn_config* cfg, xy_attn_ctx** out) {
     alloc(reinterpret_cast<void**>(&c->d_reqs), sizeof(ReqInfo) * cfg->max_requests);
     alloc(reinterpret_cast<void**>(&c->d_tasks), sizeof(xy_attn_task) * c->cap_tasks);
     alloc(reinterpret_cast<void**>(&c->d_worker_off), sizeof(int32_t) * (c->num_workers + 1));
+    alloc(reinterpret_cast<void**>(&c->d_queue), sizeof(int32_t) * c->cap_tasks);
     alloc(reinterpret_cast<void**>(&c->d_tree), sizeof(uint64_t) * c->cap_tree_words);
     alloc(reinterpret_cast<void**>(&c->d_merges), sizeof(xy_attn_merge_unit) * c->cap_merges);
     alloc(reinterpret_cast<void**>(&c->d_o_part), sizeof(float) * kHeadDim * c->cap_partial_rows);
     alloc(reinterpret_cast<void**>(&c->d_lse_part), sizeof(float) * c->cap_partial_rows);
     alloc(reinterpret_cast<void**>(&c->d_status), 256);
+    alloc(reinterpret_cast<void**>(&c->d_worker_times), sizeof(unsigned long long) * 2 * c->num_workers);
     if (e == cudaSuccess) e = cudaMemset(c->d_status, 0, 256);
     const char* tr = getenv("XY_ATTN_TRACE");
     if (tr != nullptr && tr[0] == '1') {
@@ -202,6 +208,9 @@ int xy_attn_plan(xy_attn_ctx* ctx, const xy_attn_request* reqs, int32_t num_reqs
     if (!p.tasks.empty())
       XY_CUDA(ctx, cudaMemcpyAsync(ctx->d_tasks, p.tasks.data(),
                                    sizeof(xy_attn_task) * p.tasks.size(), cudaMemcpyHostToDevice, s));
+    if (!p.queue.empty())
+      XY_CUDA(ctx, cudaMemcpyAsync(ctx->d_queue, p.queue.data(), sizeof(int32_t) * p.queue.size(),
+                                   cudaMemcpyHostToDevice, s));
     XY_CUDA(ctx, cudaMemcpyAsync(ctx->d_worker_off, p.worker_off.data(),
                                  sizeof(int32_t) * p.worker_off.size(), cudaMemcpyHostToDevice, s));
     if (!p.tree_mask.empty())
@@ -269,10 +278,18 @@ int xy_attn_run(xy_attn_ctx* ctx, const void* q, int64_t q_token_stride, const v
   a.lse_part = ctx->d_lse_part;
   a.status = ctx->d_status;
   a.trace = ctx->d_trace;
+  a.worker_times = ctx->d_worker_times;
   a.num_q_heads = cfg.num_q_heads;
   a.num_kv_heads = cfg.num_kv_heads;
   a.page_size = cfg.page_size;
   a.page_shift = ctx->page_shift;
+  a.queue = ctx->d_queue;
+  a.queue_head = ctx->d_status + 16;  // second cache line of the status block
+  a.num_tasks = static_cast<int32_t>(p.tasks.size());
+  // Balanced plans are dealt dynamically by the meta-kernel; paper-mode plans keep the static
+  // Task-Table (each worker walks its own list), as does the reference kernel.
+  a.dynamic = (cfg.plan_mode == XY_PLAN_BALANCED && cfg.kernel != XY_KERNEL_REFERENCE) ? 1 : 0;
+  if (a.dynamic) XY_CUDA(ctx, cudaMemsetAsync(a.queue_head, 0, sizeof(int32_t), s));
 
   const bool timed = ctx->timing && ctx->timed_runs < kMaxTimedRuns;
   if (timed) {
@@ -419,6 +436,18 @@ XY_GETTER(xy_attn_get_worker_offsets, int32_t, worker_off)
 XY_GETTER(xy_attn_get_merge_units, xy_attn_merge_unit, merges)
 XY_GETTER(xy_attn_get_tree_mask, uint64_t, tree_mask)
 XY_GETTER(xy_attn_get_q_start, int32_t, q_start)
+
+int xy_attn_worker_times(xy_attn_ctx* ctx, uint64_t* out, int32_t cap) {
+  if (ctx == nullptr || (out == nullptr && cap > 0)) return XY_ERR_INVALID_ARG;
+  if (ctx->host_only) return set_err(ctx, XY_ERR_UNSUPPORTED, "host-only context");
+  const int n = 2 * ctx->num_workers;
+  if (cap >= n) {
+    XY_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+    XY_CUDA(ctx, cudaDeviceSynchronize());
+    XY_CUDA(ctx, cudaMemcpy(out, ctx->d_worker_times, sizeof(uint64_t) * n, cudaMemcpyDeviceToHost));
+  }
+  return n;
+}
 
 int xy_attn_debug_trace(xy_attn_ctx* ctx, uint64_t* out, int32_t cap) {
   if (ctx == nullptr || (out == nullptr && cap > 0)) return XY_ERR_INVALID_ARG;

@@ -50,7 +50,7 @@ struct __align__(8) SmemBarriers {
 constexpr int kSmemQ = 2 * kTileBytes;
 constexpr int kSmemRing = kStages * kTileBytes;
 constexpr int kSmemMl = kConsumerWarps * 16 * 2 * 4;
-constexpr int kSmemTotal = 1024 /*align slack*/ + kSmemQ + kSmemRing + kSmemMl + sizeof(SmemBarriers) + 128;
+constexpr int kSmemTotal = 1024 /*align slack*/ + kSmemQ + kSmemRing + kSmemMl + sizeof(SmemBarriers) + 128 + 256;
 
 __device__ __forceinline__ uint32_t swz(uint32_t row, uint32_t chunk16 /*0..15*/) {
   return (chunk16 >> 3) * kHalfBytes + row * 128u + (((chunk16 & 7u) ^ (row & 7u)) << 4);
@@ -351,6 +351,15 @@ constexpr uint32_t kIdescBase = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3
 constexpr uint32_t kIdescQK = kIdescBase;              // A, B K-major
 constexpr uint32_t kIdescPV = kIdescBase | (1u << 16);  // B (V) MN-major
 
+// Task indices travel from the producer (which takes them from the global queue) to the other
+// roles of the CTA through a small ring in shared memory.
+constexpr int kTaskRing = 8;
+struct __align__(8) TaskRing {
+  uint64_t full[kTaskRing];   // producer -> readers: the slot holds a task index (or -1: no more)
+  uint64_t empty[kTaskRing];  // readers -> producer: every reader has taken the slot's index
+  int32_t ti[kTaskRing];
+};
+
 struct DenseShape {
   int n[2];  // KV tiles sub-tile A / B visits in this task
   int n_all;
@@ -400,16 +409,24 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
   float* ml = reinterpret_cast<float*>(gen_base + kSmemQ + kSmemRing);
   SmemBarriers* bars = reinterpret_cast<SmemBarriers*>(gen_base + kSmemQ + kSmemRing + kSmemMl);
   UmmaBarriers* ub = reinterpret_cast<UmmaBarriers*>(gen_base + kSmemQ + kSmemRing + kSmemMl + sizeof(SmemBarriers));
+  TaskRing* tq = reinterpret_cast<TaskRing*>(gen_base + kSmemQ + kSmemRing + kSmemMl + sizeof(SmemBarriers) + 128);
   float* xch = reinterpret_cast<float*>(gen_base);  // streaming merge area, aliases the Q tiles
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
+    unsigned long long now;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+    a.worker_times[2 * blockIdx.x] = now;
     for (int s = 0; s < kStages; ++s) {
       mbar_init(smem_u32(&bars->full[s]), 1);
       mbar_init(smem_u32(&bars->empty[s]), kConsumerWarps);
       mbar_init(smem_u32(&bars->empty_umma[s]), 2);
     }
     ub->turn = 0;
+    for (int i = 0; i < kTaskRing; ++i) {
+      mbar_init(smem_u32(&tq->full[i]), 1);
+      mbar_init(smem_u32(&tq->empty[i]), kConsumerWarps + (kUmma ? 2 : 0));
+    }
     for (int X = 0; X < 2; ++X) {
       mbar_init(smem_u32(&ub->q_full[X]), 4);
       mbar_init(smem_u32(&ub->s_full[X]), 1);
@@ -429,6 +446,29 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
   const uint32_t tmem = kUmma ? ub->tmem_base : 0u;
 
   const int t_begin = a.worker_off[blockIdx.x], t_end = a.worker_off[blockIdx.x + 1];
+  const bool dynamic = a.dynamic != 0;
+  // Every role but the producer reads its task sequence here: the worker's own Task-Table list
+  // (static dealing) or the indices the producer publishes (dynamic dealing).  Warp-uniform.
+  int seq_static = t_begin;
+  uint32_t n_read = 0;
+  bool feed_dead = false;
+  auto next_task = [&](bool whole_warp) -> int {  // whole_warp: called by all 32 lanes (else by one)
+    if (!dynamic) return seq_static < t_end ? seq_static++ : -1;
+    const uint32_t slot = n_read % kTaskRing;
+    if (!feed_dead && !mbar_wait(smem_u32(&tq->full[slot]), (n_read / kTaskRing) & 1u, a.status)) {
+      atomicExch(a.status, XY_ERR_DEVICE_TIMEOUT);
+      feed_dead = true;
+    }
+    const int ti = feed_dead ? -1 : tq->ti[slot];
+    if (whole_warp) {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&tq->empty[slot]));
+    } else {
+      mbar_arrive(smem_u32(&tq->empty[slot]));
+    }
+    ++n_read;
+    return ti;
+  };
   const int G = a.num_q_heads / a.num_kv_heads;
   const float scale_log2 = a.sm_scale * kLog2e;
 
@@ -499,6 +539,28 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
         bool by_umma, valid;
       };
       int f_ti = t_begin, f_kt = 0, f_hi = 0, f_head = 0, f_npages = 1;
+      uint32_t n_pub = 0;
+      bool f_done = false;
+      // Next task of this worker: its own list, or the head of the global queue (published to the
+      // other roles through the ring; -1 is published once, when the queue is exhausted).
+      auto grab = [&]() -> int {
+        if (!dynamic) return f_ti < t_end ? f_ti++ : -1;
+        if (f_done) return -1;
+        int ti = -1;
+        const int k = atomicAdd(a.queue_head, 1);
+        if (k < a.num_tasks) ti = __ldg(a.queue + k);
+        const uint32_t slot = n_pub % kTaskRing;
+        if (n_pub >= kTaskRing &&
+            !mbar_wait(smem_u32(&tq->empty[slot]), ((n_pub / kTaskRing) - 1u) & 1u, a.status)) {
+          report_timeout(a);
+          dead = true;
+        }
+        tq->ti[slot] = ti;
+        mbar_arrive(smem_u32(&tq->full[slot]));
+        ++n_pub;
+        if (ti < 0) f_done = true;
+        return ti;
+      };
       const int32_t* f_bt = a.block_table;
       bool f_umma = false, f_open = false;
       auto next_tile = [&]() {
@@ -509,9 +571,9 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
         x.npages = 1;
         x.by_umma = false;
         while (!f_open || f_kt >= f_hi) {
-          if (f_open) ++f_ti;
-          if (f_ti >= t_end) return x;
-          const xy_attn_task t = a.tasks[f_ti];
+          const int ti = grab();
+          if (ti < 0) return x;
+          const xy_attn_task t = a.tasks[ti];
           const ReqInfo rq = a.reqs[t.req];
           f_kt = t.kt_lo;
           f_hi = t.kt_hi;
@@ -628,7 +690,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
         }
       };
       auto pass_turn = [&](uint32_t g) { ub->turn = g + 1; };
-      for (int ti = t_begin; ti < t_end; ++ti) {
+      for (int ti = next_task(false); ti >= 0; ti = next_task(false)) {
         const xy_attn_task t = a.tasks[ti];
         const uint32_t n_all = t.kt_hi - t.kt_lo;
         const uint32_t pos0 = pos;
@@ -696,7 +758,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
     Tracer tr;
     tr.init(a, warp >> 2, (threadIdx.x & 127) == 0);
     const int X = warp >> 2;       // sub-tile this warpgroup owns on the tcgen05 path
-    for (int ti = t_begin; ti < t_end; ++ti) {
+    for (int ti = next_task(true); ti >= 0; ti = next_task(true)) {
       TaskView tv;
       tv.t = a.tasks[ti];
       tv.rq = a.reqs[tv.t.req];
@@ -1059,6 +1121,11 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
   }
   tc_fence_before();
   __syncthreads();
+  if (threadIdx.x == 0) {
+    unsigned long long now;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+    a.worker_times[2 * blockIdx.x + 1] = now;
+  }
   if (kUmma && warp == kConsumerWarps + 1) {
     tc_fence_after();
     tmem_dealloc(tmem, kTmemCols);

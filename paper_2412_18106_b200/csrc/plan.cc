@@ -249,6 +249,7 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
     lists[w].push_back(order[pos]);
   }
   out->worker_off.assign(C + 1, 0);
+  std::vector<int32_t> where(pend.size(), 0);  // position of each pending task in the table
   out->tasks.reserve(pend.size());
   out->task_cost.reserve(pend.size());
   float lmin = 0.f, lmax = 0.f, lsum = 0.f, tmax = 0.f;
@@ -256,6 +257,7 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
   for (int w = 0; w < C; ++w) {
     float load = 0.f;
     for (int id : lists[w]) {
+      where[id] = static_cast<int32_t>(out->tasks.size());
       out->tasks.push_back(pend[id].t);
       out->task_cost.push_back(pend[id].cost);
       load += pend[id].cost;
@@ -267,6 +269,10 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
     lmax = std::max(lmax, load);
     lsum += load;
   }
+
+  // The same sorted list as one queue, for workers that take tasks as they become free.
+  out->queue.resize(order.size());
+  for (size_t pos = 0; pos < order.size(); ++pos) out->queue[pos] = where[order[pos]];
 
   xy_attn_plan_info& info = out->info;
   info.num_tasks = static_cast<int32_t>(out->tasks.size());

@@ -33,6 +33,7 @@ struct PlanResult {
   std::vector<xy_attn_task> tasks;         // grouped by worker
   std::vector<float> task_cost;            // parallel to tasks
   std::vector<int32_t> worker_off;         // num_workers + 1
+  std::vector<int32_t> queue;              // task indices by descending cost (dynamic dealing)
   std::vector<xy_attn_merge_unit> merges;
   int64_t partial_rows = 0;
   int64_t total_q = 0;
@@ -68,8 +69,13 @@ struct RunArgs {
   float* o_part;
   float* lse_part;
   int32_t* status;
+  unsigned long long* worker_times;  // [2 * workers]: globaltimer at entry and exit of each worker
   unsigned long long* trace;  // null unless tracing: kTraceRoles x kTraceLen (tag << 48 | cycle) records
   int32_t num_q_heads, num_kv_heads, page_size, page_shift;
+  // dynamic dealing: workers take the next task of `queue` with an atomic counter
+  const int32_t* queue;
+  int32_t* queue_head;
+  int32_t num_tasks, dynamic;
 };
 
 }  // namespace xy
