@@ -31,6 +31,9 @@ constexpr int kMinChunkTiles = 4;
 // split (measured on the five benchmark batches: finer splits lose more to per-task overhead
 // and partial traffic than they gain in balance).
 constexpr float kTaskCapFraction = 0.77f;
+// Dense tasks are split a little finer (cap x 0.65): their per-task overhead is small next to a
+// key-tile visit, and finer dense tasks even out the tail of the dynamically dealt queue.
+constexpr float kDenseCapFactor = 0.65f;
 
 struct Unit {
   int32_t req, kv_head, tok0, ntok, kind;
@@ -181,6 +184,7 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
   double total_cost = 0.0;
   for (const Unit& u : units) total_cost += kTaskFixedUs + u.visit_cost * u.nkt;
   float cap = static_cast<float>(total_cost / std::max(1, num_workers) * kTaskCapFraction);
+  const float dense_factor = kDenseCapFactor;
   std::vector<int> chunk_tiles(units.size(), 0);
   for (int attempt = 0; attempt < 64; ++attempt) {
     int64_t prow = 0;
@@ -189,7 +193,8 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
       int nsplit = 1;
       if (!paper) {
         const float cost = u.visit_cost * u.nkt;
-        nsplit = static_cast<int>(std::ceil(cost / std::max(cap, 1e-3f)));
+        const float cap_u = u.kind == 1 ? cap : cap * dense_factor;
+        nsplit = static_cast<int>(std::ceil(cost / std::max(cap_u, 1e-3f)));
         nsplit = std::min(nsplit, max_splits);
         nsplit = std::min(nsplit, std::max(1, u.nkt / kMinChunkTiles));
         nsplit = std::max(nsplit, 1);
