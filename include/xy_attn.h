@@ -220,8 +220,9 @@ int xy_attn_debug_gather(xy_attn_ctx* ctx, int32_t req, int32_t kv_head, const v
                          int32_t block_table_stride, void* out_k, void* out_v, void* stream);
 
 /* Per-worker wall time of the last xy_attn_run (load-balance metric): synchronises the device
- * and copies 2 x num_workers nanosecond time stamps (entry, exit of each persistent worker, from
- * the GPU's global timer) to `out` (HOST).  Returns the number of entries; copies only if `cap`
+ * and copies 4 x num_workers values to `out` (HOST): for each persistent worker its entry and
+ * exit time stamps (nanoseconds of the GPU's global timer) and the nanoseconds it spent in dense
+ * and in streaming tasks.  Returns the number of entries; copies only if `cap`
  * is large enough.  Only the attention meta-kernel records them (not XY_KERNEL_REFERENCE). */
 int xy_attn_worker_times(xy_attn_ctx* ctx, uint64_t* out, int32_t cap);
 

@@ -258,13 +258,14 @@ class XYAttn:
         return float(a.value), float(m.value), int(n.value)
 
     def worker_times(self) -> np.ndarray:
-        """uint64 [num_workers, 2]: (entry, exit) nanosecond stamps of each worker in the last run."""
+        """uint64 [num_workers, 4]: entry and exit stamps (ns) of each worker in the last run and
+        the ns it spent in dense and in streaming tasks."""
         n = self.lib.xy_attn_worker_times(self._ctx, ctypes.c_void_p(0), 0)
         if n <= 0:
             self._check(n)
         out = np.zeros(n, dtype=np.uint64)
         self.lib.xy_attn_worker_times(self._ctx, ctypes.c_void_p(out.ctypes.data), n)
-        return out.reshape(-1, 2)
+        return out.reshape(-1, 4)
 
     def debug_trace(self) -> np.ndarray:
         """uint64 [4, 2048] trace records of worker 0 (empty unless XY_ATTN_TRACE=1 at create)."""

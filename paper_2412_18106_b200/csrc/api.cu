@@ -151,7 +151,7 @@ int xy_attn_create(const xy_attn_config* cfg, xy_attn_ctx** out) {
     alloc(reinterpret_cast<void**>(&c->d_o_part), sizeof(float) * kHeadDim * c->cap_partial_rows);
     alloc(reinterpret_cast<void**>(&c->d_lse_part), sizeof(float) * c->cap_partial_rows);
     alloc(reinterpret_cast<void**>(&c->d_status), 256);
-    alloc(reinterpret_cast<void**>(&c->d_worker_times), sizeof(unsigned long long) * 2 * c->num_workers);
+    alloc(reinterpret_cast<void**>(&c->d_worker_times), sizeof(unsigned long long) * 4 * c->num_workers);
     if (e == cudaSuccess) e = cudaMemset(c->d_status, 0, 256);
     const char* tr = getenv("XY_ATTN_TRACE");
     if (tr != nullptr && tr[0] == '1') {
@@ -440,7 +440,7 @@ XY_GETTER(xy_attn_get_q_start, int32_t, q_start)
 int xy_attn_worker_times(xy_attn_ctx* ctx, uint64_t* out, int32_t cap) {
   if (ctx == nullptr || (out == nullptr && cap > 0)) return XY_ERR_INVALID_ARG;
   if (ctx->host_only) return set_err(ctx, XY_ERR_UNSUPPORTED, "host-only context");
-  const int n = 2 * ctx->num_workers;
+  const int n = 4 * ctx->num_workers;
   if (cap >= n) {
     XY_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
     XY_CUDA(ctx, cudaDeviceSynchronize());

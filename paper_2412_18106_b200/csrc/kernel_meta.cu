@@ -18,6 +18,7 @@
 // to bf16 before P.V; masked scores are selected to -inf, never added.
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <type_traits>
 #include <cuda_runtime.h>
 
 #include "ptx.cuh"
@@ -328,6 +329,112 @@ __device__ __forceinline__ void report_timeout(const RunArgs& a) {
 }
 
 // ------------------------------------------------------------------------------------------
+// One streaming task (at most 16 packed rows: decode steps, short verify windows and the thin
+// tails of prefill chunks), run by the eight consumer warps.  Every warp owns 16 keys of each
+// 128-key tile, keeps its own online-softmax state over those keys, and the eight partial
+// results are merged through shared memory when the task ends (the in-CTA Update stage of
+// Section 4.2.1).  It is a function of its own, not inlined into the kernel, so that the
+// register allocation of this bandwidth-critical loop is independent of the dense paths'.
+// pipe_state: ring stage | phase << 8 | dead << 16, returned updated.
+__device__ __noinline__ uint32_t stream_task(const RunArgs& a, const TaskView& tv, uint32_t q_smem, uint32_t ring,
+                                             SmemBarriers* bars, float* xch, float* ml, uint32_t pipe_state,
+                                             float scale_log2) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  Pipe pipe{static_cast<int>(pipe_state & 0xFFu), (pipe_state >> 8) & 1u};
+  bool dead = (pipe_state >> 16) & 1u;
+  const int h = tv.rq.kv_len;
+  const bool tree = tv.rq.mask_kind == XY_MASK_TREE;
+  const int koff = warp * 16;
+  WarpTile<2, false> w;
+  w.init();
+  w.load_q(q_smem, 0, lane);
+  const int r_lo = min(lane >> 2, tv.rows - 1), r_hi = min((lane >> 2) + 8, tv.rows - 1);
+  const int i_lo = tv.t.tok0 + r_lo / tv.G, i_hi = tv.t.tok0 + r_hi / tv.G;
+  const int i_max = tv.t.tok0 + tv.t.ntok - 1;
+  // Tiles that every row of the task sees in full need neither the mask nor the mask-aware
+  // skip test; the loop over them is compiled without either.  The last tiles (the causal
+  // frontier or the speculative corner) take the general step.
+  auto step = [&](int kt, auto tail_tag) {
+    constexpr bool kTail = decltype(tail_tag)::value;
+    const int col0 = kt * kKeyTile + koff;
+    const bool work = kTail ? (col0 <= h + i_max) : true;
+    float s[2][4];
+    uint32_t p[1][4];
+    if (!dead && !mbar_wait(smem_u32(&bars->full[pipe.stage]), pipe.phase, a.status)) {
+      report_timeout(a);
+      dead = true;
+    }
+    if (work) w.qk(ring + pipe.stage * kTileBytes, koff, lane, s);
+    __syncwarp();
+    if (lane == 0) mbar_arrive(smem_u32(&bars->empty[pipe.stage]));
+    pipe.advance();
+    if (work) {
+      const bool need_mask = kTail ? (tree ? (col0 + 16 > h) : (col0 + 16 > h + tv.t.tok0 + 1)) : false;
+      w.softmax(a, tv.rq, s, p, col0, i_lo, i_hi, need_mask, scale_log2, lane);
+    }
+    if (!dead && !mbar_wait(smem_u32(&bars->full[pipe.stage]), pipe.phase, a.status)) {
+      report_timeout(a);
+      dead = true;
+    }
+    if (work) w.pv(ring + pipe.stage * kTileBytes, koff, lane, p);
+    __syncwarp();
+    if (lane == 0) mbar_arrive(smem_u32(&bars->empty[pipe.stage]));
+    pipe.advance();
+  };
+  const int full_cols = tree ? h : h + tv.t.tok0 + 1;  // columns below this are visible to every row
+  const int kt_mid = max(tv.t.kt_lo, min(tv.t.kt_hi, full_cols / kKeyTile));
+  int kt = tv.t.kt_lo;
+  for (; kt < kt_mid; ++kt) step(kt, std::false_type{});
+  for (; kt < tv.t.kt_hi; ++kt) step(kt, std::true_type{});
+  // ---- merge the eight warps' partials (in-CTA Update stage)
+  w.reduce_l();
+  named_bar_sync(1, kConsumerThreads);  // every warp holds its Q fragments: Q smem is free
+  {
+    const int xl = lane >> 2, xh = xl + 8;
+    float* mine = xch + warp * (16 * kHeadDim);
+#pragma unroll
+    for (int n = 0; n < 16; ++n) {
+      const int col = n * 8 + 2 * (lane & 3);
+      *reinterpret_cast<float2*>(mine + xl * kHeadDim + col) = make_float2(w.o[n][0], w.o[n][1]);
+      *reinterpret_cast<float2*>(mine + xh * kHeadDim + col) = make_float2(w.o[n][2], w.o[n][3]);
+    }
+    if ((lane & 3) == 0) {
+      ml[(warp * 16 + xl) * 2 + 0] = w.m_lo;
+      ml[(warp * 16 + xl) * 2 + 1] = w.l_lo;
+      ml[(warp * 16 + xh) * 2 + 0] = w.m_hi;
+      ml[(warp * 16 + xh) * 2 + 1] = w.l_hi;
+    }
+  }
+  named_bar_sync(1, kConsumerThreads);
+  {
+    const int x = threadIdx.x >> 4, seg = threadIdx.x & 15;  // row, 8-column segment
+    if (x < tv.rows) {
+      float M = -INFINITY;
+#pragma unroll
+      for (int ww = 0; ww < kConsumerWarps; ++ww) M = fmaxf(M, ml[(ww * 16 + x) * 2]);
+      float L = 0.f, acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int ww = 0; ww < kConsumerWarps; ++ww) {
+        const float mw = ml[(ww * 16 + x) * 2], lw = ml[(ww * 16 + x) * 2 + 1];
+        if (mw == -INFINITY) continue;
+        const float f = ex2(mw - M);
+        L += f * lw;
+        const float4* src = reinterpret_cast<const float4*>(xch + ww * (16 * kHeadDim) + x * kHeadDim + seg * 8);
+        const float4 v0 = src[0], v1 = src[1];
+        acc[0] += f * v0.x; acc[1] += f * v0.y; acc[2] += f * v0.z; acc[3] += f * v0.w;
+        acc[4] += f * v1.x; acc[5] += f * v1.y; acc[6] += f * v1.z; acc[7] += f * v1.w;
+      }
+      const float inv = L > 0.f ? 1.f / L : 0.f;
+#pragma unroll
+      for (int e = 0; e < 8; e += 2)
+        write_row_pair(a, tv, x, seg * 8 + e, acc[e] * inv, acc[e + 1] * inv);
+      if (seg == 0) write_lse(a, tv, x, L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY);
+    }
+  }
+  return static_cast<uint32_t>(pipe.stage) | (pipe.phase << 8) | (dead ? 1u << 16 : 0u);
+}
+
+// ------------------------------------------------------------------------------------------
 // tcgen05 dense path.  TMEM columns: S_A [0,128) S_B [128,256) O_A [256,384) O_B [384,512);
 // P (bf16, two keys per 32-bit column) overwrites the first 64 columns of its S block.
 constexpr uint32_t kTmemCols = 512;
@@ -416,7 +523,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
   if (threadIdx.x == 0) {
     unsigned long long now;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
-    a.worker_times[2 * blockIdx.x] = now;
+    a.worker_times[4 * blockIdx.x] = now;
     for (int s = 0; s < kStages; ++s) {
       mbar_init(smem_u32(&bars->full[s]), 1);
       mbar_init(smem_u32(&bars->empty[s]), kConsumerWarps);
@@ -758,6 +865,16 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
     Tracer tr;
     tr.init(a, warp >> 2, (threadIdx.x & 127) == 0);
     const int X = warp >> 2;       // sub-tile this warpgroup owns on the tcgen05 path
+    unsigned long long ns_kind[2] = {0ull, 0ull}, t_prev = 0ull;  // time in dense / streaming tasks
+    if (threadIdx.x == 0) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_prev));
+    int prev_kind = -1;
+    auto account = [&](int kind_now) {  // called by thread 0 at every task boundary
+      unsigned long long now;
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+      if (prev_kind >= 0) ns_kind[prev_kind] += now - t_prev;
+      t_prev = now;
+      prev_kind = kind_now;
+    };
     for (int ti = next_task(true); ti >= 0; ti = next_task(true)) {
       TaskView tv;
       tv.t = a.tasks[ti];
@@ -767,6 +884,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
       const int h = tv.rq.kv_len;
       const bool tree = tv.rq.mask_kind == XY_MASK_TREE;
       const bool stream = tv.t.kind == 1;
+      if (threadIdx.x == 0) account(stream ? 1 : 0);
 
       if (kUmma && !stream) {
         // ---------------- dense on tcgen05: this thread owns packed row x of sub-tile X ----
@@ -1036,87 +1154,19 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
         }
         named_bar_sync(1, kConsumerThreads);  // Q tile may be overwritten by the next task
       } else {
-        // ---------------- streaming: this warp owns keys koff .. koff+15 of every tile ----
-        const int koff = warp * 16;
-        WarpTile<2, false> w;
-        w.init();
-        w.load_q(q_smem, 0, lane);
-        const int r_lo = min(lane >> 2, tv.rows - 1), r_hi = min((lane >> 2) + 8, tv.rows - 1);
-        const int i_lo = tv.t.tok0 + r_lo / G, i_hi = tv.t.tok0 + r_hi / G;
-        const int i_max = tv.t.tok0 + tv.t.ntok - 1;
-        for (int kt = tv.t.kt_lo; kt < tv.t.kt_hi; ++kt) {
-          const int col0 = kt * kKeyTile + koff;
-          const bool work = col0 <= h + i_max;
-          float s[2][4];
-          uint32_t p[1][4];
-          if (!dead && !mbar_wait(smem_u32(&bars->full[pipe.stage]), pipe.phase, a.status)) {
-            report_timeout(a);
-            dead = true;
-          }
-          if (work) w.qk(ring + pipe.stage * kTileBytes, koff, lane, s);
-          __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&bars->empty[pipe.stage]));
-          pipe.advance();
-          if (work) {
-            const bool need_mask = tree ? (col0 + 16 > h) : (col0 + 16 > h + tv.t.tok0 + 1);
-            w.softmax(a, tv.rq, s, p, col0, i_lo, i_hi, need_mask, scale_log2, lane);
-          }
-          if (!dead && !mbar_wait(smem_u32(&bars->full[pipe.stage]), pipe.phase, a.status)) {
-            report_timeout(a);
-            dead = true;
-          }
-          if (work) w.pv(ring + pipe.stage * kTileBytes, koff, lane, p);
-          __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&bars->empty[pipe.stage]));
-          pipe.advance();
-        }
-        // ---- merge the eight warps' partials (in-CTA Update stage)
-        w.reduce_l();
-        named_bar_sync(1, kConsumerThreads);  // every warp holds its Q fragments: Q smem is free
-        {
-          const int xl = lane >> 2, xh = xl + 8;
-          float* mine = xch + warp * (16 * kHeadDim);
-#pragma unroll
-          for (int n = 0; n < 16; ++n) {
-            const int col = n * 8 + 2 * (lane & 3);
-            *reinterpret_cast<float2*>(mine + xl * kHeadDim + col) = make_float2(w.o[n][0], w.o[n][1]);
-            *reinterpret_cast<float2*>(mine + xh * kHeadDim + col) = make_float2(w.o[n][2], w.o[n][3]);
-          }
-          if ((lane & 3) == 0) {
-            ml[(warp * 16 + xl) * 2 + 0] = w.m_lo;
-            ml[(warp * 16 + xl) * 2 + 1] = w.l_lo;
-            ml[(warp * 16 + xh) * 2 + 0] = w.m_hi;
-            ml[(warp * 16 + xh) * 2 + 1] = w.l_hi;
-          }
-        }
-        named_bar_sync(1, kConsumerThreads);
-        {
-          const int x = threadIdx.x >> 4, seg = threadIdx.x & 15;  // row, 8-column segment
-          if (x < tv.rows) {
-            float M = -INFINITY;
-#pragma unroll
-            for (int ww = 0; ww < kConsumerWarps; ++ww) M = fmaxf(M, ml[(ww * 16 + x) * 2]);
-            float L = 0.f, acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int ww = 0; ww < kConsumerWarps; ++ww) {
-              const float mw = ml[(ww * 16 + x) * 2], lw = ml[(ww * 16 + x) * 2 + 1];
-              if (mw == -INFINITY) continue;
-              const float f = ex2(mw - M);
-              L += f * lw;
-              const float4* src = reinterpret_cast<const float4*>(xch + ww * (16 * kHeadDim) + x * kHeadDim + seg * 8);
-              const float4 v0 = src[0], v1 = src[1];
-              acc[0] += f * v0.x; acc[1] += f * v0.y; acc[2] += f * v0.z; acc[3] += f * v0.w;
-              acc[4] += f * v1.x; acc[5] += f * v1.y; acc[6] += f * v1.z; acc[7] += f * v1.w;
-            }
-            const float inv = L > 0.f ? 1.f / L : 0.f;
-#pragma unroll
-            for (int e = 0; e < 8; e += 2)
-              write_row_pair(a, tv, x, seg * 8 + e, acc[e] * inv, acc[e + 1] * inv);
-            if (seg == 0) write_lse(a, tv, x, L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY);
-          }
-        }
+        // ---------------- streaming: compiled as a function of its own (see stream_task) ----
+        const uint32_t st = stream_task(a, tv, q_smem, ring, bars, xch, ml, pipe.stage | (pipe.phase << 8) |
+                                        (dead ? 1u << 16 : 0u), scale_log2);
+        pipe.stage = st & 0xFFu;
+        pipe.phase = (st >> 8) & 1u;
+        dead = (st >> 16) & 1u;
         named_bar_sync(1, kConsumerThreads);
       }
+    }
+    if (threadIdx.x == 0) {
+      account(-1);
+      a.worker_times[4 * blockIdx.x + 2] = ns_kind[0];
+      a.worker_times[4 * blockIdx.x + 3] = ns_kind[1];
     }
   }
   tc_fence_before();
@@ -1124,7 +1174,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
   if (threadIdx.x == 0) {
     unsigned long long now;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
-    a.worker_times[2 * blockIdx.x + 1] = now;
+    a.worker_times[4 * blockIdx.x + 1] = now;
   }
   if (kUmma && warp == kConsumerWarps + 1) {
     tc_fence_after();
