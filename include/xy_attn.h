@@ -242,6 +242,9 @@ int xy_attn_get_worker_offsets(const xy_attn_ctx* ctx, int32_t* out /* num_worke
 int xy_attn_get_merge_units(const xy_attn_ctx* ctx, xy_attn_merge_unit* out, int32_t cap);
 int xy_attn_get_tree_mask(const xy_attn_ctx* ctx, uint64_t* out, int32_t cap_words);
 int xy_attn_get_q_start(const xy_attn_ctx* ctx, int32_t* out /* num_reqs+1 */, int32_t cap);
+/* The order in which free workers take tasks (indices into the task table, a permutation of it)
+ * when the plan is dealt dynamically: XY_PLAN_BALANCED with the MMA kernels. */
+int xy_attn_get_queue(const xy_attn_ctx* ctx, int32_t* out /* num_tasks */, int32_t cap);
 
 /* Per-kernel device timing.  With timing enabled every xy_attn_run records CUDA events on
  * its stream around the attention launch and around the merge launch (at most 4096 runs

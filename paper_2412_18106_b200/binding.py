@@ -74,7 +74,7 @@ EXPORTS = (
     "xy_attn_get_merge_units", "xy_attn_get_tree_mask", "xy_attn_get_q_start",
     "xy_attn_last_launches", "xy_attn_last_error", "xy_attn_device_status",
     "xy_attn_set_timing", "xy_attn_get_timing", "xy_attn_debug_trace", "xy_attn_decode_static",
-    "xy_attn_append_kv", "xy_attn_worker_times",
+    "xy_attn_append_kv", "xy_attn_worker_times", "xy_attn_get_queue",
 )
 
 _lib = None
@@ -100,7 +100,7 @@ def load() -> ctypes.CDLL:
     L.xy_attn_append_kv.argtypes = [vp, vp, i64, vp, vp, i64, i64, i64, i64, vp, i32, vp]
     L.xy_attn_debug_gather.argtypes = [vp, i32, i32, vp, vp, i64, i64, i64, vp, i32, vp, vp, vp]
     for name in ("xy_attn_get_tasks", "xy_attn_get_worker_offsets", "xy_attn_get_merge_units",
-                 "xy_attn_get_tree_mask", "xy_attn_get_q_start"):
+                 "xy_attn_get_tree_mask", "xy_attn_get_q_start", "xy_attn_get_queue"):
         getattr(L, name).argtypes = [vp, vp, i32]
     L.xy_attn_set_timing.argtypes = [vp, i32]
     L.xy_attn_get_timing.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float),
@@ -247,6 +247,9 @@ class XYAttn:
 
     def get_q_start(self) -> np.ndarray:
         return self._get(self.lib.xy_attn_get_q_start, np.int32)
+
+    def get_queue(self) -> np.ndarray:
+        return self._get(self.lib.xy_attn_get_queue, np.int32)
 
     def set_timing(self, enable: bool) -> None:
         self._check(self.lib.xy_attn_set_timing(self._ctx, 1 if enable else 0))

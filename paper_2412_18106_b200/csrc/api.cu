@@ -436,6 +436,7 @@ XY_GETTER(xy_attn_get_worker_offsets, int32_t, worker_off)
 XY_GETTER(xy_attn_get_merge_units, xy_attn_merge_unit, merges)
 XY_GETTER(xy_attn_get_tree_mask, uint64_t, tree_mask)
 XY_GETTER(xy_attn_get_q_start, int32_t, q_start)
+XY_GETTER(xy_attn_get_queue, int32_t, queue)
 
 int xy_attn_worker_times(xy_attn_ctx* ctx, uint64_t* out, int32_t cap) {
   if (ctx == nullptr || (out == nullptr && cap > 0)) return XY_ERR_INVALID_ARG;

@@ -19,12 +19,13 @@ namespace xy {
 namespace {
 
 // Per-SM time model in microseconds (free design constants; parity does not depend on them).
-// Measured on B200 with the cycle-stamp trace: a dense task advances one key tile per ~3400
-// cycles whether one or both of its 128-row sub-tiles are in use (the softmax -> MMA chain of a
-// sub-tile sets the pace and the two sub-tiles overlap each other); a streaming task one key tile
-// per ~2700 cycles; a task boundary costs ~6000 cycles (Q load, pipeline refill, epilogue).
-constexpr float kDenseVisitUs = 1.80f;
-constexpr float kStreamVisitUs = 1.40f;
+// Measured on B200 from the per-worker time each kind of task takes: a dense task advances one
+// key tile per 2.2 - 2.6 us whether one or both of its 128-row sub-tiles are in use (the softmax
+// -> MMA chain of a sub-tile sets the pace and the two sub-tiles overlap each other); a streaming
+// task one key tile per ~1.0 us while HBM is not saturated (1.4 us when every SM streams); a
+// task boundary costs ~3 us (Q load, pipeline refill, epilogue).
+constexpr float kDenseVisitUs = 2.30f;
+constexpr float kStreamVisitUs = 1.00f;
 constexpr float kTaskFixedUs = 3.0f;
 constexpr int kMinChunkTiles = 4;
 // A task may cost at most this fraction of the mean per-worker load before its KV range is
@@ -34,6 +35,7 @@ constexpr float kTaskCapFraction = 0.77f;
 // Dense tasks are split a little finer (cap x 0.65): their per-task overhead is small next to a
 // key-tile visit, and finer dense tasks even out the tail of the dynamically dealt queue.
 constexpr float kDenseCapFactor = 0.65f;
+
 
 struct Unit {
   int32_t req, kv_head, tok0, ntok, kind;
@@ -275,9 +277,41 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
     lsum += load;
   }
 
-  // The same sorted list as one queue, for workers that take tasks as they become free.
+  // The queue for workers that take tasks as they become free.  Paper mode: the sorted list.
+  // Balanced mode: the dense and the streaming tasks, each in descending order of cost, merged
+  // so that at every point of the queue the two kinds have handed out the same fraction of
+  // their total cost.  Dense tasks are bound by the SM (tensor pipe + softmax), streaming tasks
+  // by HBM; a queue that hands out all of one kind first makes every SM stream at once (HBM
+  // saturates) and then leaves HBM idle, while the mixed order keeps both busy throughout.
   out->queue.resize(order.size());
-  for (size_t pos = 0; pos < order.size(); ++pos) out->queue[pos] = where[order[pos]];
+  if (paper) {
+    for (size_t pos = 0; pos < order.size(); ++pos) out->queue[pos] = where[order[pos]];
+  } else {
+    std::vector<int> by_kind[2];
+    double total[2] = {0.0, 0.0}, given[2] = {0.0, 0.0};
+    for (int id : order) {
+      const int kd = pend[id].t.kind == 1 ? 1 : 0;
+      by_kind[kd].push_back(id);
+      total[kd] += pend[id].cost;
+    }
+    size_t next[2] = {0, 0};
+    for (size_t pos = 0; pos < order.size(); ++pos) {
+      int kd;
+      if (next[0] >= by_kind[0].size()) kd = 1;
+      else if (next[1] >= by_kind[1].size()) kd = 0;
+      else {
+        // A task must start while at least its own length of work per worker remains, or it
+        // runs past the end of everything else: from that point on the longer head goes first.
+        const double remaining = (total[0] + total[1] - given[0] - given[1]) / C;
+        const float c0 = pend[by_kind[0][next[0]]].cost, c1 = pend[by_kind[1][next[1]]].cost;
+        if (std::max(c0, c1) > remaining) kd = c0 >= c1 ? 0 : 1;
+        else kd = (given[0] * total[1] <= given[1] * total[0]) ? 0 : 1;
+      }
+      const int id = by_kind[kd][next[kd]++];
+      given[kd] += pend[id].cost;
+      out->queue[pos] = where[id];
+    }
+  }
 
   xy_attn_plan_info& info = out->info;
   info.num_tasks = static_cast<int32_t>(out->tasks.size());

@@ -155,6 +155,9 @@ def coverage_check(batch, ctx, info):
     keys = {(t["req"], t["kv_head"], t["tok0"]) for t in unsplit}
     assert len(keys) == len(unsplit)
     assert info.num_tasks == len(tasks) and info.num_merge_units == len(merges)
+    # the queue free workers take tasks from is a permutation of the task table
+    queue = ctx.get_queue()
+    assert sorted(queue.tolist()) == list(range(len(tasks)))
 
 
 @pytest.mark.parametrize("name", ["tiny_hybrid", "decode_only", "splitfuse_mix", "verify_trees", "full_mix"])
@@ -172,6 +175,25 @@ def test_balanced_plan_invariants_on_configs(name):
     t1 = c.get_tasks().copy()
     c.plan_batch(b)
     assert np.array_equal(t1, c.get_tasks())
+
+
+def test_queue_mixes_kinds_and_puts_long_tasks_early():
+    """Balanced plans hand out dense and streaming tasks side by side (each kind in descending
+    order of key tiles), and no long task is left for the end of the queue."""
+    b = W.CONFIGS["splitfuse_mix"]()
+    c = host_ctx(b.num_q_heads, b.num_kv_heads, b.page_size)
+    info = c.plan_batch(b)
+    tasks, queue = c.get_tasks(), c.get_queue()
+    kinds = tasks["kind"][queue]
+    ntiles = (tasks["kt_hi"] - tasks["kt_lo"])[queue]
+    first = kinds[: info.num_workers]
+    assert 0 < int(first.sum()) < info.num_workers  # both kinds among the first tasks handed out
+    for kd in (0, 1):
+        seq = ntiles[kinds == kd]
+        assert np.all(np.diff(seq) <= 0)
+    # the last tenth of the queue holds only tasks shorter than the median task
+    tail = ntiles[-len(queue) // 10:]
+    assert tail.max() <= np.median(ntiles)
 
 
 def test_plan_edge_shapes():
