@@ -333,10 +333,8 @@ __device__ __forceinline__ void report_timeout(const RunArgs& a) {
 // tails of prefill chunks), run by the eight consumer warps.  Every warp owns 16 keys of each
 // 128-key tile, keeps its own online-softmax state over those keys, and the eight partial
 // results are merged through shared memory when the task ends (the in-CTA Update stage of
-// Section 4.2.1).  It is a function of its own, not inlined into the kernel, so that the
-// register allocation of this bandwidth-critical loop is independent of the dense paths'.
-// pipe_state: ring stage | phase << 8 | dead << 16, returned updated.
-__device__ __noinline__ uint32_t stream_task(const RunArgs& a, const TaskView& tv, uint32_t q_smem, uint32_t ring,
+// Section 4.2.1).  pipe_state: ring stage | phase << 8 | dead << 16, returned updated.
+__device__ __forceinline__ uint32_t stream_task(const RunArgs& a, const TaskView& tv, uint32_t q_smem, uint32_t ring,
                                              SmemBarriers* bars, float* xch, float* ml, uint32_t pipe_state,
                                              float scale_log2) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -354,38 +352,58 @@ __device__ __noinline__ uint32_t stream_task(const RunArgs& a, const TaskView& t
   // Tiles that every row of the task sees in full need neither the mask nor the mask-aware
   // skip test; the loop over them is compiled without either.  The last tiles (the causal
   // frontier or the speculative corner) take the general step.
+#ifdef XY_ENABLE_TRACE
+  long long ph[6] = {0, 0, 0, 0, 0, 0};
+#define XY_PH(i) { const long long c_now = clock64(); ph[i] += c_now - c_prev; c_prev = c_now; }
+#else
+#define XY_PH(i)
+#endif
   auto step = [&](int kt, auto tail_tag) {
     constexpr bool kTail = decltype(tail_tag)::value;
     const int col0 = kt * kKeyTile + koff;
     const bool work = kTail ? (col0 <= h + i_max) : true;
     float s[2][4];
     uint32_t p[1][4];
+#ifdef XY_ENABLE_TRACE
+    long long c_prev = clock64();
+    ph[5] += 1;
+#endif
     if (!dead && !mbar_wait(smem_u32(&bars->full[pipe.stage]), pipe.phase, a.status)) {
       report_timeout(a);
       dead = true;
     }
+    XY_PH(0)
     if (work) w.qk(ring + pipe.stage * kTileBytes, koff, lane, s);
     __syncwarp();
     if (lane == 0) mbar_arrive(smem_u32(&bars->empty[pipe.stage]));
     pipe.advance();
+    XY_PH(1)
     if (work) {
       const bool need_mask = kTail ? (tree ? (col0 + 16 > h) : (col0 + 16 > h + tv.t.tok0 + 1)) : false;
       w.softmax(a, tv.rq, s, p, col0, i_lo, i_hi, need_mask, scale_log2, lane);
     }
+    XY_PH(2)
     if (!dead && !mbar_wait(smem_u32(&bars->full[pipe.stage]), pipe.phase, a.status)) {
       report_timeout(a);
       dead = true;
     }
+    XY_PH(3)
     if (work) w.pv(ring + pipe.stage * kTileBytes, koff, lane, p);
     __syncwarp();
     if (lane == 0) mbar_arrive(smem_u32(&bars->empty[pipe.stage]));
     pipe.advance();
+    XY_PH(4)
   };
   const int full_cols = tree ? h : h + tv.t.tok0 + 1;  // columns below this are visible to every row
   const int kt_mid = max(tv.t.kt_lo, min(tv.t.kt_hi, full_cols / kKeyTile));
   int kt = tv.t.kt_lo;
   for (; kt < kt_mid; ++kt) step(kt, std::false_type{});
   for (; kt < tv.t.kt_hi; ++kt) step(kt, std::true_type{});
+#ifdef XY_ENABLE_TRACE
+  if (a.trace != nullptr && blockIdx.x == 0 && threadIdx.x == 0)
+    for (int i = 0; i < 6; ++i) a.trace[4 * kTraceLen - 8 + i] += ph[i];
+#endif
+#undef XY_PH
   // ---- merge the eight warps' partials (in-CTA Update stage)
   w.reduce_l();
   named_bar_sync(1, kConsumerThreads);  // every warp holds its Q fragments: Q smem is free
@@ -865,15 +883,20 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
     Tracer tr;
     tr.init(a, warp >> 2, (threadIdx.x & 127) == 0);
     const int X = warp >> 2;       // sub-tile this warpgroup owns on the tcgen05 path
-    unsigned long long ns_kind[2] = {0ull, 0ull}, t_prev = 0ull;  // time in dense / streaming tasks
-    if (threadIdx.x == 0) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_prev));
-    int prev_kind = -1;
+    // Time this worker spends in dense / streaming tasks, kept by thread 0 in shared memory.
+    __shared__ unsigned long long acct_ns[2], acct_prev;
+    __shared__ int acct_kind;
+    if (threadIdx.x == 0) {
+      acct_ns[0] = acct_ns[1] = 0ull;
+      acct_kind = -1;
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(acct_prev));
+    }
     auto account = [&](int kind_now) {  // called by thread 0 at every task boundary
       unsigned long long now;
       asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
-      if (prev_kind >= 0) ns_kind[prev_kind] += now - t_prev;
-      t_prev = now;
-      prev_kind = kind_now;
+      if (acct_kind >= 0) acct_ns[acct_kind] += now - acct_prev;
+      acct_prev = now;
+      acct_kind = kind_now;
     };
     for (int ti = next_task(true); ti >= 0; ti = next_task(true)) {
       TaskView tv;
@@ -1154,7 +1177,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
         }
         named_bar_sync(1, kConsumerThreads);  // Q tile may be overwritten by the next task
       } else {
-        // ---------------- streaming: compiled as a function of its own (see stream_task) ----
+        // ---------------- streaming (see stream_task) ----
         const uint32_t st = stream_task(a, tv, q_smem, ring, bars, xch, ml, pipe.stage | (pipe.phase << 8) |
                                         (dead ? 1u << 16 : 0u), scale_log2);
         pipe.stage = st & 0xFFu;
@@ -1165,8 +1188,8 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
     }
     if (threadIdx.x == 0) {
       account(-1);
-      a.worker_times[4 * blockIdx.x + 2] = ns_kind[0];
-      a.worker_times[4 * blockIdx.x + 3] = ns_kind[1];
+      a.worker_times[4 * blockIdx.x + 2] = acct_ns[0];
+      a.worker_times[4 * blockIdx.x + 3] = acct_ns[1];
     }
   }
   tc_fence_before();
