@@ -908,6 +908,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
       const bool tree = tv.rq.mask_kind == XY_MASK_TREE;
       const bool stream = tv.t.kind == 1;
       if (threadIdx.x == 0) account(stream ? 1 : 0);
+      tr(30);
 
       if (kUmma && !stream) {
         // ---------------- dense on tcgen05: this thread owns packed row x of sub-tile X ----
@@ -943,6 +944,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
           cp_async_commit_wait_all();
           fence_proxy_async_smem();
           __syncwarp();
+          tr(29);
           if (lane == 0) mbar_arrive(smem_u32(&ub->q_full[X]));
         }
         const uint32_t lane_base = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
@@ -968,30 +970,45 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
           tr(22);
           const bool need_mask = tree ? (col0 + kKeyTile > h) : (col0 + kKeyTile > h + i_min + 1);
           if (need_mask) {
-            const int frontier = h + i_row;  // last visible column of this row
-            TreeWords tw;
-            tw.wbase = 0;
-            tw.w[0] = tw.w[1] = tw.w[2] = 0ull;
+            // 128-bit visibility mask of this row for columns col0 .. col0 + 127, built with word
+            // operations and applied with one test + select per element (no per-element branches).
+            const int nvis = min(max(h + i_row - col0 + 1, 0), kKeyTile);  // causal frontier
+            uint64_t v_lo = nvis >= 64 ? ~0ull : ((1ull << nvis) - 1ull);
+            uint64_t v_hi = nvis >= 128 ? ~0ull : (nvis <= 64 ? 0ull : ((1ull << (nvis - 64)) - 1ull));
             if (tree) {
-              const int jp0 = max(col0 - h, 0);
-              tw.wbase = jp0 >> 6;
+              // corner bit of column col is bit (col - h) of the row's ancestor-or-self words;
+              // columns below h (the cached prefix) are visible to every row.
+              const int jp0 = col0 - h;
+              const int wbase = max(jp0, 0) >> 6;
               const uint64_t* mrow = a.tree_mask + tv.rq.tree_off + static_cast<int64_t>(i_row) * tv.rq.tree_words;
-#pragma unroll
-              for (int q = 0; q < 3; ++q)
-                if (tw.wbase + q < tv.rq.tree_words) tw.w[q] = __ldg(mrow + tw.wbase + q);
-            }
-#pragma unroll
-            for (int k = 0; k < 128; ++k) {
-              const int col = col0 + k;
-              bool vis = col <= frontier;
-              if (tree && col >= h) {
-                const int jp = col - h;
-                const int wi = (jp >> 6) - tw.wbase;
-                const uint64_t word = wi == 0 ? tw.w[0] : (wi == 1 ? tw.w[1] : tw.w[2]);
-                vis = vis && ((word >> (jp & 63)) & 1ull);
+              uint64_t w0 = 0ull, w1 = 0ull, w2 = 0ull;
+              if (wbase < tv.rq.tree_words) w0 = __ldg(mrow + wbase);
+              if (wbase + 1 < tv.rq.tree_words) w1 = __ldg(mrow + wbase + 1);
+              if (wbase + 2 < tv.rq.tree_words) w2 = __ldg(mrow + wbase + 2);
+              uint64_t t_lo, t_hi;
+              if (jp0 >= 0) {
+                const int sh = jp0 & 63;
+                t_lo = sh ? ((w0 >> sh) | (w1 << (64 - sh))) : w0;
+                t_hi = sh ? ((w1 >> sh) | (w2 << (64 - sh))) : w1;
+              } else {
+                const int pre = -jp0;  // 1 .. 127 prefix columns lead the tile
+                if (pre < 64) {
+                  t_lo = ((1ull << pre) - 1ull) | (w0 << pre);
+                  t_hi = (w0 >> (64 - pre)) | (w1 << pre);
+                } else {
+                  const int p2 = pre - 64;
+                  t_lo = ~0ull;
+                  t_hi = p2 ? (((1ull << p2) - 1ull) | (w0 << p2)) : w0;
+                }
               }
-              if (!vis) sr[k] = 0xff800000u;  // -inf, selected (never added)
+              v_lo &= t_lo;
+              v_hi &= t_hi;
             }
+            const uint32_t vm[4] = {static_cast<uint32_t>(v_lo), static_cast<uint32_t>(v_lo >> 32),
+                                    static_cast<uint32_t>(v_hi), static_cast<uint32_t>(v_hi >> 32)};
+#pragma unroll
+            for (int k = 0; k < 128; ++k)
+              sr[k] = (vm[k >> 5] & (1u << (k & 31))) ? sr[k] : 0xff800000u;  // -inf, selected (never added)
           }
           float mx;
           {  // eight independent chains of three-input max, then a short tree
@@ -1070,6 +1087,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
         }
         ph_o ^= 1u;
         tc_fence_after();
+        tr(27);
         const float inv = l > 0.f ? 1.f / l : 0.f;
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
@@ -1101,6 +1119,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
         }
         if (valid) write_lse(a, tv, x, l > 0.f ? (m_ref + log2f(l)) * kLn2 : -INFINITY);
         tc_fence_before();  // order this task's TMEM reads before the next task's MMAs
+        tr(28);
         continue;
       }
 
