@@ -913,7 +913,11 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
       if (kUmma && !stream) {
         // ---------------- dense on tcgen05: this thread owns packed row x of sub-tile X ----
         const DenseShape ds = dense_shape(tv.t, tv.rq, G);
-        for (int c = 0; c < 2 * ds.n_all; ++c) pipe.advance();  // the ring moves on without us
+        {  // the ring moves on without us: 2 n_all positions
+          const uint32_t np = static_cast<uint32_t>(pipe.stage) + 2u * static_cast<uint32_t>(ds.n_all);
+          pipe.stage = static_cast<int>(np % kStages);
+          pipe.phase ^= (np / kStages) & 1u;
+        }
         const int r = (warp & 3) * 32 + lane;
         const int x = X * 128 + r;
         const bool exists = X * 128 < tv.rows;
@@ -930,17 +934,30 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
         }
         // packed Q sub-tile -> shared memory, then hand it to the async proxy
         {
+          // Thread t copies 16-byte chunk (t & 15) of rows (t >> 4) + 8 it; the (token, head) of
+          // a row advances by 8 packed rows per step, so one division per task suffices.
+          tr(31);
           const int t128 = threadIdx.x & 127;
-          for (int c = t128; c < 128 * 16; c += 128) {
-            const int rr = c >> 4, ch = c & 15;
-            const int xr = X * 128 + rr;
-            const bool ok = xr < tv.rows;
-            const int xx = ok ? xr : 0;
-            const int i = tv.t.tok0 + xx / G, head = tv.t.kv_head * G + xx % G;
-            const uint16_t* src =
-                a.q + static_cast<int64_t>(tv.rq.q_start + i) * a.q_token_stride + head * kHeadDim + ch * 8;
+          const int ch = t128 & 15;
+          const int x0 = X * 128 + (t128 >> 4);
+          int i_q = x0 / G, h_q = x0 - i_q * G;
+          const int di = 8 / G, dh = 8 - di * G;
+          const uint16_t* qbase = a.q + static_cast<int64_t>(tv.rq.q_start + tv.t.tok0) * a.q_token_stride +
+                                  static_cast<int64_t>(tv.t.kv_head) * G * kHeadDim + ch * 8;
+#pragma unroll 4
+          for (int it = 0; it < 16; ++it) {
+            const int rr = (t128 >> 4) + 8 * it;
+            const bool ok = X * 128 + rr < tv.rows;
+            const uint16_t* src = ok ? qbase + static_cast<int64_t>(i_q) * a.q_token_stride + h_q * kHeadDim : qbase;
             cp_async_16(q_smem + X * kTileBytes + swz(rr, ch), src, ok);
+            i_q += di;
+            h_q += dh;
+            if (h_q >= G) {
+              h_q -= G;
+              ++i_q;
+            }
           }
+          tr(32);
           cp_async_commit_wait_all();
           fence_proxy_async_smem();
           __syncwarp();
@@ -1089,26 +1106,59 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
         tc_fence_after();
         tr(27);
         const float inv = l > 0.f ? 1.f / l : 0.f;
+        if (tv.t.part < 0) {
+          // Final output.  A thread holds one row, so direct stores would touch 32 rows per warp
+          // instruction.  The bf16 rows go through this sub-tile's Q area of shared memory instead
+          // (its MMAs have completed; 16-byte chunks XOR-swizzled by row so that neither side has
+          // bank conflicts) and leave as row-contiguous 256-byte stores, two rows per instruction.
+          uint8_t* stage = gen_base + X * kTileBytes;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint32_t orow[32];
-          tmem_ld_32x32b_x32(t_o + c * 32, orow);
-          tmem_wait_ld();
-          if (valid) {
-            if (tv.t.part < 0) {
-              const int head = tv.t.kv_head * G + x % G;
-              uint4* dst = reinterpret_cast<uint4*>(a.o + static_cast<int64_t>(tv.rq.q_start + i_row) * a.o_token_stride +
-                                                    head * kHeadDim + c * 32);
+          for (int c = 0; c < 4; ++c) {
+            uint32_t orow[32];
+            tmem_ld_32x32b_x32(t_o + c * 32, orow);
+            tmem_wait_ld();
 #pragma unroll
-              for (int q = 0; q < 4; ++q) {
-                uint4 v;
-                v.x = pack_bf16(__uint_as_float(orow[q * 8 + 0]) * inv, __uint_as_float(orow[q * 8 + 1]) * inv);
-                v.y = pack_bf16(__uint_as_float(orow[q * 8 + 2]) * inv, __uint_as_float(orow[q * 8 + 3]) * inv);
-                v.z = pack_bf16(__uint_as_float(orow[q * 8 + 4]) * inv, __uint_as_float(orow[q * 8 + 5]) * inv);
-                v.w = pack_bf16(__uint_as_float(orow[q * 8 + 6]) * inv, __uint_as_float(orow[q * 8 + 7]) * inv);
-                dst[q] = v;
+            for (int q = 0; q < 4; ++q) {
+              uint4 v;
+              v.x = pack_bf16(__uint_as_float(orow[q * 8 + 0]) * inv, __uint_as_float(orow[q * 8 + 1]) * inv);
+              v.y = pack_bf16(__uint_as_float(orow[q * 8 + 2]) * inv, __uint_as_float(orow[q * 8 + 3]) * inv);
+              v.z = pack_bf16(__uint_as_float(orow[q * 8 + 4]) * inv, __uint_as_float(orow[q * 8 + 5]) * inv);
+              v.w = pack_bf16(__uint_as_float(orow[q * 8 + 6]) * inv, __uint_as_float(orow[q * 8 + 7]) * inv);
+              *reinterpret_cast<uint4*>(stage + r * 256 + (((c * 4 + q) ^ (r & 15)) << 4)) = v;
+            }
+          }
+          __syncwarp();
+          {
+            const int ch = lane & 15;
+            int rr = (warp & 3) * 32 + (lane >> 4);  // row of the sub-tile this lane stores first
+            const int xs = X * 128 + rr;
+            int i_o = xs / G, h_o = xs - i_o * G;
+            const int di = 2 / G, dh = 2 - di * G;
+            uint16_t* obase = a.o + static_cast<int64_t>(tv.rq.q_start + tv.t.tok0) * a.o_token_stride +
+                              static_cast<int64_t>(tv.t.kv_head) * G * kHeadDim + ch * 8;
+#pragma unroll 4
+            for (int it = 0; it < 16; ++it) {
+              if (X * 128 + rr < tv.rows) {
+                const uint4 v = *reinterpret_cast<const uint4*>(stage + rr * 256 + ((ch ^ (rr & 15)) << 4));
+                *reinterpret_cast<uint4*>(obase + static_cast<int64_t>(i_o) * a.o_token_stride + h_o * kHeadDim) = v;
               }
-            } else {
+              rr += 2;
+              i_o += di;
+              h_o += dh;
+              if (h_o >= G) {
+                h_o -= G;
+                ++i_o;
+              }
+            }
+          }
+          named_bar_sync(2 + X, 128);  // staging reads done before the next task's Q lands here
+        } else {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            uint32_t orow[32];
+            tmem_ld_32x32b_x32(t_o + c * 32, orow);
+            tmem_wait_ld();
+            if (valid) {
               float4* dst = reinterpret_cast<float4*>(a.o_part + static_cast<int64_t>(tv.t.part + x) * kHeadDim + c * 32);
 #pragma unroll
               for (int q = 0; q < 8; ++q)
