@@ -1112,19 +1112,21 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
           // (its MMAs have completed; 16-byte chunks XOR-swizzled by row so that neither side has
           // bank conflicts) and leave as row-contiguous 256-byte stores, two rows per instruction.
           uint8_t* stage = gen_base + X * kTileBytes;
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            uint32_t orow[32];
-            tmem_ld_32x32b_x32(t_o + c * 32, orow);
+          {
+            uint32_t orow[128];  // the whole row with one wait: four loads in flight together
+            tmem_ld_32x32b_x32(t_o, &orow[0]);
+            tmem_ld_32x32b_x32(t_o + 32, &orow[32]);
+            tmem_ld_32x32b_x32(t_o + 64, &orow[64]);
+            tmem_ld_32x32b_x32(t_o + 96, &orow[96]);
             tmem_wait_ld();
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
+            for (int q = 0; q < 16; ++q) {
               uint4 v;
               v.x = pack_bf16(__uint_as_float(orow[q * 8 + 0]) * inv, __uint_as_float(orow[q * 8 + 1]) * inv);
               v.y = pack_bf16(__uint_as_float(orow[q * 8 + 2]) * inv, __uint_as_float(orow[q * 8 + 3]) * inv);
               v.z = pack_bf16(__uint_as_float(orow[q * 8 + 4]) * inv, __uint_as_float(orow[q * 8 + 5]) * inv);
               v.w = pack_bf16(__uint_as_float(orow[q * 8 + 6]) * inv, __uint_as_float(orow[q * 8 + 7]) * inv);
-              *reinterpret_cast<uint4*>(stage + r * 256 + (((c * 4 + q) ^ (r & 15)) << 4)) = v;
+              *reinterpret_cast<uint4*>(stage + r * 256 + ((q ^ (r & 15)) << 4)) = v;
             }
           }
           __syncwarp();
