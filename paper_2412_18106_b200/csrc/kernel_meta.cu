@@ -1176,6 +1176,9 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
       }
 
       // ---- packed Q tile -> shared memory (rows past the tile are zero-filled)
+      // A warpgroup that had no sub-tile in the previous dense task arrives here while the other
+      // one may still be computing on its Q tile, which this load overwrites: meet first.
+      if (kUmma) named_bar_sync(1, kConsumerThreads);
       {
         const int rows_pad = stream ? 16 : 128;
         for (int c = threadIdx.x; c < rows_pad * 16; c += kConsumerThreads) {
