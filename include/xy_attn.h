@@ -142,6 +142,17 @@ int xy_attn_plan(xy_attn_ctx* ctx, const xy_attn_request* reqs /*HOST*/, int32_t
                  const int32_t* tree_parents /*HOST, nullable if no tree*/, int32_t num_parents,
                  void* stream, xy_attn_plan_info* info /*HOST, nullable*/);
 
+/* Task-Table cache (Section 3.3: the Task-Table is what the kernels consume; Section 3.3.2 keeps
+ * pre-built Task-Tables for recurring shapes).  xy_attn_plan keeps the Task-Tables of the last
+ * `capacity` distinct decompositions (default 8).  A plan whose decomposition — per request, kv
+ * head and q tile: token range, task kind and number of visible 128-key tiles — equals a cached
+ * one reuses that Task-Table (bit-identical to a fresh build) and, if it is the one already in
+ * the device tables, skips their upload; the Token-Table, the request facts and the tree masks
+ * are rebuilt and uploaded every time.  Consecutive decode steps change kvLen by one token and
+ * hit until a request crosses a 128-key tile.  capacity = -1 leaves the setting, 0 disables the
+ * cache; hits / misses (HOST, nullable) receive the counts since create. */
+int xy_attn_plan_cache(xy_attn_ctx* ctx, int32_t capacity, int64_t* hits /*HOST*/, int64_t* misses /*HOST*/);
+
 /* Meta-Attention over the planned batch (Sections 4.1-4.2, 5.2, 5.4).
  * Asynchronous on `stream`; no allocation, no host synchronisation.
  *   q            DEVICE bf16; row of token t, head a at q + t*q_token_stride + a*D

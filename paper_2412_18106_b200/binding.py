@@ -74,7 +74,7 @@ EXPORTS = (
     "xy_attn_get_merge_units", "xy_attn_get_tree_mask", "xy_attn_get_q_start",
     "xy_attn_last_launches", "xy_attn_last_error", "xy_attn_device_status",
     "xy_attn_set_timing", "xy_attn_get_timing", "xy_attn_debug_trace", "xy_attn_decode_static",
-    "xy_attn_append_kv", "xy_attn_worker_times", "xy_attn_get_queue",
+    "xy_attn_append_kv", "xy_attn_worker_times", "xy_attn_get_queue", "xy_attn_plan_cache",
 )
 
 _lib = None
@@ -107,6 +107,7 @@ def load() -> ctypes.CDLL:
                                      ctypes.POINTER(i32)]
     L.xy_attn_debug_trace.argtypes = [vp, vp, i32]
     L.xy_attn_worker_times.argtypes = [vp, vp, i32]
+    L.xy_attn_plan_cache.argtypes = [vp, i32, ctypes.POINTER(i64), ctypes.POINTER(i64)]
     L.xy_attn_decode_static.argtypes = [vp, i64, vp, vp, i64, i64, i64, vp, i32, vp, i32, i32, i32, i32, i32,
                                         ctypes.c_float, vp, i64, vp, vp]
     L.xy_attn_last_launches.argtypes = [vp]
@@ -250,6 +251,12 @@ class XYAttn:
 
     def get_queue(self) -> np.ndarray:
         return self._get(self.lib.xy_attn_get_queue, np.int32)
+
+    def plan_cache(self, capacity: int = -1):
+        """Sets the Task-Table cache capacity (-1: leave) and returns (hits, misses)."""
+        hits, misses = ctypes.c_int64(0), ctypes.c_int64(0)
+        self._check(self.lib.xy_attn_plan_cache(self._ctx, int(capacity), ctypes.byref(hits), ctypes.byref(misses)))
+        return int(hits.value), int(misses.value)
 
     def set_timing(self, enable: bool) -> None:
         self._check(self.lib.xy_attn_set_timing(self._ctx, 1 if enable else 0))

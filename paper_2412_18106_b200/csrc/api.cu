@@ -21,6 +21,9 @@ struct xy_attn_ctx {
   int page_shift = 0;
   bool planned = false;
   PlanResult plan;
+  PlanCache cache;                  // Task-Tables of recent plans
+  std::vector<int32_t> dev_shape;   // decomposition whose Task-Table is in the device tables
+  bool dev_shape_valid = false;
   // capacities of the device tables
   int64_t cap_tasks = 0, cap_merges = 0, cap_tree_words = 0, cap_partial_rows = 0;
   ReqInfo* d_reqs = nullptr;
@@ -186,7 +189,7 @@ int xy_attn_plan(xy_attn_ctx* ctx, const xy_attn_request* reqs, int32_t num_reqs
   ctx->planned = false;
   std::string err;
   int rc = build_plan(ctx->cfg, ctx->num_workers, ctx->cap_partial_rows, reqs, num_reqs,
-                      tree_parents, num_parents, &ctx->plan, &err);
+                      tree_parents, num_parents, &ctx->plan, &err, ctx->cache.capacity > 0 ? &ctx->cache : nullptr);
   if (rc != XY_OK) {
     ctx->plan = PlanResult();
     return set_err(ctx, rc, err);
@@ -205,21 +208,29 @@ int xy_attn_plan(xy_attn_ctx* ctx, const xy_attn_request* reqs, int32_t num_reqs
     if (!p.reqs.empty())
       XY_CUDA(ctx, cudaMemcpyAsync(ctx->d_reqs, p.reqs.data(), sizeof(ReqInfo) * p.reqs.size(),
                                    cudaMemcpyHostToDevice, s));
-    if (!p.tasks.empty())
-      XY_CUDA(ctx, cudaMemcpyAsync(ctx->d_tasks, p.tasks.data(),
-                                   sizeof(xy_attn_task) * p.tasks.size(), cudaMemcpyHostToDevice, s));
-    if (!p.queue.empty())
-      XY_CUDA(ctx, cudaMemcpyAsync(ctx->d_queue, p.queue.data(), sizeof(int32_t) * p.queue.size(),
-                                   cudaMemcpyHostToDevice, s));
-    XY_CUDA(ctx, cudaMemcpyAsync(ctx->d_worker_off, p.worker_off.data(),
-                                 sizeof(int32_t) * p.worker_off.size(), cudaMemcpyHostToDevice, s));
     if (!p.tree_mask.empty())
       XY_CUDA(ctx, cudaMemcpyAsync(ctx->d_tree, p.tree_mask.data(),
                                    sizeof(uint64_t) * p.tree_mask.size(), cudaMemcpyHostToDevice, s));
-    if (!p.merges.empty())
-      XY_CUDA(ctx, cudaMemcpyAsync(ctx->d_merges, p.merges.data(),
-                                   sizeof(xy_attn_merge_unit) * p.merges.size(),
-                                   cudaMemcpyHostToDevice, s));
+    // The Task-Table part stays on the device while the decomposition does not change (all of
+    // these copies are ordered on `stream`; a caller that plans on several streams must order them).
+    const bool same_tables = ctx->dev_shape_valid && ctx->dev_shape == p.shape;
+    ctx->dev_shape_valid = false;
+    if (!same_tables) {
+      if (!p.tasks.empty())
+        XY_CUDA(ctx, cudaMemcpyAsync(ctx->d_tasks, p.tasks.data(),
+                                     sizeof(xy_attn_task) * p.tasks.size(), cudaMemcpyHostToDevice, s));
+      if (!p.queue.empty())
+        XY_CUDA(ctx, cudaMemcpyAsync(ctx->d_queue, p.queue.data(), sizeof(int32_t) * p.queue.size(),
+                                     cudaMemcpyHostToDevice, s));
+      XY_CUDA(ctx, cudaMemcpyAsync(ctx->d_worker_off, p.worker_off.data(),
+                                   sizeof(int32_t) * p.worker_off.size(), cudaMemcpyHostToDevice, s));
+      if (!p.merges.empty())
+        XY_CUDA(ctx, cudaMemcpyAsync(ctx->d_merges, p.merges.data(),
+                                     sizeof(xy_attn_merge_unit) * p.merges.size(),
+                                     cudaMemcpyHostToDevice, s));
+      ctx->dev_shape = p.shape;
+    }
+    ctx->dev_shape_valid = true;
   }
   if (info) *info = p.info;
   ctx->planned = true;
@@ -437,6 +448,17 @@ XY_GETTER(xy_attn_get_merge_units, xy_attn_merge_unit, merges)
 XY_GETTER(xy_attn_get_tree_mask, uint64_t, tree_mask)
 XY_GETTER(xy_attn_get_q_start, int32_t, q_start)
 XY_GETTER(xy_attn_get_queue, int32_t, queue)
+
+int xy_attn_plan_cache(xy_attn_ctx* ctx, int32_t capacity, int64_t* hits, int64_t* misses) {
+  if (ctx == nullptr || capacity < -1) return XY_ERR_INVALID_ARG;
+  if (capacity >= 0) {
+    ctx->cache.capacity = static_cast<size_t>(capacity);
+    if (ctx->cache.entries.size() > ctx->cache.capacity) ctx->cache.entries.clear();
+  }
+  if (hits) *hits = static_cast<int64_t>(ctx->cache.hits);
+  if (misses) *misses = static_cast<int64_t>(ctx->cache.misses);
+  return XY_OK;
+}
 
 int xy_attn_worker_times(xy_attn_ctx* ctx, uint64_t* out, int32_t cap) {
   if (ctx == nullptr || (out == nullptr && cap > 0)) return XY_ERR_INVALID_ARG;

@@ -13,6 +13,8 @@
 #include <cstdio>
 #include <numeric>
 
+#include <climits>
+
 #include "xy_internal.h"
 
 namespace xy {
@@ -50,7 +52,7 @@ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
 int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_capacity,
                const xy_attn_request* reqs, int32_t num_reqs, const int32_t* tree_parents,
-               int32_t num_parents, PlanResult* out, std::string* err) {
+               int32_t num_parents, PlanResult* out, std::string* err, PlanCache* cache) {
   *out = PlanResult();
   char buf[256];
   auto fail = [&](int code, const char* msg) {
@@ -179,6 +181,50 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
         units.push_back(u);
       }
     }
+  }
+
+  // ---- Task-Table cache: everything below depends on the requests only through the units
+  // (request, kv head, q tile, kind, visible key tiles), so an equal decomposition has an equal
+  // Task-Table.  The useful-flop and byte counts depend on the exact kvLen and are always fresh.
+  out->shape.reserve(units.size() * 6 + 4);
+  out->shape.push_back(num_workers);
+  out->shape.push_back(static_cast<int32_t>(std::min<int64_t>(partial_row_capacity, INT32_MAX)));
+  out->shape.push_back(cfg.plan_mode * 4 + cfg.kernel);
+  out->shape.push_back(cfg.max_splits);
+  for (const Unit& u : units) {
+    out->shape.push_back(u.req);
+    out->shape.push_back(u.kv_head);
+    out->shape.push_back(u.tok0);
+    out->shape.push_back(u.ntok);
+    out->shape.push_back(u.kind);
+    out->shape.push_back(paper ? static_cast<int32_t>(reqs[u.req].kv_len) : u.nkt);
+  }
+  {
+    uint64_t hsh = 1469598103934665603ull;  // FNV-1a over the 32-bit words
+    for (int32_t v : out->shape) hsh = (hsh ^ static_cast<uint32_t>(v)) * 1099511628211ull;
+    out->shape_hash = hsh;
+  }
+  const int64_t flops_now = 4ll * kHeadDim * cfg.num_q_heads * pairs;
+  const int64_t kv_bytes_now = 2ll * kv_tokens * cfg.num_kv_heads * kHeadDim * 2;
+  if (cache != nullptr) {
+    ++cache->clock;
+    for (PlanCache::Entry& e : cache->entries) {
+      if (e.hash != out->shape_hash || e.shape != out->shape) continue;
+      e.last_use = cache->clock;
+      ++cache->hits;
+      out->tasks = e.tasks;
+      out->task_cost = e.task_cost;
+      out->worker_off = e.worker_off;
+      out->queue = e.queue;
+      out->merges = e.merges;
+      out->partial_rows = e.partial_rows;
+      out->info = e.info;
+      out->info.useful_flops = flops_now;
+      out->info.kv_bytes = kv_bytes_now;
+      out->from_cache = true;
+      return XY_OK;
+    }
+    ++cache->misses;
   }
 
   // KV splits: cap the cost of one task at a fraction of the mean per-worker load.
@@ -318,13 +364,34 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
   info.num_dense_tasks = ndense;
   info.num_merge_units = static_cast<int32_t>(out->merges.size());
   info.num_workers = C;
-  info.useful_flops = 4ll * kHeadDim * cfg.num_q_heads * pairs;
-  info.kv_bytes = 2ll * kv_tokens * cfg.num_kv_heads * kHeadDim * 2;
+  info.useful_flops = flops_now;
+  info.kv_bytes = kv_bytes_now;
   info.partial_rows = prow;
   info.load_min = lmin;
   info.load_mean = lsum / C;
   info.load_max = lmax;
   info.max_task_cost = tmax;
+  if (cache != nullptr && cache->capacity > 0) {
+    PlanCache::Entry* slot = nullptr;
+    if (cache->entries.size() < cache->capacity) {
+      cache->entries.emplace_back();
+      slot = &cache->entries.back();
+    } else {
+      slot = &cache->entries[0];
+      for (PlanCache::Entry& e : cache->entries)
+        if (e.last_use < slot->last_use) slot = &e;
+    }
+    slot->shape = out->shape;
+    slot->hash = out->shape_hash;
+    slot->tasks = out->tasks;
+    slot->task_cost = out->task_cost;
+    slot->worker_off = out->worker_off;
+    slot->queue = out->queue;
+    slot->merges = out->merges;
+    slot->partial_rows = out->partial_rows;
+    slot->info = out->info;
+    slot->last_use = cache->clock;
+  }
   return XY_OK;
 }
 

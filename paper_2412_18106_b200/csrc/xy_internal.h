@@ -38,15 +38,41 @@ struct PlanResult {
   int64_t partial_rows = 0;
   int64_t total_q = 0;
   xy_attn_plan_info info{};
+  // Identity of the Task-Table part (tasks, worker_off, queue, merges): the decomposition it was
+  // built from.  Two plans with equal `shape` have identical Task-Tables even when the requests'
+  // kvLen differ (a decode step moves kvLen by one token but rarely crosses a 128-key tile).
+  std::vector<int32_t> shape;
+  uint64_t shape_hash = 0;
+  bool from_cache = false;
+};
+
+// Task-Tables of recent plans, keyed by their decomposition (least recently used goes first).
+struct PlanCache {
+  struct Entry {
+    std::vector<int32_t> shape;
+    uint64_t hash = 0;
+    std::vector<xy_attn_task> tasks;
+    std::vector<float> task_cost;
+    std::vector<int32_t> worker_off, queue;
+    std::vector<xy_attn_merge_unit> merges;
+    int64_t partial_rows = 0;
+    xy_attn_plan_info info{};
+    uint64_t last_use = 0;
+  };
+  std::vector<Entry> entries;
+  size_t capacity = 8;
+  uint64_t clock = 0, hits = 0, misses = 0;
 };
 
 // 128-row sub-tiles one dense task may hold (the tcgen05 path ping-pongs two; the others one).
 inline int dense_subtiles(const xy_attn_config& cfg) { return cfg.kernel == XY_KERNEL_AUTO ? 2 : 1; }
 
 // Host-only planning.  Returns XY_OK or an error code and fills `err`.
+// `cache` (nullable): Task-Tables of earlier plans; a plan whose decomposition equals a cached one
+// takes its Task-Table from there and only rebuilds the Token-Table and the tree masks.
 int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_capacity,
                const xy_attn_request* reqs, int32_t num_reqs, const int32_t* tree_parents,
-               int32_t num_parents, PlanResult* out, std::string* err);
+               int32_t num_parents, PlanResult* out, std::string* err, PlanCache* cache = nullptr);
 
 // Arguments every attention kernel takes.
 struct RunArgs {

@@ -202,3 +202,27 @@ def test_run_error_paths_do_not_launch():
                              d.block_table.data_ptr(), 1, 0, 1.0, d.o.data_ptr(), 1024, d.lse.data_ptr(), 0)
     assert rc == xb.XY_ERR_INVALID_ARG
     assert ctx.last_launches() == 0
+
+
+def test_consecutive_steps_through_the_task_table_cache():
+    """Three decode steps on one context: the second and third plan hit the Task-Table cache and
+    leave the Task-Table on the device as it is (only the request facts are uploaded); each step
+    must still match the oracle, including the step where a request enters a new key tile."""
+    rng = np.random.default_rng(11)
+    kv = [int(x) for x in rng.integers(130, 900, size=12)]
+    kv[0] = 254  # crosses into its third 128-key tile at the third step
+    tree = W.random_tree(rng, 12, 4)
+    ctx = None
+    for step in range(4):
+        reqs = [(1, h + step, 0, None) for h in kv] + [(40, 100, 0, None), (12, 300 + step, 1, tree)]
+        b = W.custom("steps%d" % step, 8, 2, 32, reqs, seed=3)
+        t = W.make_tensors(b)
+        if ctx is None:
+            ctx = H.make_ctx(b)
+        ctx.plan_batch(b)
+        O, LSE = H.run_gpu(b, t, ctx=ctx)
+        O_ref, LSE_ref = oracle.attention(b, t, H.SCALE)
+        H.check_against_oracle(O, LSE, O_ref, LSE_ref, "step %d" % step)
+    hits, misses = ctx.plan_cache()
+    assert hits >= 1 and misses >= 2 and hits + misses == 4
+    ctx.close()

@@ -245,3 +245,42 @@ def test_paper_mode_equals_python_task_table_and_fig3b():
     assert owners == [0, 1, 2, 3, 3, 2, 1, 0]
     coverage_check(W.custom("fig3b", hq, hkv, 16, [(300, 0, 0, None), (1, 700, 0, None),
                                                    (16, 900, 1, W.chain_tree(16)), (1, 350, 0, None)]), c, info)
+
+
+def test_task_table_cache_reuses_equal_decompositions_bit_exactly():
+    """A decode step moves every kvLen by one token; while no request crosses a 128-key tile the
+    decomposition, hence the Task-Table, is unchanged: the plan comes from the cache and is
+    bit-identical to a fresh context's plan.  Crossing a tile (or any other change) misses."""
+    rng = np.random.default_rng(5)
+    kv = rng.integers(200, 5000, size=24)
+    kv = kv - (kv % 128) + rng.integers(1, 60, size=24)  # at least 60 steps before a tile ends
+    reqs = [(1, int(x), 0, None) for x in kv] + [(700, 300, 0, None)]
+    c = host_ctx(8, 2, 128)
+    b0 = W.custom("s0", 8, 2, 128, reqs, seed=1)
+    c.plan_batch(b0)
+    assert c.plan_cache() == (0, 1)
+    for step in range(1, 4):
+        reqs_s = [(1, int(x) + step, 0, None) for x in kv] + [(700, 300, 0, None)]
+        b = W.custom("s%d" % step, 8, 2, 128, reqs_s, seed=1)
+        info = c.plan_batch(b)
+        assert c.plan_cache() == (step, 1)
+        fresh = host_ctx(8, 2, 128)
+        info_f = fresh.plan_batch(b)
+        assert np.array_equal(c.get_tasks(), fresh.get_tasks())
+        assert np.array_equal(c.get_queue(), fresh.get_queue())
+        assert np.array_equal(c.get_worker_offsets(), fresh.get_worker_offsets())
+        assert np.array_equal(c.get_merge_units(), fresh.get_merge_units())
+        assert (info.useful_flops, info.kv_bytes) == (info_f.useful_flops, info_f.kv_bytes)
+        assert info.useful_flops == W.useful_flops(b)
+        coverage_check(b, c, info)
+    # one request crosses into its next key tile: different decomposition
+    reqs_x = [(1, int(kv[0]) + 128, 0, None)] + [(1, int(x), 0, None) for x in kv[1:]] + [(700, 300, 0, None)]
+    c.plan_batch(W.custom("x", 8, 2, 128, reqs_x, seed=1))
+    assert c.plan_cache() == (3, 2)
+    # back to the first shape: still cached
+    c.plan_batch(b0)
+    assert c.plan_cache() == (4, 2)
+    # disabled: every plan is built
+    assert c.plan_cache(0) == (4, 2)
+    c.plan_batch(b0)
+    assert c.plan_cache() == (4, 2)
