@@ -238,6 +238,102 @@ def measure_other(name, kernel, dev, peaks, steps=20, warmup=3):
             "steps": steps}
 
 
+def measure_stream(kernel, dev, peaks, chunks=48, budget=4096, reserved=512, sessions=96, seed=0):
+    """A serving-like request stream through the scheduling front (Section 3.1): sessions arrive
+    with prompts (prefix-cache hits included), then decode one token per step, a fifth of them
+    verify a token tree instead; the chunk former cuts fixed-budget chunks, every chunk is planned
+    (Task-Table cache on) and run.  K/V pool and Q are random and resident; the block table maps
+    every session onto random pages of one pool (contents do not matter for timing).  Reports the
+    host time of chunk forming and planning and the device time of attention per chunk."""
+    import torch
+
+    from paper_2412_18106_b200 import binding as xb
+    from paper_2412_18106_b200 import sched as xs
+    from paper_2412_18106_b200 import workloads as W
+    rng = np.random.default_rng(seed)
+    Hq, Hkv, B, D = 32, 8, 128, 128
+    max_kv = 12288
+    pages_per_req = max_kv // B + 1
+    num_pages = 6144  # 2 x 1.6 GB of K/V: far beyond L2
+    g = torch.Generator(device=dev).manual_seed(seed)
+    k_pool = torch.randn((num_pages, Hkv, B, D), device=dev, generator=g).to(torch.bfloat16)
+    v_pool = torch.randn((num_pages, Hkv, B, D), device=dev, generator=g).to(torch.bfloat16)
+    q = torch.randn((budget, Hq, D), device=dev, generator=g).to(torch.bfloat16)
+    o = torch.empty((budget, Hq, D), dtype=torch.bfloat16, device=dev)
+    lse = torch.empty((budget, Hq), dtype=torch.float32, device=dev)
+    cap = 256
+    ctx = xb.XYAttn(Hq, Hkv, B, device=dev.index, kernel=kernel, max_requests=cap, max_q_tokens=budget,
+                    max_pages_per_req=pages_per_req, max_tree_nodes=64)
+    sch = xs.XYSched(budget, reserved, cap)
+    bt_all = torch.from_numpy(rng.integers(0, num_pages, size=(sessions, pages_per_req)).astype(np.int32))
+    bt_dev = torch.zeros((cap, pages_per_req), dtype=torch.int32, device=dev)
+    kv_of = {}
+    for sid in range(sessions):
+        prompt = int(round(math.exp(rng.uniform(math.log(256), math.log(4096)))))
+        hit = int(prompt * rng.uniform(0.0, 0.9)) if rng.random() < 0.5 else 0
+        sch.add_prefill(sid, prompt, min(hit, prompt - 1))
+        kv_of[sid] = prompt
+    t_sched = t_plan = 0.0
+    flops = kvb = 0.0
+    tokens = 0
+    ctx.set_timing(True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    done = 0
+    e0.record()
+    while done < chunks and sch.pending() != (0, 0):
+        t0 = time.perf_counter()
+        chunk = sch.next_chunk()
+        t1 = time.perf_counter()
+        ql = [e["q_len"] for e in chunk]
+        kl = [e["kv_len"] for e in chunk]
+        mk = [1 if e["parents"] is not None else 0 for e in chunk]
+        par, off = [], []
+        for e in chunk:
+            off.append(len(par) if e["parents"] is not None else -1)
+            par += e["parents"] or []
+        t2 = time.perf_counter()
+        info = ctx.plan(ql, kl, mk, off, np.asarray(par, np.int32) if par else None)
+        t3 = time.perf_counter()
+        rows = torch.tensor([e["id"] for e in chunk], dtype=torch.long)
+        bt_dev[: len(chunk)].copy_(bt_all[rows], non_blocking=False)
+        T = int(sum(ql))
+        ctx.run(q[:T], k_pool, v_pool, bt_dev, SCALE, o[:T], lse[:T])
+        t_sched += t1 - t0
+        t_plan += t3 - t2
+        flops += float(info.useful_flops)
+        kvb += float(info.kv_bytes)
+        tokens += T
+        done += 1
+        # the serving loop: finished prompts and decoded / verified sessions come back
+        for e in chunk:
+            if not e["last"]:
+                continue
+            sid = e["id"]
+            if e["kind"] != xs.XY_SCHED_PREFILL:
+                kv_of[sid] = e["kv_len"] + (1 if e["kind"] == xs.XY_SCHED_DECODE else 3)
+            if kv_of[sid] + 64 >= max_kv:
+                continue
+            if sid % 5 == 0:
+                sch.add_verify(sid, kv_of[sid], W.random_tree(rng, int(rng.integers(4, 33)), 6))
+            else:
+                sch.add_decode(sid, kv_of[sid])
+    e1.record()
+    torch.cuda.synchronize()
+    wall_ms = e0.elapsed_time(e1)
+    attn_ms, merge_ms, runs = ctx.get_timing()
+    assert ctx.device_status() == 0
+    hits, misses = ctx.plan_cache()
+    ctx.close()
+    sch.close()
+    n = max(1, done)
+    return {"chunks": done, "budget_tokens": budget, "reserved_dv_tokens": reserved, "sessions": sessions,
+            "tokens": tokens, "sched_us_per_chunk": 1e6 * t_sched / n, "plan_us_per_chunk": 1e6 * t_plan / n,
+            "attn_ms_per_chunk": (attn_ms + merge_ms) / n, "wall_ms_per_chunk": wall_ms / n,
+            "tflops_attention": flops / ((attn_ms + merge_ms) * 1e-3) / 1e12,
+            "kv_gbs_attention": kvb / ((attn_ms + merge_ms) * 1e-3) / 1e9,
+            "task_table_cache": {"hits": hits, "misses": misses}}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -482,6 +578,11 @@ def main():
                 others[name] = measure_other(name, kernel, dev, peaks)
             except Exception as e:  # report, never hide the primary line
                 others[name] = {"error": repr(e)}
+        try:
+            torch.cuda.empty_cache()
+            others["serving_stream"] = measure_stream(kernel, dev, peaks)
+        except Exception as e:
+            others["serving_stream"] = {"error": repr(e)}
 
     line = {
         "metric": "hybrid_attention_useful_tflops", "value": value, "unit": "TFLOP/s",
