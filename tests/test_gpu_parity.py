@@ -226,3 +226,37 @@ def test_consecutive_steps_through_the_task_table_cache():
     hits, misses = ctx.plan_cache()
     assert hits >= 1 and misses >= 2 and hits + misses == 4
     ctx.close()
+
+
+@pytest.mark.parametrize("workers", [1, 2, 5])
+def test_many_task_kind_transitions_per_worker(workers):
+    """Few workers, many short tasks of alternating kinds: one-sub-tile dense tasks (<= 128 packed
+    rows), two-sub-tile dense tasks and streaming tasks follow each other on the same worker in
+    every order, which exercises the hand-over of the shared Q tiles and of tensor memory between
+    tasks.  Whole output against the oracle, and bit-identical when repeated."""
+    rng = np.random.default_rng(100 + workers)
+    reqs = []
+    for k in range(36):
+        kind = k % 4
+        if kind == 0:
+            reqs.append((int(rng.integers(17, 33)), int(rng.integers(0, 400)), 0, None))   # one sub-tile
+        elif kind == 1:
+            reqs.append((1, int(rng.integers(1, 700)), 0, None))                          # streaming
+        elif kind == 2:
+            reqs.append((int(rng.integers(40, 64)), int(rng.integers(0, 300)), 0, None))   # two sub-tiles
+        else:
+            n = int(rng.integers(5, 30))
+            reqs.append((n, int(rng.integers(10, 500)), 1, W.random_tree(rng, n, 5)))
+    b = W.custom("transitions", 8, 2, 32, reqs, seed=workers)
+    t = W.make_tensors(b)
+    ctx = H.make_ctx(b, num_workers=workers)
+    ctx.plan_batch(b)
+    O_ref, LSE_ref = oracle.attention(b, t, H.SCALE)
+    first = None
+    for _ in range(3):
+        O, LSE = H.run_gpu(b, t, ctx=ctx)
+        H.check_against_oracle(O, LSE, O_ref, LSE_ref, "transitions")
+        if first is None:
+            first = (O, LSE)
+        assert np.array_equal(O, first[0]) and np.array_equal(LSE, first[1])
+    ctx.close()
