@@ -1,0 +1,47 @@
+/* SmoothGEMM for sm_100a (Section 5): a fixed-tile tensor-core GEMM for the Linear operators
+ * (QKV, OProj, GateUp, Down) whose token dimension M takes any value.
+ *
+ *     C[M, N] = A[M, K] * W[N, K]^T      bf16 inputs, fp32 accumulation, bf16 output
+ *
+ * The kernel always computes whole 128 x tile_n tiles (Section 5.1: computation on fixed shapes).
+ * M is padded virtually: the tile loads read rows past M as zeros on chip (selective read; no
+ * padded copy of A exists in global memory) and the epilogue stores only rows below M (selective
+ * write).  N and K come from the model (Section 5.2) and need no padding beyond 8-element
+ * alignment; a last partial tile in N or K is handled the same way (zeros in, clipped store).
+ * Tiles are handed to the SMs with the M tiles of one N tile next to each other, so the SMs that
+ * run at the same time share the weight tile through L2 (Section 5.3's task order).
+ */
+#ifndef XY_GEMM_H_
+#define XY_GEMM_H_
+
+#include <stdint.h>
+
+#include "xy_attn.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Asynchronous on `stream` (a cudaStream_t, may be 0); allocates nothing; no host sync.
+ *   a  DEVICE bf16, row m at a + m*lda (elements), K contiguous; lda >= K
+ *   w  DEVICE bf16, row n at w + n*ldw, K contiguous (the layout of a Linear weight); ldw >= K
+ *   c  DEVICE bf16, row m at c + m*ldc, N contiguous; ldc >= N; written for m < M, n < N only
+ *   M >= 0 (0: nothing to do), N >= 8, K >= 8; N, K, lda, ldw, ldc multiples of 8; the three base
+ *   pointers 16-byte aligned
+ *   tile_n  columns per tile: 128, 256, or 0 to let the library choose (256 when the 128 x 256
+ *           tiles fill the SMs at least once, else 128)
+ * Returns XY_OK, XY_ERR_INVALID_ARG (null pointer, bad size or alignment), XY_ERR_UNSUPPORTED
+ * (tile_n not in {0, 128, 256}) or XY_ERR_CUDA.  Calls on one stream are ordered; the caller
+ * owns all buffers. */
+int xy_gemm_run(const void* a, int64_t lda, const void* w, int64_t ldw, void* c, int64_t ldc, int32_t M,
+                int32_t N, int32_t K, int32_t tile_n, void* stream);
+
+/* Status of the device-side waits of the GEMM kernels on the current device since the last call of
+ * this function: 0, or XY_ERR_DEVICE_TIMEOUT if a bounded wait inside a kernel gave up (the
+ * kernel then returns early and its output is invalid).  Synchronises the device. */
+int xy_gemm_device_status(int32_t* status /*HOST*/);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* XY_GEMM_H_ */

@@ -1,0 +1,281 @@
+// SmoothGEMM (Section 5): C[M,N] = A[M,K] W[N,K]^T on tcgen05, fixed 128 x kTileN tiles with
+// virtual padding of M (TMA zero-fills rows past M; the epilogue stores rows below M only).
+//
+// One persistent CTA per SM, 192 threads:
+//   warp 0, one lane   TMA producer: per 64-element K chunk one box of A (128 rows) and one of W
+//                      (kTileN rows) into the next free stage of a shared-memory ring
+//   warp 1, one lane   MMA issuer: four tcgen05.mma (K = 16 each) per chunk into one of two
+//                      accumulators in tensor memory; tcgen05.commit frees the stage and, after
+//                      the last chunk, hands the accumulator to the epilogue
+//   warps 2-5          epilogue: tensor memory -> bf16 -> global (thread = row), then return the
+//                      accumulator; runs while the issuer fills the other accumulator
+// Every wait is bounded; on expiry the kernel records XY_ERR_DEVICE_TIMEOUT and returns.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "ptx.cuh"
+#include "xy_gemm.h"
+
+namespace xy {
+namespace {
+
+using namespace ptx;
+
+constexpr int kTileM = 128;
+constexpr int kChunkK = 64;  // elements per K chunk = one 128-byte swizzle row
+constexpr int kGemmThreads = 192;
+constexpr int kABytes = kTileM * kChunkK * 2;  // 16 KiB
+
+__device__ int32_t g_gemm_status;
+
+template <int kTileN>
+struct GemmCfg {
+  static constexpr int kWBytes = kTileN * kChunkK * 2;
+  static constexpr int kStageBytes = kABytes + kWBytes;
+  static constexpr int kStages = kTileN == 256 ? 4 : 6;
+  static constexpr int kSmem = 1024 + kStages * kStageBytes + 256;
+  static constexpr uint32_t kTmemCols = 2 * kTileN;  // two accumulators
+};
+
+struct GemmParams {
+  uint16_t* c;
+  int64_t ldc;
+  int32_t M, N, K;
+  int32_t m_tiles, n_tiles;
+};
+
+struct __align__(8) GemmBarriers {
+  uint64_t full[6], empty[6];
+  uint64_t acc_full[2], acc_empty[2];
+  uint32_t tmem_base;
+};
+
+template <int kTileN>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+smooth_gemm_kernel(const GemmParams P, const __grid_constant__ CUtensorMap a_map,
+                   const __grid_constant__ CUtensorMap w_map) {
+  using Cfg = GemmCfg<kTileN>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  GemmBarriers* bars =
+      reinterpret_cast<GemmBarriers*>(smem_raw + (base - smem_u32(smem_raw)) + Cfg::kStages * Cfg::kStageBytes);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const volatile int32_t* status = &g_gemm_status;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < Cfg::kStages; ++s) {
+      mbar_init(smem_u32(&bars->full[s]), 1);
+      mbar_init(smem_u32(&bars->empty[s]), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&bars->acc_full[b]), 1);
+      mbar_init(smem_u32(&bars->acc_empty[b]), 4);
+    }
+    fence_mbar_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&bars->tmem_base), Cfg::kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = bars->tmem_base;
+  const int num_tiles = P.m_tiles * P.n_tiles;
+  const int k_chunks = (P.K + kChunkK - 1) / kChunkK;
+
+  if (warp == 0 && lane == 0) {
+    // ---------------------------------------------------------------- producer
+    prefetch_tensormap(&a_map);
+    prefetch_tensormap(&w_map);
+    uint32_t pos = 0;
+    bool dead = false;
+    for (int t = blockIdx.x; t < num_tiles && !dead; t += gridDim.x) {
+      const int m0 = (t % P.m_tiles) * kTileM, n0 = (t / P.m_tiles) * kTileN;
+      for (int kc = 0; kc < k_chunks; ++kc, ++pos) {
+        const uint32_t s = pos % Cfg::kStages, use = pos / Cfg::kStages;
+        if (use > 0 && !mbar_wait(smem_u32(&bars->empty[s]), (use - 1) & 1u, status)) {
+          atomicExch(&g_gemm_status, XY_ERR_DEVICE_TIMEOUT);
+          dead = true;
+          break;
+        }
+        const uint32_t full = smem_u32(&bars->full[s]);
+        mbar_arrive_expect_tx(full, Cfg::kStageBytes);
+        const uint32_t dst = base + s * Cfg::kStageBytes;
+        tma_load_2d(dst, &a_map, full, kc * kChunkK, m0);           // rows past M arrive as zeros
+        tma_load_2d(dst + kABytes, &w_map, full, kc * kChunkK, n0);  // rows past N likewise
+      }
+    }
+  } else if (warp == 1 && lane == 0) {
+    // ---------------------------------------------------------------- MMA issuer
+    // Shared-memory descriptors: K-major operands in the 128-byte swizzle, 8-row groups 1024 B
+    // apart; a K step of 16 elements advances the start address by 32 B.
+    constexpr uint64_t kDescHi = static_cast<uint64_t>((1024u >> 4) | (1u << 14) | (2u << 29)) << 32;
+    constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((static_cast<uint32_t>(kTileN) >> 3) << 17) |
+                                ((static_cast<uint32_t>(kTileM) >> 4) << 24);
+    uint32_t pos = 0, local = 0;
+    bool dead = false;
+    for (int t = blockIdx.x; t < num_tiles && !dead; t += gridDim.x, ++local) {
+      const uint32_t buf = local & 1u, use = local >> 1;
+      if (use > 0 && !mbar_wait(smem_u32(&bars->acc_empty[buf]), (use - 1) & 1u, status)) {
+        atomicExch(&g_gemm_status, XY_ERR_DEVICE_TIMEOUT);
+        break;
+      }
+      tc_fence_after();
+      const uint32_t d_tmem = tmem + buf * kTileN;
+      for (int kc = 0; kc < k_chunks; ++kc, ++pos) {
+        const uint32_t s = pos % Cfg::kStages;
+        if (!mbar_wait(smem_u32(&bars->full[s]), (pos / Cfg::kStages) & 1u, status)) {
+          atomicExch(&g_gemm_status, XY_ERR_DEVICE_TIMEOUT);
+          dead = true;
+          break;
+        }
+        tc_fence_after();
+        const uint32_t a_lo = (((base + s * Cfg::kStageBytes) >> 4) & 0x3FFFu) | (1u << 16);
+        const uint32_t w_lo = (((base + s * Cfg::kStageBytes + kABytes) >> 4) & 0x3FFFu) | (1u << 16);
+#pragma unroll
+        for (int k16 = 0; k16 < 4; ++k16)
+          umma_ss64(d_tmem, kDescHi | (a_lo + k16 * 2), kDescHi | (w_lo + k16 * 2), kIdesc, (kc | k16) ? 1u : 0u);
+        umma_commit(smem_u32(&bars->empty[s]));  // the stage is free once these MMAs have read it
+      }
+      if (!dead) umma_commit(smem_u32(&bars->acc_full[buf]));
+    }
+  } else if (warp >= 2) {
+    // ---------------------------------------------------------------- epilogue
+    const int q = warp & 3;  // tensor-memory lanes 32 q .. 32 q + 31 belong to this warp
+    const int row_in_tile = q * 32 + lane;
+    uint32_t local = 0;
+    for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++local) {
+      const uint32_t buf = local & 1u;
+      if (!mbar_wait(smem_u32(&bars->acc_full[buf]), (local >> 1) & 1u, status)) {
+        atomicExch(&g_gemm_status, XY_ERR_DEVICE_TIMEOUT);
+        break;
+      }
+      tc_fence_after();
+      const int m0 = (t % P.m_tiles) * kTileM, n0 = (t / P.m_tiles) * kTileN;
+      const int row = m0 + row_in_tile;
+      const uint32_t t_acc = tmem + (static_cast<uint32_t>(q * 32) << 16) + buf * kTileN;
+      uint16_t* crow = P.c + static_cast<int64_t>(row) * P.ldc + n0;
+#pragma unroll 2
+      for (int c0 = 0; c0 < kTileN; c0 += 32) {
+        uint32_t v[32];
+        tmem_ld_32x32b_x32(t_acc + c0, v);
+        tmem_wait_ld();
+        if (row < P.M) {  // selective write: virtual padding rows are never stored
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            if (n0 + c0 + g * 8 < P.N) {
+              uint4 o;
+              o.x = pack_bf16(__uint_as_float(v[g * 8 + 0]), __uint_as_float(v[g * 8 + 1]));
+              o.y = pack_bf16(__uint_as_float(v[g * 8 + 2]), __uint_as_float(v[g * 8 + 3]));
+              o.z = pack_bf16(__uint_as_float(v[g * 8 + 4]), __uint_as_float(v[g * 8 + 5]));
+              o.w = pack_bf16(__uint_as_float(v[g * 8 + 6]), __uint_as_float(v[g * 8 + 7]));
+              *reinterpret_cast<uint4*>(crow + c0 + g * 8) = o;
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bars->acc_empty[buf]));
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, Cfg::kTmemCols);
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn gemm_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn == nullptr) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// 2-D map over a row-major bf16 matrix [rows, K] with row stride ld: box = 64 elements x box_rows.
+bool encode_matrix_map(CUtensorMap* m, const void* ptr, int64_t rows, int64_t K, int64_t ld, int box_rows) {
+  EncodeTiledFn fn = gemm_encode_fn();
+  if (fn == nullptr) return false;
+  cuuint64_t dims[2] = {static_cast<cuuint64_t>(K), static_cast<cuuint64_t>(rows)};
+  cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld) * 2};
+  cuuint32_t box[2] = {static_cast<cuuint32_t>(kChunkK), static_cast<cuuint32_t>(box_rows)};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int kTileN>
+cudaError_t launch_gemm(const void* a, int64_t lda, const void* w, int64_t ldw, void* c, int64_t ldc, int M, int N,
+                        int K, int num_sms, cudaStream_t s) {
+  using Cfg = GemmCfg<kTileN>;
+  auto kernel = smooth_gemm_kernel<kTileN>;
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmem);
+  if (e != cudaSuccess) return e;
+  CUtensorMap a_map, w_map;
+  if (!encode_matrix_map(&a_map, a, M, K, lda, kTileM) || !encode_matrix_map(&w_map, w, N, K, ldw, kTileN))
+    return cudaErrorInvalidValue;
+  GemmParams P;
+  P.c = static_cast<uint16_t*>(c);
+  P.ldc = ldc;
+  P.M = M;
+  P.N = N;
+  P.K = K;
+  P.m_tiles = (M + kTileM - 1) / kTileM;
+  P.n_tiles = (N + kTileN - 1) / kTileN;
+  const int tiles = P.m_tiles * P.n_tiles;
+  kernel<<<tiles < num_sms ? tiles : num_sms, kGemmThreads, Cfg::kSmem, s>>>(P, a_map, w_map);
+  return cudaGetLastError();
+}
+
+}  // namespace
+}  // namespace xy
+
+extern "C" int xy_gemm_run(const void* a, int64_t lda, const void* w, int64_t ldw, void* c, int64_t ldc, int32_t M,
+                           int32_t N, int32_t K, int32_t tile_n, void* stream) {
+  if (M < 0 || N < 8 || K < 8 || (N % 8) || (K % 8) || (lda % 8) || (ldw % 8) || (ldc % 8) || lda < K || ldw < K ||
+      ldc < N)
+    return XY_ERR_INVALID_ARG;
+  if (tile_n != 0 && tile_n != 128 && tile_n != 256) return XY_ERR_UNSUPPORTED;
+  if (M == 0) return XY_OK;
+  if (!a || !w || !c || (reinterpret_cast<uintptr_t>(a) & 15) || (reinterpret_cast<uintptr_t>(w) & 15) ||
+      (reinterpret_cast<uintptr_t>(c) & 15))
+    return XY_ERR_INVALID_ARG;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+    return XY_ERR_CUDA;
+  if (tile_n == 0) {
+    const int64_t tiles256 = static_cast<int64_t>((M + 127) / 128) * ((N + 255) / 256);
+    tile_n = tiles256 >= sms ? 256 : 128;
+  }
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const cudaError_t e = tile_n == 256 ? xy::launch_gemm<256>(a, lda, w, ldw, c, ldc, M, N, K, sms, s)
+                                      : xy::launch_gemm<128>(a, lda, w, ldw, c, ldc, M, N, K, sms, s);
+  return e == cudaSuccess ? XY_OK : XY_ERR_CUDA;
+}
+
+extern "C" int xy_gemm_device_status(int32_t* status) {
+  if (status == nullptr) return XY_ERR_INVALID_ARG;
+  if (cudaDeviceSynchronize() != cudaSuccess) return XY_ERR_CUDA;
+  int32_t v = 0;
+  if (cudaMemcpyFromSymbol(&v, xy::g_gemm_status, sizeof v) != cudaSuccess) return XY_ERR_CUDA;
+  const int32_t zero = 0;
+  if (cudaMemcpyToSymbol(xy::g_gemm_status, &zero, sizeof zero) != cudaSuccess) return XY_ERR_CUDA;
+  *status = v;
+  return XY_OK;
+}

@@ -1,0 +1,51 @@
+"""Thin ctypes binding of SmoothGEMM (include/xy_gemm.h): argument marshalling only."""
+from __future__ import annotations
+
+import ctypes
+from typing import Optional
+
+import torch
+
+from . import binding as xb
+
+GEMM_EXPORTS = ("xy_gemm_run", "xy_gemm_device_status")
+
+_ready = False
+
+
+def _lib():
+    global _ready
+    L = xb.load()
+    if not _ready:
+        vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+        L.xy_gemm_run.argtypes = [vp, i64, vp, i64, vp, i64, i32, i32, i32, i32, vp]
+        L.xy_gemm_run.restype = ctypes.c_int
+        L.xy_gemm_device_status.argtypes = [ctypes.POINTER(i32)]
+        L.xy_gemm_device_status.restype = ctypes.c_int
+        _ready = True
+    return L
+
+
+def xy_gemm_run(a: torch.Tensor, w: torch.Tensor, c: torch.Tensor, tile_n: int = 0, stream=None) -> None:
+    """c[M, N] = a[M, K] w[N, K]^T (bf16 CUDA tensors, last dimension contiguous; rows may be strided)."""
+    for t in (a, w, c):
+        if t.dtype != torch.bfloat16 or not t.is_cuda or t.dim() != 2 or (t.numel() and t.stride(1) != 1):
+            raise ValueError("xy_gemm_run takes 2-D bf16 CUDA tensors with a contiguous last dimension")
+    M, K = a.shape
+    N = w.shape[0]
+    if w.shape[1] != K or tuple(c.shape) != (M, N):
+        raise ValueError("shape mismatch")
+    lda = a.stride(0) if M > 1 else max(K, a.stride(0))
+    rc = _lib().xy_gemm_run(a.data_ptr(), lda, w.data_ptr(), w.stride(0), c.data_ptr(),
+                            c.stride(0) if M > 1 else max(N, c.stride(0)), M, N, K, int(tile_n),
+                            xb._stream_ptr(stream))
+    if rc != 0:
+        raise xb.XYAttnError(rc, "xy_gemm_run failed")
+
+
+def xy_gemm_device_status() -> int:
+    s = ctypes.c_int32(0)
+    rc = _lib().xy_gemm_device_status(ctypes.byref(s))
+    if rc != 0:
+        raise xb.XYAttnError(rc, "xy_gemm_device_status failed")
+    return int(s.value)
