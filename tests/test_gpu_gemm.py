@@ -1,0 +1,83 @@
+"""SmoothGEMM on the GPU through the C-ABI against the fp64 oracle, element by element: the
+virtual padding of M (Section 5.1) and the partial tiles in N and K must not change any result."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import gemm_oracle as G
+from paper_2412_18106_b200 import binding as xb
+from paper_2412_18106_b200 import gemm as xg
+
+pytestmark = pytest.mark.gpu
+
+
+def check(M, N, K, tile_n, seed=0, lda=None, ldc=None):
+    """Tolerance: the output is rounded once to bf16 (relative 2^-9 of the result, bounded here by
+    2^-8 |ref|); the fp32 accumulation of K products of bf16 values adds at most about
+    K 2^-24 sum|a||w|, far below that for K <= 8192; results near zero after cancellation get an
+    absolute floor of 2^-8 sqrt(K) 2^-6 (a few fp32 roundings of partial sums of size sqrt(K))."""
+    g = torch.Generator().manual_seed(seed)
+    lda = K if lda is None else lda
+    ldc = N if ldc is None else ldc
+    a_buf = torch.randn((max(M, 1), lda), generator=g).to(torch.bfloat16)
+    w = torch.randn((N, K), generator=g).to(torch.bfloat16)
+    a = a_buf[:M, :K]
+    c_buf = torch.full((max(M, 1) + 1, ldc), float("nan"), dtype=torch.bfloat16, device="cuda")
+    c = c_buf[:M, :N]
+    xg.xy_gemm_run(a_buf.cuda()[:M, :K], w.cuda(), c, tile_n=tile_n)
+    assert xg.xy_gemm_device_status() == 0
+    got = c.float().cpu().numpy().astype(np.float64)
+    ref = G.linear(a.contiguous(), w)
+    assert not np.isnan(got).any()
+    tol = 2.0 ** -8 * np.abs(ref) + 2.0 ** -14 * np.sqrt(K)
+    bad = np.abs(got - ref) > tol
+    assert not bad.any(), (M, N, K, tile_n, float(np.abs(got - ref).max()), int(bad.sum()))
+    # selective write: nothing outside [0, M) x [0, N) was touched
+    rest = c_buf.float().cpu().numpy()
+    assert np.isnan(rest[M:, :]).all() and np.isnan(rest[:M, N:]).all()
+
+
+@pytest.mark.parametrize("tile_n", [128, 256])
+@pytest.mark.parametrize("M", [1, 7, 16, 127, 128, 129, 300])
+def test_any_token_count_matches_oracle(M, tile_n):
+    check(M, 384, 320, tile_n, seed=M)  # N and K both end in partial tiles / chunks
+
+
+@pytest.mark.parametrize("tile_n", [0, 128, 256])
+def test_linear_shapes_several_tiles_per_sm(tile_n):
+    check(1000, 1536, 1024, tile_n, seed=3)
+
+
+def test_strided_rows_and_small_sizes():
+    check(33, 64, 64, 128, seed=5, lda=96, ldc=80)
+    check(5, 8, 8, 128, seed=6)
+    check(200, 520, 72, 256, seed=7, lda=80, ldc=528)
+
+
+def test_zero_rows_is_a_no_op():
+    w = torch.zeros((64, 64), dtype=torch.bfloat16, device="cuda")
+    a = torch.zeros((0, 64), dtype=torch.bfloat16, device="cuda")
+    c = torch.zeros((0, 64), dtype=torch.bfloat16, device="cuda")
+    xg.xy_gemm_run(a, w, c)
+    assert xg.xy_gemm_device_status() == 0
+
+
+def test_full_size_qkv_projection_sampled():
+    """The QKV projection of the benchmark model at a full chunk: sampled outputs against dot
+    products, and the whole output against the library GEMM within two bf16 roundings."""
+    M, N, K = 4096, 6144, 4096
+    g = torch.Generator(device="cuda").manual_seed(9)
+    a = torch.randn((M, K), device="cuda", generator=g).to(torch.bfloat16)
+    w = torch.randn((N, K), device="cuda", generator=g).to(torch.bfloat16)
+    c = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    xg.xy_gemm_run(a, w, c)
+    assert xg.xy_gemm_device_status() == 0
+    rng = np.random.default_rng(1)
+    rows = np.concatenate([rng.integers(0, M, size=60), [0, M - 1, 127, 128]])
+    cols = np.concatenate([rng.integers(0, N, size=60), [0, N - 1, 255, 256]])
+    ref = G.linear_rows(a.cpu(), w.cpu(), rows, cols)
+    got = c[torch.from_numpy(rows).cuda(), torch.from_numpy(cols).cuda()].float().cpu().numpy()
+    assert np.all(np.abs(got - ref) <= 2.0 ** -8 * np.abs(ref) + 2.0 ** -14 * np.sqrt(K))
+    lib = (a @ w.T).float()
+    d = (c.float() - lib).abs()
+    assert float((d - 2.0 ** -7 * lib.abs()).max()) <= 2.0 ** -13 * np.sqrt(K)
