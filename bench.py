@@ -334,6 +334,45 @@ def measure_stream(kernel, dev, peaks, chunks=48, budget=4096, reserved=512, ses
             "task_table_cache": {"hits": hits, "misses": misses}}
 
 
+def measure_gemm(dev, peaks, steps=20):
+    """SmoothGEMM (Section 5) on the Linear shapes of the benchmark model (hidden 4096, 32 + 2 x 8
+    heads of 128, MLP 14336) for token counts from a decode batch to a full chunk.  Device-timed
+    back-to-back launches (the smallest cases are bound by launch latency, not by the kernel).
+    Fractions: flops against the measured burst bf16 peak (each kernel is timed alone), bytes
+    (A + W + C once) against the measured copy bandwidth; the larger of the two is the roofline.
+    The library GEMM (torch.matmul) is timed beside it for context."""
+    import torch
+
+    from paper_2412_18106_b200 import gemm as xg
+    out = {}
+    for name, N, K in (("qkv", 6144, 4096), ("oproj", 4096, 4096), ("gate_up", 28672, 4096), ("down", 4096, 14336)):
+        g = torch.Generator(device=dev).manual_seed(N + K)
+        w = torch.randn((N, K), device=dev, generator=g).to(torch.bfloat16)
+        for M in (16, 256, 4096):
+            a = torch.randn((M, K), device=dev, generator=g).to(torch.bfloat16)
+            c = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+
+            def timed(fn):
+                for _ in range(3):
+                    fn()
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for _ in range(steps):
+                    fn()
+                e1.record()
+                torch.cuda.synchronize()
+                return e0.elapsed_time(e1) / steps
+            ms = timed(lambda: xg.xy_gemm_run(a, w, c))
+            ms_lib = timed(lambda: torch.matmul(a, w.T, out=c))
+            flops, byts = 2.0 * M * N * K, 2.0 * (M * K + N * K + M * N)
+            t_roof = max(flops / (peaks["bf16_tflops"] * 1e12), byts / (peaks["hbm_gbs"] * 1e9))
+            out["%s_M%d" % (name, M)] = {"ms": ms, "tflops": flops / ms / 1e9, "gbs": byts / ms / 1e6,
+                                         "roofline_frac_measured": t_roof / (ms * 1e-3), "library_ms": ms_lib}
+    assert xg.xy_gemm_device_status() == 0
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -583,6 +622,11 @@ def main():
             others["serving_stream"] = measure_stream(kernel, dev, peaks)
         except Exception as e:
             others["serving_stream"] = {"error": repr(e)}
+        try:
+            torch.cuda.empty_cache()
+            others["smoothgemm"] = measure_gemm(dev, peaks)
+        except Exception as e:
+            others["smoothgemm"] = {"error": repr(e)}
 
     line = {
         "metric": "hybrid_attention_useful_tflops", "value": value, "unit": "TFLOP/s",

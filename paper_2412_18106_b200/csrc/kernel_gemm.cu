@@ -35,9 +35,9 @@ template <int kTileN>
 struct GemmCfg {
   static constexpr int kWBytes = kTileN * kChunkK * 2;
   static constexpr int kStageBytes = kABytes + kWBytes;
-  static constexpr int kStages = kTileN == 256 ? 4 : 6;
+  static constexpr int kStages = kTileN == 256 ? 4 : (kTileN == 128 ? 6 : 8);
   static constexpr int kSmem = 1024 + kStages * kStageBytes + 256;
-  static constexpr uint32_t kTmemCols = 2 * kTileN;  // two accumulators
+  static constexpr uint32_t kTmemCols = 2 * kTileN < 32 ? 32 : 2 * kTileN;  // two accumulators (power of two >= 32)
 };
 
 struct GemmParams {
@@ -48,7 +48,7 @@ struct GemmParams {
 };
 
 struct __align__(8) GemmBarriers {
-  uint64_t full[6], empty[6];
+  uint64_t full[8], empty[8];
   uint64_t acc_full[2], acc_empty[2];
   uint32_t tmem_base;
 };
@@ -224,8 +224,15 @@ cudaError_t launch_gemm(const void* a, int64_t lda, const void* w, int64_t ldw, 
                         int K, int num_sms, cudaStream_t s) {
   using Cfg = GemmCfg<kTileN>;
   auto kernel = smooth_gemm_kernel<kTileN>;
-  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmem);
+  static bool attr_set[64] = {false};  // per device: the opt-in to large dynamic shared memory
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmem);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64) attr_set[dev] = true;
+  }
   CUtensorMap a_map, w_map;
   if (!encode_matrix_map(&a_map, a, M, K, lda, kTileM) || !encode_matrix_map(&w_map, w, N, K, ldw, kTileN))
     return cudaErrorInvalidValue;
@@ -250,22 +257,35 @@ extern "C" int xy_gemm_run(const void* a, int64_t lda, const void* w, int64_t ld
   if (M < 0 || N < 8 || K < 8 || (N % 8) || (K % 8) || (lda % 8) || (ldw % 8) || (ldc % 8) || lda < K || ldw < K ||
       ldc < N)
     return XY_ERR_INVALID_ARG;
-  if (tile_n != 0 && tile_n != 128 && tile_n != 256) return XY_ERR_UNSUPPORTED;
+  if (tile_n != 0 && tile_n != 32 && tile_n != 64 && tile_n != 128 && tile_n != 256) return XY_ERR_UNSUPPORTED;
   if (M == 0) return XY_OK;
   if (!a || !w || !c || (reinterpret_cast<uintptr_t>(a) & 15) || (reinterpret_cast<uintptr_t>(w) & 15) ||
       (reinterpret_cast<uintptr_t>(c) & 15))
     return XY_ERR_INVALID_ARG;
-  int dev = 0, sms = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess ||
-      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
-    return XY_ERR_CUDA;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return XY_ERR_CUDA;
+  static int sm_count[64] = {0};
+  int sms = (dev >= 0 && dev < 64) ? sm_count[dev] : 0;
+  if (sms == 0) {
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+      return XY_ERR_CUDA;
+    if (dev >= 0 && dev < 64) sm_count[dev] = sms;
+  }
   if (tile_n == 0) {
+    // 128 x 256 tiles read the least of A and W per flop; they are used when they give every SM
+    // a tile.  Below that 128 x 128 (measured: narrower tiles are not faster for small M, where
+    // the time is launch and pipeline-fill latency).
     const int64_t tiles256 = static_cast<int64_t>((M + 127) / 128) * ((N + 255) / 256);
     tile_n = tiles256 >= sms ? 256 : 128;
   }
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  const cudaError_t e = tile_n == 256 ? xy::launch_gemm<256>(a, lda, w, ldw, c, ldc, M, N, K, sms, s)
-                                      : xy::launch_gemm<128>(a, lda, w, ldw, c, ldc, M, N, K, sms, s);
+  cudaError_t e;
+  switch (tile_n) {
+    case 256: e = xy::launch_gemm<256>(a, lda, w, ldw, c, ldc, M, N, K, sms, s); break;
+    case 128: e = xy::launch_gemm<128>(a, lda, w, ldw, c, ldc, M, N, K, sms, s); break;
+    case 64: e = xy::launch_gemm<64>(a, lda, w, ldw, c, ldc, M, N, K, sms, s); break;
+    default: e = xy::launch_gemm<32>(a, lda, w, ldw, c, ldc, M, N, K, sms, s); break;
+  }
   return e == cudaSuccess ? XY_OK : XY_ERR_CUDA;
 }
 

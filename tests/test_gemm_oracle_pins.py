@@ -69,7 +69,7 @@ def test_library_exports_every_gemm_symbol_and_rejects_bad_arguments():
     L = xg._lib()
     one = ctypes.c_void_p(16)
     # argument checks come before any CUDA call, so they can be exercised without a GPU
-    assert L.xy_gemm_run(one, 64, one, 64, one, 64, 4, 64, 64, 64, None) == xb.XY_ERR_UNSUPPORTED   # tile_n
+    assert L.xy_gemm_run(one, 64, one, 64, one, 64, 4, 64, 64, 48, None) == xb.XY_ERR_UNSUPPORTED   # tile_n
     assert L.xy_gemm_run(one, 64, one, 64, one, 64, -1, 64, 64, 0, None) == xb.XY_ERR_INVALID_ARG   # M < 0
     assert L.xy_gemm_run(one, 64, one, 64, one, 64, 4, 60, 64, 0, None) == xb.XY_ERR_INVALID_ARG    # N % 8
     assert L.xy_gemm_run(one, 60, one, 64, one, 64, 4, 64, 64, 0, None) == xb.XY_ERR_INVALID_ARG    # lda < K

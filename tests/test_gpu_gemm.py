@@ -37,13 +37,13 @@ def check(M, N, K, tile_n, seed=0, lda=None, ldc=None):
     assert np.isnan(rest[M:, :]).all() and np.isnan(rest[:M, N:]).all()
 
 
-@pytest.mark.parametrize("tile_n", [128, 256])
+@pytest.mark.parametrize("tile_n", [32, 64, 128, 256])
 @pytest.mark.parametrize("M", [1, 7, 16, 127, 128, 129, 300])
 def test_any_token_count_matches_oracle(M, tile_n):
     check(M, 384, 320, tile_n, seed=M)  # N and K both end in partial tiles / chunks
 
 
-@pytest.mark.parametrize("tile_n", [0, 128, 256])
+@pytest.mark.parametrize("tile_n", [0, 32, 64, 128, 256])
 def test_linear_shapes_several_tiles_per_sm(tile_n):
     check(1000, 1536, 1024, tile_n, seed=3)
 
