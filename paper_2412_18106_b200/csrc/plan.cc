@@ -329,6 +329,7 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
   // their total cost.  Dense tasks are bound by the SM (tensor pipe + softmax), streaming tasks
   // by HBM; a queue that hands out all of one kind first makes every SM stream at once (HBM
   // saturates) and then leaves HBM idle, while the mixed order keeps both busy throughout.
+  // Within the dense kind, sibling q tiles of one (request, kv head) are kept together (below).
   out->queue.resize(order.size());
   if (paper) {
     for (size_t pos = 0; pos < order.size(); ++pos) out->queue[pos] = where[order[pos]];
@@ -339,6 +340,32 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
       const int kd = pend[id].t.kind == 1 ? 1 : 0;
       by_kind[kd].push_back(id);
       total[kd] += pend[id].cost;
+    }
+    {
+      // Dense tasks of one (request, kv head) read the same K/V: all but the last tenth of the
+      // dense list is regrouped so that such siblings are handed out together (groups in the
+      // order of their most expensive task, tasks by descending cost inside a group) and share
+      // the K/V through L2 instead of re-reading it from HBM at different times.  The last tenth
+      // stays in plain descending order, which is what balances the end of the run.
+      std::vector<int>& d = by_kind[0];
+      const size_t head = d.size() - d.size() / 10;
+      std::vector<int64_t> group_of(head);
+      std::vector<int64_t> first_seen;  // group keys in order of first appearance
+      for (size_t i = 0; i < head; ++i) {
+        group_of[i] = static_cast<int64_t>(pend[d[i]].t.req) * cfg.num_kv_heads + pend[d[i]].t.kv_head;
+      }
+      std::vector<size_t> idx(head);
+      std::iota(idx.begin(), idx.end(), size_t{0});
+      std::vector<size_t> first_pos(static_cast<size_t>(num_reqs) * cfg.num_kv_heads, SIZE_MAX);
+      for (size_t i = 0; i < head; ++i)
+        if (first_pos[group_of[i]] == SIZE_MAX) first_pos[group_of[i]] = i;
+      std::stable_sort(idx.begin(), idx.end(),
+                       [&](size_t x, size_t y) { return first_pos[group_of[x]] < first_pos[group_of[y]]; });
+      std::vector<int> regrouped;
+      regrouped.reserve(d.size());
+      for (size_t i : idx) regrouped.push_back(d[i]);
+      for (size_t i = head; i < d.size(); ++i) regrouped.push_back(d[i]);
+      d.swap(regrouped);
     }
     size_t next[2] = {0, 0};
     for (size_t pos = 0; pos < order.size(); ++pos) {

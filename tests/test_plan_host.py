@@ -178,8 +178,8 @@ def test_balanced_plan_invariants_on_configs(name):
 
 
 def test_queue_mixes_kinds_and_puts_long_tasks_early():
-    """Balanced plans hand out dense and streaming tasks side by side (each kind in descending
-    order of key tiles), and no long task is left for the end of the queue."""
+    """Balanced plans hand out dense and streaming tasks side by side, dense siblings together,
+    and no long task is left for the end of the queue."""
     b = W.CONFIGS["splitfuse_mix"]()
     c = host_ctx(b.num_q_heads, b.num_kv_heads, b.page_size)
     info = c.plan_batch(b)
@@ -188,9 +188,21 @@ def test_queue_mixes_kinds_and_puts_long_tasks_early():
     ntiles = (tasks["kt_hi"] - tasks["kt_lo"])[queue]
     first = kinds[: info.num_workers]
     assert 0 < int(first.sum()) < info.num_workers  # both kinds among the first tasks handed out
-    for kd in (0, 1):
-        seq = ntiles[kinds == kd]
-        assert np.all(np.diff(seq) <= 0)
+    assert np.all(np.diff(ntiles[kinds == 1]) <= 0)  # streaming tasks: longest first
+    # dense tasks: sibling q tiles of one (request, kv head) are handed out together (longest
+    # first inside a group) except for the last tenth, which is in plain descending order
+    dq = queue[kinds == 0]
+    head = len(dq) - len(dq) // 10
+    grp = tasks["req"][dq].astype(np.int64) * 64 + tasks["kv_head"][dq]
+    dt = (tasks["kt_hi"] - tasks["kt_lo"])[dq]
+    seen = set()
+    for i in range(head):
+        if i and grp[i] == grp[i - 1]:
+            assert dt[i] <= dt[i - 1]
+        else:
+            assert int(grp[i]) not in seen  # a group appears as one run
+            seen.add(int(grp[i]))
+    assert np.all(np.diff(dt[head:]) <= 0)
     # the last tenth of the queue holds only tasks shorter than the median task
     tail = ntiles[-len(queue) // 10:]
     assert tail.max() <= np.median(ntiles)
