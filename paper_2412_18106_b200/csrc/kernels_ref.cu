@@ -90,34 +90,61 @@ __global__ void __launch_bounds__(128) ref_attention_kernel(RunArgs a) {
 }
 
 // Cross-task form of the Update stage (Section 4.2.1): combine the partials of every tile
-// unit whose KV range was split.  kMergeSlices blocks per merge unit, one warp per packed row.
-constexpr int kMergeSlices = 8;
+// unit whose KV range was split.  One warp per packed row (a unit has at most 256): lane c holds
+// LSE_c of split c, the maximum and the sum go through warp shuffles, and the weights
+// exp(LSE_c - LSE) are broadcast while the lanes accumulate four output columns each.
+constexpr int kMergeBlocksPerUnit = 64;  // x 4 warps = 256 rows
 __global__ void __launch_bounds__(128) merge_units_kernel(MergeArgs a) {
   const xy_attn_merge_unit u = a.units[blockIdx.x];
-  const ReqInfo rq = a.reqs[u.req];
   const int G = a.num_q_heads / a.num_kv_heads;
   const int rows = u.ntok * G;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (int x = blockIdx.y * 4 + warp; x < rows; x += 4 * kMergeSlices) {
-    float mx = -INFINITY;
-    for (int c = 0; c < u.nsplit; ++c) mx = fmaxf(mx, a.lse_part[u.part0 + c * rows + x]);
-    float z = 0.f;
-    for (int c = 0; c < u.nsplit; ++c) {
-      const float lc = a.lse_part[u.part0 + c * rows + x];
-      if (lc != -INFINITY) z += __expf(lc - mx);
-    }
-    const float lse = mx + logf(z);
+  if (blockIdx.y * 4 >= rows) return;
+  const ReqInfo rq = a.reqs[u.req];
+  for (int x = blockIdx.y * 4 + warp; x < rows; x += 4 * kMergeBlocksPerUnit) {
+    float lse;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int c = 0; c < u.nsplit; ++c) {
-      const float lc = a.lse_part[u.part0 + c * rows + x];
-      if (lc == -INFINITY) continue;
-      const float w = __expf(lc - lse);
-      const float4 v = *reinterpret_cast<const float4*>(
-          a.o_part + static_cast<int64_t>(u.part0 + c * rows + x) * kHeadDim + lane * 4);
-      acc.x += w * v.x;
-      acc.y += w * v.y;
-      acc.z += w * v.z;
-      acc.w += w * v.w;
+    if (u.nsplit <= 32) {
+      const float lc = lane < u.nsplit ? a.lse_part[u.part0 + lane * rows + x] : -INFINITY;
+      float mx = lc;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      const float e = lc != -INFINITY ? __expf(lc - mx) : 0.f;
+      float z = e;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
+      lse = mx + logf(z);
+      const float w_mine = z > 0.f ? e / z : 0.f;
+      for (int c = 0; c < u.nsplit; ++c) {
+        const float w = __shfl_sync(0xffffffffu, w_mine, c);
+        if (w == 0.f) continue;  // empty split (LSE_c = -inf): its O_c is not read
+        const float4 v = *reinterpret_cast<const float4*>(
+            a.o_part + static_cast<int64_t>(u.part0 + c * rows + x) * kHeadDim + lane * 4);
+        acc.x += w * v.x;
+        acc.y += w * v.y;
+        acc.z += w * v.z;
+        acc.w += w * v.w;
+      }
+    } else {
+      float mx = -INFINITY;
+      for (int c = 0; c < u.nsplit; ++c) mx = fmaxf(mx, a.lse_part[u.part0 + c * rows + x]);
+      float z = 0.f;
+      for (int c = 0; c < u.nsplit; ++c) {
+        const float lc = a.lse_part[u.part0 + c * rows + x];
+        if (lc != -INFINITY) z += __expf(lc - mx);
+      }
+      lse = mx + logf(z);
+      for (int c = 0; c < u.nsplit; ++c) {
+        const float lc = a.lse_part[u.part0 + c * rows + x];
+        if (lc == -INFINITY) continue;
+        const float w = __expf(lc - lse);
+        const float4 v = *reinterpret_cast<const float4*>(
+            a.o_part + static_cast<int64_t>(u.part0 + c * rows + x) * kHeadDim + lane * 4);
+        acc.x += w * v.x;
+        acc.y += w * v.y;
+        acc.z += w * v.z;
+        acc.w += w * v.w;
+      }
     }
     const int i = u.tok0 + x / G;
     const int head = u.kv_head * G + x % G;
@@ -227,7 +254,7 @@ cudaError_t launch_reference(const RunArgs& a, int num_workers, cudaStream_t s) 
 
 cudaError_t launch_merge_units(const MergeArgs& a, int num_units, cudaStream_t s) {
   if (num_units == 0) return cudaSuccess;
-  merge_units_kernel<<<dim3(num_units, kMergeSlices), 128, 0, s>>>(a);
+  merge_units_kernel<<<dim3(num_units, kMergeBlocksPerUnit), 128, 0, s>>>(a);
   return cudaGetLastError();
 }
 
