@@ -57,10 +57,15 @@ enum {
 
 /* Task-Table construction (Section 3.3.1). */
 enum {
-  XY_PLAN_BALANCED = 0, /* cost = max(tensor time, HBM time) of the visible page run; long
-                           runs are cut into KV splits; sorted + symmetric round-robin */
+  XY_PLAN_BALANCED = 0, /* cost = a measured time per visited 128-key tile (by task kind) plus a
+                           per-task term; long runs are cut into KV splits; the Task-Table is
+                           sorted + dealt by symmetric round-robin as in the paper, and the
+                           MMA kernels take the same tasks from one queue as workers become
+                           free (dense and streaming tasks side by side, sibling q tiles of a
+                           request together, long tasks first) */
   XY_PLAN_PAPER = 1     /* the paper's table literally: one task per tile unit, no KV split,
-                           load = rows x visible keys, sorted + symmetric round-robin */
+                           load = rows x visible keys, sorted + symmetric round-robin, every
+                           worker runs its own list */
 };
 
 typedef struct {
