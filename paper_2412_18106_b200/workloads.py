@@ -129,9 +129,11 @@ def assemble(
 def random_tree(rng: np.random.Generator, n: int, max_depth: int = 8) -> np.ndarray:
     """Random parent array in topological order: parent[0] = -1 and
     parent[i] uniform in [0, i-1], redrawn until the node's depth (root = 1)
-    does not exceed `max_depth`."""
+    does not exceed `max_depth` (max_depth <= 1: every node is a root)."""
     parent = np.full(n, -1, dtype=np.int32)
     depth = np.ones(n, dtype=np.int32)
+    if max_depth <= 1:
+        return parent
     for i in range(1, n):
         while True:
             p = int(rng.integers(0, i))
