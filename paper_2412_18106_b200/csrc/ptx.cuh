@@ -1,4 +1,4 @@
-// Thin inline-PTX wrappers for sm_100a: mbarrier, TMA (cp.async.bulk.tensor, no multicast),
+// Thin inline-PTX wrappers for sm_100a: mbarrier, TMA (cp.async.bulk.tensor into the issuing CTA only),
 // ldmatrix / mma.sync, tcgen05 (TMEM alloc, MMA, commit, ld/st, fences).
 #pragma once
 
