@@ -1,25 +1,33 @@
 // Hybrid-batch attention meta-kernel (Meta-Attention, Sections 4.1-4.2), sm_100a.
 //
-// One persistent CTA per worker walks its Task-Table list (Section 3.3.1).  Warp roles:
-//   warps 0..7  consumers: load the packed Q tile, compute QK -> softmax -> PV, write O / LSE
-//   warp  8     producer: looks page ids up in the block table and stages 128-key K and V
-//               tiles (one TMA box per page and 64-element half) into a ring of shared-memory
-//               stages; it runs ahead across task boundaries
+// One persistent CTA per worker (SM) of 384 threads runs meta-tasks until none are left: its own
+// Task-Table list (Section 3.3.1) or, for balanced plans, the head of one global queue.  Roles:
+//   warps 0..7  consumers: softmax (and, on the warp-level paths, the MMAs), O / LSE output
+//   warp  8     producer (one lane): takes the next task, looks page ids up in the block table and
+//               stages 128-key K and V tiles (one TMA box per page and 64-element half) into a
+//               ring of four shared-memory stages; it runs ahead across task boundaries
+//   warps 9-10  tcgen05 issuers (one lane each), one per 128-row sub-tile of a dense task
 // Shared-memory tiles use the 128-byte TMA swizzle: element (row, d) of a tile lives at
 //   (d / 64) * 16 KiB + row * 128 B + (((d % 64) / 8) ^ (row % 8)) * 16 B + (d % 8) * 2 B,
 // which both ldmatrix and the tcgen05 shared-memory descriptors read without bank conflicts.
 //
 // Two task kinds share the ring:
-//   dense     (rows > 16): each consumer warp owns 16 packed rows against all 128 keys of a tile
+//   dense     (rows > 16: prefill, verify): two 128-row sub-tiles of packed Q rows; S = Q K^T
+//             and O += P V run on tcgen05 with S, P and O in tensor memory, and each consumer
+//             warpgroup does the online softmax of one sub-tile (thread = row).  In the variant
+//             without tensor memory (kUmma = false) a dense task is one 128-row tile on
+//             mma.sync, each consumer warp owning 16 rows.
 //   streaming (rows <= 16: decode, tiny verify): each consumer warp owns 16 keys of every tile
-//             against all rows; the warps' partial (m, l, O) are merged in shared memory at
-//             the end of the task.  HBM-bound: the tensor work is a 16-row warp-level MMA.
-// Online softmax runs in the log2 domain in fp32 registers with quad shuffles; P is rounded
-// to bf16 before P.V; masked scores are selected to -inf, never added.
+//             against all rows on mma.sync; the warps' partial (m, l, O) are merged in shared
+//             memory at the end of the task.  HBM-bound.
+// Online softmax runs in the log2 domain in fp32; P is rounded to bf16 before P V; masked scores
+// are selected to -inf, never added.  Every wait is bounded and reports a timeout in the status
+// word instead of spinning forever.
 #include <cuda.h>
 #include <cuda_bf16.h>
-#include <type_traits>
 #include <cuda_runtime.h>
+
+#include <type_traits>
 
 #include "ptx.cuh"
 #include "xy_kernels.h"

@@ -13,7 +13,7 @@ constexpr int kHeadDim = 128;
 constexpr int kKeyTile = 128;      // keys per KV tile (one MMA N extent)
 constexpr int kStreamRowsMax = 16;
 constexpr int kTraceRoles = 4;      // sub-tile A, sub-tile B, MMA issuer, producer (worker 0 only)
-constexpr int kTraceLen = 2048; // packed rows a streaming task may hold
+constexpr int kTraceLen = 2048;    // records per role and run
 
 // Per-request facts the kernels need (device-visible, 32 bytes).
 struct ReqInfo {
