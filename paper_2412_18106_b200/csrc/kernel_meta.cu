@@ -1202,7 +1202,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
         named_bar_sync(1, kConsumerThreads);
       }
 
-      if (!stream) {
+      if (!kUmma && !stream) {  // (with kUmma every dense task took the tcgen05 path above)
         // ---------------- dense: this warp owns rows x0 .. x0+15 -------------------------
         const int x0 = warp * 16;
         const bool active = x0 < tv.rows;
