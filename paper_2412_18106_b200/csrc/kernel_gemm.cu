@@ -190,6 +190,184 @@ smooth_gemm_kernel(const GemmParams P, const __grid_constant__ CUtensorMap a_map
   }
 }
 
+
+// ------------------------------------------------------------------------------------------
+// Split-K variant for small token counts (M <= 128, few N tiles).  A whole-K tile is one serial
+// chain of K/64 chunks on one SM, and with fewer tiles than SMs most of the chip idles while the
+// weights stream through a few SMs.  Here a cluster of `splits` CTAs shares one 128 x 128 tile:
+// CTA r computes the partial product over its slice of K, writes the valid rows of its fp32
+// accumulator into its own shared memory, and after a cluster barrier every CTA adds the slices
+// of the rows it owns (row mod splits = rank) through distributed shared memory and stores those
+// bf16 rows.  One tile per CTA.
+struct SplitKParams {
+  uint16_t* c;
+  int64_t ldc;
+  int32_t M, N, K;
+  int32_t splits, chunks_per_split;
+};
+
+__global__ void __launch_bounds__(kGemmThreads, 1)
+smooth_gemm_splitk_kernel(const SplitKParams P, const __grid_constant__ CUtensorMap a_map,
+                          const __grid_constant__ CUtensorMap w_map) {
+  constexpr int kTileN = 128;
+  using Cfg = GemmCfg<kTileN>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
+  GemmBarriers* bars = reinterpret_cast<GemmBarriers*>(gen_base + Cfg::kStages * Cfg::kStageBytes);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const volatile int32_t* status = &g_gemm_status;
+  const uint32_t rank = cluster_ctarank();
+  const int n0 = static_cast<int>(blockIdx.x / P.splits) * kTileN;
+  const int k_chunks = (P.K + kChunkK - 1) / kChunkK;
+  const int kc_lo = static_cast<int>(rank) * P.chunks_per_split;
+  const int kc_hi = min(k_chunks, kc_lo + P.chunks_per_split);
+  const int my_chunks = max(0, kc_hi - kc_lo);
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < Cfg::kStages; ++s) {
+      mbar_init(smem_u32(&bars->full[s]), 1);
+      mbar_init(smem_u32(&bars->empty[s]), 1);
+    }
+    mbar_init(smem_u32(&bars->acc_full[0]), 1);
+    fence_mbar_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&bars->tmem_base), 128);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = bars->tmem_base;
+
+  if (warp == 0 && lane == 0) {
+    prefetch_tensormap(&a_map);
+    prefetch_tensormap(&w_map);
+    for (int i = 0; i < my_chunks; ++i) {
+      const uint32_t s = i % Cfg::kStages, use = i / Cfg::kStages;
+      if (use > 0 && !mbar_wait(smem_u32(&bars->empty[s]), (use - 1) & 1u, status)) {
+        atomicExch(&g_gemm_status, XY_ERR_DEVICE_TIMEOUT);
+        break;
+      }
+      const uint32_t full = smem_u32(&bars->full[s]);
+      mbar_arrive_expect_tx(full, Cfg::kStageBytes);
+      const uint32_t dst = base + s * Cfg::kStageBytes;
+      tma_load_2d(dst, &a_map, full, (kc_lo + i) * kChunkK, 0);
+      tma_load_2d(dst + kABytes, &w_map, full, (kc_lo + i) * kChunkK, n0);
+    }
+  } else if (warp == 1 && lane == 0) {
+    constexpr uint64_t kDescHi = static_cast<uint64_t>((1024u >> 4) | (1u << 14) | (2u << 29)) << 32;
+    constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((static_cast<uint32_t>(kTileN) >> 3) << 17) |
+                                ((static_cast<uint32_t>(kTileM) >> 4) << 24);
+    bool dead = false;
+    for (int i = 0; i < my_chunks; ++i) {
+      const uint32_t s = i % Cfg::kStages;
+      if (!mbar_wait(smem_u32(&bars->full[s]), (i / Cfg::kStages) & 1u, status)) {
+        atomicExch(&g_gemm_status, XY_ERR_DEVICE_TIMEOUT);
+        dead = true;
+        break;
+      }
+      tc_fence_after();
+      const uint32_t a_lo = (((base + s * Cfg::kStageBytes) >> 4) & 0x3FFFu) | (1u << 16);
+      const uint32_t w_lo = (((base + s * Cfg::kStageBytes + kABytes) >> 4) & 0x3FFFu) | (1u << 16);
+#pragma unroll
+      for (int k16 = 0; k16 < 4; ++k16)
+        umma_ss64(tmem, kDescHi | (a_lo + k16 * 2), kDescHi | (w_lo + k16 * 2), kIdesc, (i | k16) ? 1u : 0u);
+      umma_commit(smem_u32(&bars->empty[s]));
+    }
+    if (!dead && my_chunks > 0) umma_commit(smem_u32(&bars->acc_full[0]));
+  }
+  // ---- every CTA: valid rows of the partial accumulator -> own shared memory (fp32, row r at
+  // r * 512 B, 16-byte chunks XOR-swizzled by row so that a warp's 32 rows do not collide).
+  // The ring is free by then: acc_full completes only after every MMA has read its stage.
+  bool ok = true;
+  if (warp >= 2) {
+    const int q = warp & 3;
+    const int row = q * 32 + lane;
+    if (my_chunks > 0) {
+      if (!mbar_wait(smem_u32(&bars->acc_full[0]), 0u, status)) {
+        atomicExch(&g_gemm_status, XY_ERR_DEVICE_TIMEOUT);
+        ok = false;
+      }
+      tc_fence_after();
+    }
+    if (ok && q * 32 < P.M) {  // warps whose 32 rows are all padding skip the copy
+      const uint32_t t_acc = tmem + (static_cast<uint32_t>(q * 32) << 16);
+#pragma unroll 1
+      for (int c0 = 0; c0 < kTileN; c0 += 32) {
+        uint32_t v[32];
+        if (my_chunks > 0) {
+          tmem_ld_32x32b_x32(t_acc + c0, v);
+          tmem_wait_ld();
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] = 0u;
+        }
+        if (row < P.M) {
+#pragma unroll
+          for (int g = 0; g < 8; ++g) {
+            const int chunk = (c0 >> 2) + g;
+            *reinterpret_cast<uint4*>(gen_base + row * 512 + ((chunk ^ (row & 31)) << 4)) =
+                make_uint4(v[g * 4 + 0], v[g * 4 + 1], v[g * 4 + 2], v[g * 4 + 3]);
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncwarp();
+  cluster_sync_all();
+  if (warp >= 2) {
+    // Reduce-scatter: CTA r owns the rows congruent to r modulo `splits`; its 128 epilogue threads
+    // add that row's slices of all CTAs (thread t: 16-byte chunk t & 31 of every fourth owned
+    // row) through distributed shared memory and store the bf16 row.  Two rows are in flight per
+    // thread so that the remote loads overlap.
+    const int t = threadIdx.x - 64;
+    const int chunk = t & 31;
+    const int col = n0 + chunk * 4;
+    const int step = 4 * P.splits;
+    auto reduce_row = [&](int row, float4& acc) {
+      const uint32_t off = static_cast<uint32_t>(row * 512 + ((chunk ^ (row & 31)) << 4));
+      acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int r = 0; r < P.splits; ++r) {
+        const float4 v = ld_cluster_f4(cluster_map(base + off, static_cast<uint32_t>(r)));
+        acc.x += v.x;
+        acc.y += v.y;
+        acc.z += v.z;
+        acc.w += v.w;
+      }
+    };
+    auto store_row = [&](int row, const float4& acc) {
+      if (col < P.N) {  // N is a multiple of 8, chunks of 4 columns are all in or all out
+        uint2 o;
+        o.x = pack_bf16(acc.x, acc.y);
+        o.y = pack_bf16(acc.z, acc.w);
+        *reinterpret_cast<uint2*>(P.c + static_cast<int64_t>(row) * P.ldc + col) = o;
+      }
+    };
+    const int m_end = min(P.M, kTileM);
+    int row = static_cast<int>(rank) + P.splits * (t >> 5);
+    for (; row + step < m_end; row += 2 * step) {
+      float4 a0, a1;
+      reduce_row(row, a0);
+      reduce_row(row + step, a1);
+      store_row(row, a0);
+      store_row(row + step, a1);
+    }
+    if (row < m_end) {
+      float4 a0;
+      reduce_row(row, a0);
+      store_row(row, a0);
+    }
+  }
+  __syncwarp();
+  cluster_sync_all();  // every CTA's shared memory stays alive until all of them have read it
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 128);
+  }
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -249,6 +427,47 @@ cudaError_t launch_gemm(const void* a, int64_t lda, const void* w, int64_t ldw, 
   return cudaGetLastError();
 }
 
+
+cudaError_t launch_gemm_splitk(const void* a, int64_t lda, const void* w, int64_t ldw, void* c, int64_t ldc, int M,
+                               int N, int K, int splits, cudaStream_t s) {
+  using Cfg = GemmCfg<128>;
+  static bool attr_set[64] = {false};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+    e = cudaFuncSetAttribute(smooth_gemm_splitk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmem);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64) attr_set[dev] = true;
+  }
+  CUtensorMap a_map, w_map;
+  if (!encode_matrix_map(&a_map, a, M, K, lda, kTileM) || !encode_matrix_map(&w_map, w, N, K, ldw, 128))
+    return cudaErrorInvalidValue;
+  SplitKParams P;
+  P.c = static_cast<uint16_t*>(c);
+  P.ldc = ldc;
+  P.M = M;
+  P.N = N;
+  P.K = K;
+  P.splits = splits;
+  const int k_chunks = (K + kChunkK - 1) / kChunkK;
+  P.chunks_per_split = (k_chunks + splits - 1) / splits;
+  const int n_tiles = (N + 127) / 128;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(n_tiles * splits), 1, 1);
+  cfg.blockDim = dim3(kGemmThreads, 1, 1);
+  cfg.dynamicSmemBytes = Cfg::kSmem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = static_cast<unsigned>(splits);
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, smooth_gemm_splitk_kernel, P, a_map, w_map);
+}
+
 }  // namespace
 }  // namespace xy
 
@@ -270,6 +489,20 @@ extern "C" int xy_gemm_run(const void* a, int64_t lda, const void* w, int64_t ld
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
       return XY_ERR_CUDA;
     if (dev >= 0 && dev < 64) sm_count[dev] = sms;
+  }
+  if (tile_n == 0 && M <= 128) {
+    // Few tiles and one long serial chain over K per tile: split K over a cluster when that
+    // puts at least four times as many SMs to work (Down / OProj projections of a decode batch;
+    // measured: with three slices the reduction costs what the shorter chain saves).
+    const int n_tiles = (N + 127) / 128, k_chunks = (K + 63) / 64;
+    int splits = sms / n_tiles;
+    if (splits > 8) splits = 8;
+    if (splits > k_chunks / 8) splits = k_chunks / 8;
+    if (splits >= 4) {
+      const cudaError_t e =
+          xy::launch_gemm_splitk(a, lda, w, ldw, c, ldc, M, N, K, splits, static_cast<cudaStream_t>(stream));
+      return e == cudaSuccess ? XY_OK : XY_ERR_CUDA;
+    }
   }
   if (tile_n == 0) {
     // 128 x 256 tiles read the least of A and W per flop; they are used when they give every SM
