@@ -29,8 +29,8 @@ extern "C" {
  *   M >= 0 (0: nothing to do), N >= 8, K >= 8; N, K, lda, ldw, ldc multiples of 8; the three base
  *   pointers 16-byte aligned
  *   tile_n  columns per tile: 32, 64, 128, 256, or 0 to let the library choose: 256 when the
- *           128 x 256 tiles give every SM a tile, else 128; and for M <= 128 with few N tiles a
- *           split of K over a thread-block cluster (4..8 CTAs per 128 x 128 tile, partial sums
+ *           128 x 256 tiles give every SM a tile, else 128; and for M <= 512 with few tiles a
+ *           split of K over a thread-block cluster (2..8 CTAs per 128 x 128 tile, partial sums
  *           added through distributed shared memory), which puts the idle SMs to work
  * Returns XY_OK, XY_ERR_INVALID_ARG (null pointer, bad size or alignment), XY_ERR_UNSUPPORTED
  * (tile_n not in {0, 32, 64, 128, 256}) or XY_ERR_CUDA.  Calls on one stream are ordered; the caller

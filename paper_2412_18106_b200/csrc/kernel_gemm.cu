@@ -192,7 +192,7 @@ smooth_gemm_kernel(const GemmParams P, const __grid_constant__ CUtensorMap a_map
 
 
 // ------------------------------------------------------------------------------------------
-// Split-K variant for small token counts (M <= 128, few N tiles).  A whole-K tile is one serial
+// Split-K variant for small token counts (few tiles).  A whole-K tile is one serial
 // chain of K/64 chunks on one SM, and with fewer tiles than SMs most of the chip idles while the
 // weights stream through a few SMs.  Here a cluster of `splits` CTAs shares one 128 x 128 tile:
 // CTA r computes the partial product over its slice of K, writes the valid rows of its fp32
@@ -203,7 +203,7 @@ struct SplitKParams {
   uint16_t* c;
   int64_t ldc;
   int32_t M, N, K;
-  int32_t splits, chunks_per_split;
+  int32_t splits, chunks_per_split, m_tiles;
 };
 
 __global__ void __launch_bounds__(kGemmThreads, 1)
@@ -218,7 +218,9 @@ smooth_gemm_splitk_kernel(const SplitKParams P, const __grid_constant__ CUtensor
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const volatile int32_t* status = &g_gemm_status;
   const uint32_t rank = cluster_ctarank();
-  const int n0 = static_cast<int>(blockIdx.x / P.splits) * kTileN;
+  const int tile = static_cast<int>(blockIdx.x / P.splits);
+  const int m0 = (tile % P.m_tiles) * kTileM, n0 = (tile / P.m_tiles) * kTileN;
+  const int m_rows = min(kTileM, P.M - m0);  // valid rows of this tile
   const int k_chunks = (P.K + kChunkK - 1) / kChunkK;
   const int kc_lo = static_cast<int>(rank) * P.chunks_per_split;
   const int kc_hi = min(k_chunks, kc_lo + P.chunks_per_split);
@@ -252,7 +254,7 @@ smooth_gemm_splitk_kernel(const SplitKParams P, const __grid_constant__ CUtensor
       const uint32_t full = smem_u32(&bars->full[s]);
       mbar_arrive_expect_tx(full, Cfg::kStageBytes);
       const uint32_t dst = base + s * Cfg::kStageBytes;
-      tma_load_2d(dst, &a_map, full, (kc_lo + i) * kChunkK, 0);
+      tma_load_2d(dst, &a_map, full, (kc_lo + i) * kChunkK, m0);
       tma_load_2d(dst + kABytes, &w_map, full, (kc_lo + i) * kChunkK, n0);
     }
   } else if (warp == 1 && lane == 0) {
@@ -291,7 +293,7 @@ smooth_gemm_splitk_kernel(const SplitKParams P, const __grid_constant__ CUtensor
       }
       tc_fence_after();
     }
-    if (ok && q * 32 < P.M) {  // warps whose 32 rows are all padding skip the copy
+    if (ok && q * 32 < m_rows) {  // warps whose 32 rows are all padding skip the copy
       const uint32_t t_acc = tmem + (static_cast<uint32_t>(q * 32) << 16);
 #pragma unroll 1
       for (int c0 = 0; c0 < kTileN; c0 += 32) {
@@ -303,7 +305,7 @@ smooth_gemm_splitk_kernel(const SplitKParams P, const __grid_constant__ CUtensor
 #pragma unroll
           for (int j = 0; j < 32; ++j) v[j] = 0u;
         }
-        if (row < P.M) {
+        if (row < m_rows) {
 #pragma unroll
           for (int g = 0; g < 8; ++g) {
             const int chunk = (c0 >> 2) + g;
@@ -342,10 +344,10 @@ smooth_gemm_splitk_kernel(const SplitKParams P, const __grid_constant__ CUtensor
         uint2 o;
         o.x = pack_bf16(acc.x, acc.y);
         o.y = pack_bf16(acc.z, acc.w);
-        *reinterpret_cast<uint2*>(P.c + static_cast<int64_t>(row) * P.ldc + col) = o;
+        *reinterpret_cast<uint2*>(P.c + static_cast<int64_t>(m0 + row) * P.ldc + col) = o;
       }
     };
-    const int m_end = min(P.M, kTileM);
+    const int m_end = m_rows;
     int row = static_cast<int>(rank) + P.splits * (t >> 5);
     for (; row + step < m_end; row += 2 * step) {
       float4 a0, a1;
@@ -453,8 +455,9 @@ cudaError_t launch_gemm_splitk(const void* a, int64_t lda, const void* w, int64_
   const int k_chunks = (K + kChunkK - 1) / kChunkK;
   P.chunks_per_split = (k_chunks + splits - 1) / splits;
   const int n_tiles = (N + 127) / 128;
+  P.m_tiles = (M + kTileM - 1) / kTileM;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(static_cast<unsigned>(n_tiles * splits), 1, 1);
+  cfg.gridDim = dim3(static_cast<unsigned>(P.m_tiles * n_tiles * splits), 1, 1);
   cfg.blockDim = dim3(kGemmThreads, 1, 1);
   cfg.dynamicSmemBytes = Cfg::kSmem;
   cfg.stream = s;
@@ -490,15 +493,17 @@ extern "C" int xy_gemm_run(const void* a, int64_t lda, const void* w, int64_t ld
       return XY_ERR_CUDA;
     if (dev >= 0 && dev < 64) sm_count[dev] = sms;
   }
-  if (tile_n == 0 && M <= 128) {
-    // Few tiles and one long serial chain over K per tile: split K over a cluster when that
-    // puts at least four times as many SMs to work (Down / OProj projections of a decode batch;
-    // measured: with three slices the reduction costs what the shorter chain saves).
-    const int n_tiles = (N + 127) / 128, k_chunks = (K + 63) / 64;
-    int splits = sms / n_tiles;
+  if (tile_n == 0 && M <= 512) {
+    // Few tiles and one long serial chain over K per tile: split K over a cluster when that puts
+    // several times as many SMs to work (Down / OProj projections of a decode batch or a short
+    // chunk).  Measured: four or more slices pay off from 16 chunks per slice on; two or three
+    // only when the chain is long (32 chunks per slice), else the reduction costs what the
+    // shorter chain saves.
+    const int tiles = ((M + 127) / 128) * ((N + 127) / 128), k_chunks = (K + 63) / 64;
+    int splits = sms / tiles;
     if (splits > 8) splits = 8;
-    if (splits > k_chunks / 8) splits = k_chunks / 8;
-    if (splits >= 4) {
+    while (splits >= 2 && k_chunks / splits < (splits >= 4 ? 16 : 32)) --splits;
+    if (splits >= 2) {
       const cudaError_t e =
           xy::launch_gemm_splitk(a, lda, w, ldw, c, ldc, M, N, K, splits, static_cast<cudaStream_t>(stream));
       return e == cudaSuccess ? XY_OK : XY_ERR_CUDA;
