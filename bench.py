@@ -373,6 +373,53 @@ def measure_gemm(dev, peaks, steps=20):
     return out
 
 
+def measure_shared_prefix(kernel, dev, peaks, steps=20):
+    """Shared-prefix ("cascade") decode: 4 groups of 32 decode requests, each group sharing an
+    8192-token cached prefix (same pages), 0..1024 own tokens per request, 32/8 heads.  Times the
+    plain plan (every request reads its whole history) and the grouped plan (the shared keys are
+    read once per group by dense tiles).  The roofline fraction of the grouped plan counts the
+    bytes that must be read at least once: the shared prefixes once per group plus every
+    member's own keys."""
+    import torch
+
+    from paper_2412_18106_b200 import binding as xb
+    from paper_2412_18106_b200 import workloads as W
+    batch, groups = W.shared_prefix_decode(seed=0)
+    tensors = W.make_tensors(batch)
+    q, k_pool, v_pool = tensors.q.to(dev), tensors.k_pool.to(dev), tensors.v_pool.to(dev)
+    bt = torch.from_numpy(np.where(batch.block_table < 0, 0, batch.block_table).astype(np.int32)).to(dev)
+    o = torch.empty((batch.total_q, batch.num_q_heads, batch.head_dim), dtype=torch.bfloat16, device=dev)
+    lse = torch.empty((batch.total_q, batch.num_q_heads), dtype=torch.float32, device=dev)
+    per_token = 2 * batch.num_kv_heads * batch.head_dim * 2
+    unique = sum(g[2] for g in groups) * per_token
+    in_group = np.zeros(batch.num_requests, bool)
+    for first, n, prefix in groups:
+        in_group[first: first + n] = True
+        unique += int((batch.kv_len[first: first + n] + 1 - prefix).sum()) * per_token
+    unique += int((batch.kv_len[~in_group] + 1).sum()) * per_token
+    out = {"requests": batch.num_requests, "groups": len(groups), "prefix_tokens": groups[0][2],
+           "unique_kv_bytes": unique}
+    for name, gs in (("plain", None), ("grouped", groups)):
+        ctx = xb.XYAttn(batch.num_q_heads, batch.num_kv_heads, batch.page_size, device=dev.index, kernel=kernel,
+                        max_requests=512, max_q_tokens=1 << 15, max_pages_per_req=max(1024, batch.block_table.shape[1]))
+        info = ctx.plan_batch(batch, groups=gs)
+        for _ in range(3):
+            ctx.run(q, k_pool, v_pool, bt, SCALE, o, lse)
+        torch.cuda.synchronize()
+        ctx.set_timing(True)
+        for _ in range(steps):
+            ctx.run(q, k_pool, v_pool, bt, SCALE, o, lse)
+        attn_ms, merge_ms, runs = ctx.get_timing()
+        assert ctx.device_status() == 0
+        ctx.close()
+        k_ms, m_ms = attn_ms / runs, merge_ms / runs
+        out[name] = {"kernel_ms": k_ms, "merge_ms": m_ms, "tasks": info.num_tasks, "merge_units": info.num_merge_units,
+                     "kv_bytes_read_per_request": int(info.kv_bytes)}
+    out["speedup"] = (out["plain"]["kernel_ms"] + out["plain"]["merge_ms"]) / (out["grouped"]["kernel_ms"] + out["grouped"]["merge_ms"])
+    out["grouped"]["roofline_frac_measured"] = unique / (peaks["hbm_gbs"] * 1e9) / (out["grouped"]["kernel_ms"] * 1e-3)
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -622,6 +669,11 @@ def main():
             others["serving_stream"] = measure_stream(kernel, dev, peaks)
         except Exception as e:
             others["serving_stream"] = {"error": repr(e)}
+        try:
+            torch.cuda.empty_cache()
+            others["decode_shared_prefix"] = measure_shared_prefix(kernel, dev, peaks)
+        except Exception as e:
+            others["decode_shared_prefix"] = {"error": repr(e)}
         try:
             torch.cuda.empty_cache()
             others["smoothgemm"] = measure_gemm(dev, peaks)

@@ -113,7 +113,9 @@ typedef struct {
  * start at partial row `part0` and are `rows` apart. */
 typedef struct {
   int32_t req, kv_head, tok0, ntok;
-  int32_t part0, nsplit;
+  int32_t part0, nsplit;            /* partials of the unit's own KV splits: part0 + c * rows */
+  int32_t part1, nsplit1, stride1;  /* a second family (shared-prefix groups): part1 + c * stride1 */
+  int32_t reserved;
 } xy_attn_merge_unit;
 
 typedef struct {
@@ -146,6 +148,27 @@ int xy_attn_destroy(xy_attn_ctx* ctx);
 int xy_attn_plan(xy_attn_ctx* ctx, const xy_attn_request* reqs /*HOST*/, int32_t num_reqs,
                  const int32_t* tree_parents /*HOST, nullable if no tree*/, int32_t num_parents,
                  void* stream, xy_attn_plan_info* info /*HOST, nullable*/);
+
+/* Shared-prefix ("cascade") decode, a variant the paper's related work names (requests that share
+ * a radix-tree prefix batch their queries against it).  Requests first_req .. first_req+num_reqs-1
+ * must be decode requests (q_len 1, XY_MASK_CAUSAL) with kv_len >= prefix_tokens whose
+ * block-table rows hold THE SAME page ids for the first prefix_tokens tokens (prefix_tokens a
+ * positive multiple of 128).  Their query rows are packed into tiles that read the shared K/V
+ * once (dense tcgen05 tiles from 17 packed rows on), every member keeps a task for its own keys
+ * behind the prefix, and the split-KV merge kernel combines the two partials.  The result is
+ * the same attention as without groups; only the K/V traffic differs.  Groups must not overlap. */
+typedef struct {
+  int32_t first_req, num_reqs, prefix_tokens;
+} xy_attn_prefix_group;
+
+/* xy_attn_plan with shared-prefix groups (HOST array, read before return; num_groups = 0 is
+ * xy_attn_plan).  XY_PLAN_BALANCED only.  Errors as xy_attn_plan, plus XY_ERR_INVALID_ARG for a
+ * group that breaks the rules above and XY_ERR_CAPACITY when requests + groups exceed
+ * max_requests. */
+int xy_attn_plan_shared(xy_attn_ctx* ctx, const xy_attn_request* reqs /*HOST*/, int32_t num_reqs,
+                        const int32_t* tree_parents /*HOST, nullable*/, int32_t num_parents,
+                        const xy_attn_prefix_group* groups /*HOST*/, int32_t num_groups, void* stream,
+                        xy_attn_plan_info* info /*HOST, nullable*/);
 
 /* Task-Table cache (Section 3.3: the Task-Table is what the kernels consume; Section 3.3.2 keeps
  * pre-built Task-Tables for recurring shapes).  xy_attn_plan keeps the Task-Tables of the last

@@ -53,7 +53,12 @@ class xy_attn_task(ctypes.Structure):
 
 
 class xy_attn_merge_unit(ctypes.Structure):
-    _fields_ = [(n, ctypes.c_int32) for n in ("req", "kv_head", "tok0", "ntok", "part0", "nsplit")]
+    _fields_ = [(n, ctypes.c_int32) for n in ("req", "kv_head", "tok0", "ntok", "part0", "nsplit",
+                                              "part1", "nsplit1", "stride1", "reserved")]
+
+
+class xy_attn_prefix_group(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("first_req", "num_reqs", "prefix_tokens")]
 
 
 class xy_attn_plan_info(ctypes.Structure):
@@ -66,7 +71,8 @@ class xy_attn_plan_info(ctypes.Structure):
 
 
 TASK_DTYPE = np.dtype([(n, np.int32) for n in ("req", "kv_head", "tok0", "ntok", "kt_lo", "kt_hi", "part", "kind")])
-MERGE_DTYPE = np.dtype([(n, np.int32) for n in ("req", "kv_head", "tok0", "ntok", "part0", "nsplit")])
+MERGE_DTYPE = np.dtype([(n, np.int32) for n in ("req", "kv_head", "tok0", "ntok", "part0", "nsplit",
+                                                 "part1", "nsplit1", "stride1", "reserved")])
 
 EXPORTS = (
     "xy_attn_create", "xy_attn_destroy", "xy_attn_plan", "xy_attn_run", "xy_attn_merge",
@@ -75,6 +81,7 @@ EXPORTS = (
     "xy_attn_last_launches", "xy_attn_last_error", "xy_attn_device_status",
     "xy_attn_set_timing", "xy_attn_get_timing", "xy_attn_debug_trace", "xy_attn_decode_static",
     "xy_attn_append_kv", "xy_attn_worker_times", "xy_attn_get_queue", "xy_attn_plan_cache",
+    "xy_attn_plan_shared",
 )
 
 _lib = None
@@ -94,6 +101,7 @@ def load() -> ctypes.CDLL:
     L.xy_attn_create.argtypes = [ctypes.POINTER(xy_attn_config), ctypes.POINTER(vp)]
     L.xy_attn_destroy.argtypes = [vp]
     L.xy_attn_plan.argtypes = [vp, vp, i32, vp, i32, vp, ctypes.POINTER(xy_attn_plan_info)]
+    L.xy_attn_plan_shared.argtypes = [vp, vp, i32, vp, i32, vp, i32, vp, ctypes.POINTER(xy_attn_plan_info)]
     L.xy_attn_run.argtypes = [vp, vp, i64, vp, vp, i64, i64, i64, i64, vp, i32, vp, ctypes.c_float,
                               vp, i64, vp, vp]
     L.xy_attn_merge.argtypes = [vp, vp, i32, i64, i32, vp, vp, vp]
@@ -181,7 +189,26 @@ class XYAttn:
                                           int(par.size), _stream_ptr(stream), ctypes.byref(self.info)))
         return self.info
 
-    def plan_batch(self, batch, stream=None) -> xy_attn_plan_info:
+    def plan_shared(self, q_len, kv_len, mask_kind, parent_off, parents, groups, stream=None) -> xy_attn_plan_info:
+        """xy_attn_plan_shared: `groups` is a list of (first_req, num_reqs, prefix_tokens)."""
+        R = len(q_len)
+        reqs = (xy_attn_request * max(R, 1))()
+        for r in range(R):
+            reqs[r] = xy_attn_request(int(q_len[r]), int(kv_len[r]), int(mask_kind[r]), int(parent_off[r]))
+        par = np.ascontiguousarray(np.asarray(parents if parents is not None else [], dtype=np.int32))
+        par_ptr = ctypes.c_void_p(par.ctypes.data) if par.size else ctypes.c_void_p(0)
+        gs = (xy_attn_prefix_group * max(len(groups), 1))()
+        for k, g in enumerate(groups):
+            gs[k] = xy_attn_prefix_group(int(g[0]), int(g[1]), int(g[2]))
+        self._check(self.lib.xy_attn_plan_shared(self._ctx, ctypes.cast(reqs, ctypes.c_void_p), R, par_ptr,
+                                                 int(par.size), ctypes.cast(gs, ctypes.c_void_p), len(groups),
+                                                 _stream_ptr(stream), ctypes.byref(self.info)))
+        return self.info
+
+    def plan_batch(self, batch, stream=None, groups=None) -> xy_attn_plan_info:
+        if groups:
+            return self.plan_shared(batch.q_len, batch.kv_len, batch.mask_kind, batch.parent_off, batch.parents,
+                                    groups, stream)
         return self.plan(batch.q_len, batch.kv_len, batch.mask_kind, batch.parent_off, batch.parents, stream)
 
     # -- xy_attn_run

@@ -2,6 +2,8 @@
 // marshalling only; every step of the path runs in the kernels.
 #include <cuda_runtime.h>
 
+#include <algorithm>
+
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -185,11 +187,19 @@ int xy_attn_destroy(xy_attn_ctx* ctx) {
 int xy_attn_plan(xy_attn_ctx* ctx, const xy_attn_request* reqs, int32_t num_reqs,
                  const int32_t* tree_parents, int32_t num_parents, void* stream,
                  xy_attn_plan_info* info) {
+  return xy_attn_plan_shared(ctx, reqs, num_reqs, tree_parents, num_parents, nullptr, 0, stream, info);
+}
+
+int xy_attn_plan_shared(xy_attn_ctx* ctx, const xy_attn_request* reqs, int32_t num_reqs,
+                        const int32_t* tree_parents, int32_t num_parents,
+                        const xy_attn_prefix_group* groups, int32_t num_groups, void* stream,
+                        xy_attn_plan_info* info) {
   if (ctx == nullptr) return XY_ERR_INVALID_ARG;
   ctx->planned = false;
   std::string err;
   int rc = build_plan(ctx->cfg, ctx->num_workers, ctx->cap_partial_rows, reqs, num_reqs,
-                      tree_parents, num_parents, &ctx->plan, &err, ctx->cache.capacity > 0 ? &ctx->cache : nullptr);
+                      tree_parents, num_parents, &ctx->plan, &err, ctx->cache.capacity > 0 ? &ctx->cache : nullptr,
+                      groups, num_groups);
   if (rc != XY_OK) {
     ctx->plan = PlanResult();
     return set_err(ctx, rc, err);
@@ -331,7 +341,10 @@ int xy_attn_run(xy_attn_ctx* ctx, const void* q, int64_t q_token_stride, const v
     m.lse = lse;
     m.num_q_heads = cfg.num_q_heads;
     m.num_kv_heads = cfg.num_kv_heads;
-    XY_CUDA(ctx, launch_merge_units(m, static_cast<int>(p.merges.size()), s));
+    int max_rows = 1;
+    for (const xy_attn_merge_unit& mu : p.merges)
+      max_rows = std::max(max_rows, mu.ntok * (cfg.num_q_heads / cfg.num_kv_heads));
+    XY_CUDA(ctx, launch_merge_units(m, static_cast<int>(p.merges.size()), max_rows, s));
     ctx->last_launches += 1;
   }
   if (timed) {

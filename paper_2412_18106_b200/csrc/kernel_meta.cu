@@ -712,7 +712,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
           f_hi = t.kt_hi;
           f_head = t.kv_head;
           f_npages = (rq.kv_len + rq.q_len + a.page_size - 1) >> a.page_shift;
-          f_bt = a.block_table + static_cast<int64_t>(t.req) * a.bt_stride;
+          f_bt = a.block_table + static_cast<int64_t>(rq.bt_row) * a.bt_stride;
           f_umma = kUmma && t.kind == 0;
           f_open = true;
         }

@@ -34,7 +34,7 @@ __global__ void __launch_bounds__(128) ref_attention_kernel(RunArgs a) {
     const xy_attn_task t = a.tasks[ti];
     const ReqInfo rq = a.reqs[t.req];
     const int rows = t.ntok * G;
-    const int32_t* bt = a.block_table + static_cast<int64_t>(t.req) * a.bt_stride;
+    const int32_t* bt = a.block_table + static_cast<int64_t>(rq.bt_row) * a.bt_stride;
     for (int x = warp; x < rows; x += 4) {
       const int i = t.tok0 + x / G;
       const int head = t.kv_head * G + x % G;
@@ -101,11 +101,18 @@ __global__ void __launch_bounds__(128) merge_units_kernel(MergeArgs a) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (blockIdx.y * 4 >= rows) return;
   const ReqInfo rq = a.reqs[u.req];
-  for (int x = blockIdx.y * 4 + warp; x < rows; x += 4 * kMergeBlocksPerUnit) {
+  for (int x = blockIdx.y * 4 + warp; x < rows; x += 4 * gridDim.y) {
     float lse;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (u.nsplit <= 32) {
-      const float lc = lane < u.nsplit ? a.lse_part[u.part0 + lane * rows + x] : -INFINITY;
+    // partial row of part c: the unit's own splits first, then the second family (the rows a
+    // member of a shared-prefix group has in the group tile's partials)
+    const int nparts = u.nsplit + u.nsplit1;
+    auto part_row = [&](int c) -> int64_t {
+      return c < u.nsplit ? static_cast<int64_t>(u.part0) + static_cast<int64_t>(c) * rows + x
+                          : static_cast<int64_t>(u.part1) + static_cast<int64_t>(c - u.nsplit) * u.stride1 + x;
+    };
+    if (nparts <= 32) {
+      const float lc = lane < nparts ? a.lse_part[part_row(lane)] : -INFINITY;
       float mx = lc;
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
@@ -115,11 +122,10 @@ __global__ void __launch_bounds__(128) merge_units_kernel(MergeArgs a) {
       for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
       lse = mx + logf(z);
       const float w_mine = z > 0.f ? e / z : 0.f;
-      for (int c = 0; c < u.nsplit; ++c) {
+      for (int c = 0; c < nparts; ++c) {
         const float w = __shfl_sync(0xffffffffu, w_mine, c);
         if (w == 0.f) continue;  // empty split (LSE_c = -inf): its O_c is not read
-        const float4 v = *reinterpret_cast<const float4*>(
-            a.o_part + static_cast<int64_t>(u.part0 + c * rows + x) * kHeadDim + lane * 4);
+        const float4 v = *reinterpret_cast<const float4*>(a.o_part + part_row(c) * kHeadDim + lane * 4);
         acc.x += w * v.x;
         acc.y += w * v.y;
         acc.z += w * v.z;
@@ -127,19 +133,18 @@ __global__ void __launch_bounds__(128) merge_units_kernel(MergeArgs a) {
       }
     } else {
       float mx = -INFINITY;
-      for (int c = 0; c < u.nsplit; ++c) mx = fmaxf(mx, a.lse_part[u.part0 + c * rows + x]);
+      for (int c = 0; c < nparts; ++c) mx = fmaxf(mx, a.lse_part[part_row(c)]);
       float z = 0.f;
-      for (int c = 0; c < u.nsplit; ++c) {
-        const float lc = a.lse_part[u.part0 + c * rows + x];
+      for (int c = 0; c < nparts; ++c) {
+        const float lc = a.lse_part[part_row(c)];
         if (lc != -INFINITY) z += __expf(lc - mx);
       }
       lse = mx + logf(z);
-      for (int c = 0; c < u.nsplit; ++c) {
-        const float lc = a.lse_part[u.part0 + c * rows + x];
+      for (int c = 0; c < nparts; ++c) {
+        const float lc = a.lse_part[part_row(c)];
         if (lc == -INFINITY) continue;
         const float w = __expf(lc - lse);
-        const float4 v = *reinterpret_cast<const float4*>(
-            a.o_part + static_cast<int64_t>(u.part0 + c * rows + x) * kHeadDim + lane * 4);
+        const float4 v = *reinterpret_cast<const float4*>(a.o_part + part_row(c) * kHeadDim + lane * 4);
         acc.x += w * v.x;
         acc.y += w * v.y;
         acc.z += w * v.z;
@@ -252,9 +257,12 @@ cudaError_t launch_reference(const RunArgs& a, int num_workers, cudaStream_t s) 
   return cudaGetLastError();
 }
 
-cudaError_t launch_merge_units(const MergeArgs& a, int num_units, cudaStream_t s) {
+cudaError_t launch_merge_units(const MergeArgs& a, int num_units, int max_rows, cudaStream_t s) {
   if (num_units == 0) return cudaSuccess;
-  merge_units_kernel<<<dim3(num_units, kMergeBlocksPerUnit), 128, 0, s>>>(a);
+  // one warp per row of the largest unit (four rows per block), at most kMergeBlocksPerUnit blocks
+  int by = (max_rows + 3) / 4;
+  by = by < 1 ? 1 : (by > kMergeBlocksPerUnit ? kMergeBlocksPerUnit : by);
+  merge_units_kernel<<<dim3(num_units, by), 128, 0, s>>>(a);
   return cudaGetLastError();
 }
 

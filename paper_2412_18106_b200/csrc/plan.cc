@@ -41,7 +41,9 @@ constexpr float kDenseCapFactor = 0.65f;
 
 struct Unit {
   int32_t req, kv_head, tok0, ntok, kind;
-  int32_t nkt;       // visible 128-key tiles
+  int32_t nkt;       // visible 128-key tiles: the unit's tasks cover tiles kt0 .. nkt-1
+  int32_t kt0;       // first tile (> 0: the suffix of a member of a shared-prefix group)
+  int32_t group;     // -1, or the shared-prefix group this unit belongs to (then always partial)
   float visit_cost;  // per kv tile
   float paper_load;  // rows x visible keys
 };
@@ -52,7 +54,8 @@ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
 int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_capacity,
                const xy_attn_request* reqs, int32_t num_reqs, const int32_t* tree_parents,
-               int32_t num_parents, PlanResult* out, std::string* err, PlanCache* cache) {
+               int32_t num_parents, PlanResult* out, std::string* err, PlanCache* cache,
+               const xy_attn_prefix_group* groups, int32_t num_groups) {
   *out = PlanResult();
   char buf[256];
   auto fail = [&](int code, const char* msg) {
@@ -60,7 +63,8 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
     return code;
   };
   if (num_reqs < 0 || (num_reqs > 0 && reqs == nullptr)) return fail(XY_ERR_INVALID_ARG, "reqs is null");
-  if (num_reqs > cfg.max_requests) return fail(XY_ERR_CAPACITY, "num_reqs exceeds max_requests");
+  if (static_cast<int64_t>(num_reqs) + std::max(num_groups, 0) > cfg.max_requests)
+    return fail(XY_ERR_CAPACITY, "num_reqs (+ groups) exceeds max_requests");
   if (num_parents < 0) return fail(XY_ERR_INVALID_ARG, "num_parents < 0");
   const int G = cfg.num_q_heads / cfg.num_kv_heads;
   const int B = cfg.page_size;
@@ -98,7 +102,8 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
     ri.mask_kind = q.mask_kind;
     ri.tree_off = 0;
     ri.tree_words = 0;
-    ri.pad0 = ri.pad1 = 0;
+    ri.bt_row = r;
+    ri.pad1 = 0;
     out->q_start[r + 1] = static_cast<int32_t>(total_q);
     kv_tokens += L;
     const int64_t n = q.q_len, h = q.kv_len;
@@ -142,6 +147,41 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
   }
   out->total_q = total_q;
 
+  // ---- shared-prefix groups: validation, and one virtual request per group ----------------
+  // A group's members are consecutive decode requests whose first prefix_tokens keys are the same
+  // pages.  Their queries form a virtual request (q rows of the members, kvLen = prefix_tokens,
+  // block-table row of the first member) whose tiles cover the shared keys once; every member
+  // keeps a task for its own keys behind the prefix; the merge kernel combines the two.
+  if (num_groups < 0 || (num_groups > 0 && groups == nullptr)) return fail(XY_ERR_INVALID_ARG, "groups is null");
+  if (num_groups > 0 && cfg.plan_mode == XY_PLAN_PAPER)
+    return fail(XY_ERR_UNSUPPORTED, "shared-prefix groups need the balanced plan mode");
+  std::vector<int32_t> group_of(num_reqs, -1);
+  for (int gi = 0; gi < num_groups; ++gi) {
+    const xy_attn_prefix_group& gr = groups[gi];
+    if (gr.num_reqs < 1 || gr.first_req < 0 || static_cast<int64_t>(gr.first_req) + gr.num_reqs > num_reqs ||
+        gr.prefix_tokens < kKeyTile || gr.prefix_tokens % kKeyTile != 0) {
+      snprintf(buf, sizeof buf, "group %d: bad request range or prefix_tokens not a positive multiple of 128", gi);
+      return fail(XY_ERR_INVALID_ARG, buf);
+    }
+    for (int r = gr.first_req; r < gr.first_req + gr.num_reqs; ++r) {
+      if (group_of[r] >= 0 || reqs[r].q_len != 1 || reqs[r].mask_kind != XY_MASK_CAUSAL ||
+          reqs[r].kv_len < gr.prefix_tokens) {
+        snprintf(buf, sizeof buf, "group %d: request %d is not a decode request with kv_len >= prefix_tokens, or is in two groups", gi, r);
+        return fail(XY_ERR_INVALID_ARG, buf);
+      }
+      group_of[r] = gi;
+    }
+    ReqInfo v;
+    v.q_start = out->reqs[gr.first_req].q_start;
+    v.q_len = gr.num_reqs;
+    v.kv_len = gr.prefix_tokens;
+    v.mask_kind = XY_MASK_CAUSAL;
+    v.tree_off = v.tree_words = 0;
+    v.bt_row = gr.first_req;
+    v.pad1 = 0;
+    out->reqs.push_back(v);
+  }
+
   // ---- a2: decomposition ----------------------------------------------------------------
   const bool paper = cfg.plan_mode == XY_PLAN_PAPER;
   const int sub_tok = std::max(1, 128 / G);  // tokens of one 128-row sub-tile
@@ -150,8 +190,11 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
   if (paper && cfg.kernel != XY_KERNEL_REFERENCE && dense_tok * G > 128 * subtiles)
     return fail(XY_ERR_UNSUPPORTED, "paper-mode tile_tokens x (Hq/Hkv) exceeds the rows one task may hold");
   std::vector<Unit> units;
-  for (int r = 0; r < num_reqs; ++r) {
-    const int n = reqs[r].q_len, h = reqs[r].kv_len;
+  for (int r = 0; r < num_reqs + num_groups; ++r) {
+    const bool is_virtual = r >= num_reqs;
+    const int n = is_virtual ? groups[r - num_reqs].num_reqs : reqs[r].q_len;
+    const int h = is_virtual ? groups[r - num_reqs].prefix_tokens : reqs[r].kv_len;
+    const int gidx = is_virtual ? r - num_reqs : group_of[r];
     // q tiles of this request (same for every kv head)
     std::vector<std::pair<int, int>> tiles;  // tok0, ntok
     if (paper) {
@@ -170,8 +213,11 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
         u.ntok = t.second;
         const int rows = u.ntok * G;
         u.kind = rows <= kStreamRowsMax ? 1 : 0;
-        const int visible = h + u.tok0 + u.ntok;
+        // a virtual request's tiles stop at the end of the shared prefix (its rows see all of it)
+        const int visible = is_virtual ? h : h + u.tok0 + u.ntok;
         u.nkt = ceil_div(visible, kKeyTile);
+        u.group = gidx;
+        u.kt0 = (!is_virtual && gidx >= 0) ? groups[gidx].prefix_tokens / kKeyTile : 0;
         if (u.kind == 1) {
           u.visit_cost = kStreamVisitUs;
         } else {
@@ -186,7 +232,7 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
   // ---- Task-Table cache: everything below depends on the requests only through the units
   // (request, kv head, q tile, kind, visible key tiles), so an equal decomposition has an equal
   // Task-Table.  The useful-flop and byte counts depend on the exact kvLen and are always fresh.
-  out->shape.reserve(units.size() * 6 + 4);
+  out->shape.reserve(units.size() * 8 + 4);
   out->shape.push_back(num_workers);
   out->shape.push_back(static_cast<int32_t>(std::min<int64_t>(partial_row_capacity, INT32_MAX)));
   out->shape.push_back(cfg.plan_mode * 4 + cfg.kernel);
@@ -198,6 +244,8 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
     out->shape.push_back(u.ntok);
     out->shape.push_back(u.kind);
     out->shape.push_back(paper ? static_cast<int32_t>(reqs[u.req].kv_len) : u.nkt);
+    out->shape.push_back(u.kt0);
+    out->shape.push_back(u.group);
   }
   {
     uint64_t hsh = 1469598103934665603ull;  // FNV-1a over the 32-bit words
@@ -230,7 +278,7 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
   // KV splits: cap the cost of one task at a fraction of the mean per-worker load.
   const int max_splits = cfg.max_splits > 0 ? cfg.max_splits : 32;
   double total_cost = 0.0;
-  for (const Unit& u : units) total_cost += kTaskFixedUs + u.visit_cost * u.nkt;
+  for (const Unit& u : units) total_cost += kTaskFixedUs + u.visit_cost * (u.nkt - u.kt0);
   float cap = static_cast<float>(total_cost / std::max(1, num_workers) * kTaskCapFraction);
   const float dense_factor = kDenseCapFactor;
   std::vector<int> chunk_tiles(units.size(), 0);
@@ -240,17 +288,19 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
       const Unit& u = units[k];
       int nsplit = 1;
       if (!paper) {
-        const float cost = u.visit_cost * u.nkt;
+        const int nt = u.nkt - u.kt0;
+        const float cost = u.visit_cost * nt;
         const float cap_u = u.kind == 1 ? cap : cap * dense_factor;
         nsplit = static_cast<int>(std::ceil(cost / std::max(cap_u, 1e-3f)));
         nsplit = std::min(nsplit, max_splits);
-        nsplit = std::min(nsplit, std::max(1, u.nkt / kMinChunkTiles));
+        nsplit = std::min(nsplit, std::max(1, nt / kMinChunkTiles));
         nsplit = std::max(nsplit, 1);
       }
-      int chunk = ceil_div(std::max(u.nkt, 1), nsplit);
-      nsplit = ceil_div(std::max(u.nkt, 1), chunk);
+      const int nt = std::max(u.nkt - u.kt0, 1);
+      int chunk = ceil_div(nt, nsplit);
+      nsplit = ceil_div(nt, chunk);
       chunk_tiles[k] = chunk;
-      if (nsplit > 1) prow += static_cast<int64_t>(nsplit) * u.ntok * G;
+      if (nsplit > 1 || u.group >= 0) prow += static_cast<int64_t>(nsplit) * u.ntok * G;
     }
     if (prow <= partial_row_capacity) break;
     cap *= 1.5f;  // fewer splits until the partials fit the workspace
@@ -263,13 +313,17 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
   };
   std::vector<Pending> pend;
   int64_t prow = 0;
+  std::vector<int32_t> unit_part(units.size(), -1), unit_nsplit(units.size(), 1);
   for (size_t k = 0; k < units.size(); ++k) {
     const Unit& u = units[k];
     const int chunk = chunk_tiles[k];
-    const int nsplit = ceil_div(std::max(u.nkt, 1), chunk);
+    const int nsplit = ceil_div(std::max(u.nkt - u.kt0, 1), chunk);
     const int rows = u.ntok * G;
-    if (nsplit > 1) {
-      xy_attn_merge_unit mu{u.req, u.kv_head, u.tok0, u.ntok, static_cast<int32_t>(prow), nsplit};
+    const bool partial = nsplit > 1 || u.group >= 0;  // group units always leave partials
+    unit_nsplit[k] = nsplit;
+    if (partial) unit_part[k] = static_cast<int32_t>(prow);
+    if (nsplit > 1 && u.group < 0) {
+      xy_attn_merge_unit mu{u.req, u.kv_head, u.tok0, u.ntok, static_cast<int32_t>(prow), nsplit, 0, 0, 0, 0};
       out->merges.push_back(mu);
     }
     for (int c = 0; c < nsplit; ++c) {
@@ -278,14 +332,29 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
       p.t.kv_head = u.kv_head;
       p.t.tok0 = u.tok0;
       p.t.ntok = u.ntok;
-      p.t.kt_lo = c * chunk;
-      p.t.kt_hi = std::min(u.nkt, (c + 1) * chunk);
-      p.t.part = nsplit > 1 ? static_cast<int32_t>(prow + static_cast<int64_t>(c) * rows) : -1;
+      p.t.kt_lo = u.kt0 + c * chunk;
+      p.t.kt_hi = std::min(u.nkt, u.kt0 + (c + 1) * chunk);
+      p.t.part = partial ? static_cast<int32_t>(prow + static_cast<int64_t>(c) * rows) : -1;
       p.t.kind = u.kind;
       p.cost = paper ? u.paper_load : kTaskFixedUs + u.visit_cost * (p.t.kt_hi - p.t.kt_lo);
       pend.push_back(p);
     }
-    if (nsplit > 1) prow += static_cast<int64_t>(nsplit) * rows;
+    if (partial) prow += static_cast<int64_t>(nsplit) * rows;
+  }
+  // Merge units of the members of shared-prefix groups: the member's own partials (its keys
+  // behind the prefix) plus its rows of the group tile's partials (the shared keys).
+  for (size_t k = 0; k < units.size(); ++k) {
+    const Unit& u = units[k];
+    if (u.group < 0 || u.req >= num_reqs) continue;  // members only
+    const int m = u.req - groups[u.group].first_req;   // index of the member = its token in the group
+    for (size_t v = 0; v < units.size(); ++v) {
+      const Unit& w = units[v];
+      if (w.req != num_reqs + u.group || w.kv_head != u.kv_head || m < w.tok0 || m >= w.tok0 + w.ntok) continue;
+      xy_attn_merge_unit mu{u.req, u.kv_head, 0, 1, unit_part[k], unit_nsplit[k],
+                            unit_part[v] + (m - w.tok0) * G, unit_nsplit[v], w.ntok * G, 0};
+      out->merges.push_back(mu);
+      break;
+    }
   }
   out->partial_rows = prow;
 

@@ -23,7 +23,8 @@ struct ReqInfo {
   int32_t mask_kind;  // XY_MASK_*
   int32_t tree_off;   // first 64-bit word of the request's corner mask
   int32_t tree_words; // words per corner-mask row
-  int32_t pad0, pad1;
+  int32_t bt_row;     // block-table row the request's pages are looked up in
+  int32_t pad1;
 };
 
 struct PlanResult {
@@ -70,9 +71,11 @@ inline int dense_subtiles(const xy_attn_config& cfg) { return cfg.kernel == XY_K
 // Host-only planning.  Returns XY_OK or an error code and fills `err`.
 // `cache` (nullable): Task-Tables of earlier plans; a plan whose decomposition equals a cached one
 // takes its Task-Table from there and only rebuilds the Token-Table and the tree masks.
+// `groups` (nullable): shared-prefix decode groups, see xy_attn_plan_shared.
 int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_capacity,
                const xy_attn_request* reqs, int32_t num_reqs, const int32_t* tree_parents,
-               int32_t num_parents, PlanResult* out, std::string* err, PlanCache* cache = nullptr);
+               int32_t num_parents, PlanResult* out, std::string* err, PlanCache* cache = nullptr,
+               const xy_attn_prefix_group* groups = nullptr, int32_t num_groups = 0);
 
 // Arguments every attention kernel takes.
 struct RunArgs {

@@ -20,7 +20,7 @@ struct MergeArgs {
 
 cudaError_t launch_reference(const RunArgs& a, int num_workers, cudaStream_t s);
 cudaError_t launch_meta(const RunArgs& a, int num_workers, int64_t num_pages, bool umma, cudaStream_t s);
-cudaError_t launch_merge_units(const MergeArgs& a, int num_units, cudaStream_t s);
+cudaError_t launch_merge_units(const MergeArgs& a, int num_units, int max_rows, cudaStream_t s);
 cudaError_t launch_merge_plain(const float* o_part, const float* lse_part, int num_splits,
                                int64_t rows, uint16_t* o, float* lse, cudaStream_t s);
 cudaError_t launch_append_kv(const uint16_t* qkv, int64_t qkv_token_stride, uint16_t* k_pool, uint16_t* v_pool,

@@ -251,6 +251,27 @@ CONFIGS = {
 }
 
 
+def shared_prefix_decode(seed: int = 0, num_groups: int = 4, members: int = 32, prefix: int = 8192,
+                         suffix_hi: int = 1024, hq: int = 32, hkv: int = 8, page_size: int = 128):
+    """Decode requests that share cached prefixes (a common system prompt, a radix-tree branch):
+    `num_groups` groups of `members` requests; the members of a group hold THE SAME pages for their
+    first `prefix` tokens (a multiple of 128) and then own `0 .. suffix_hi` further tokens each.
+    Returns (batch, groups) with groups = [(first_req, num_reqs, prefix_tokens), ...]."""
+    assert prefix % 128 == 0 and prefix % page_size == 0
+    rng = np.random.default_rng(seed)
+    R = num_groups * members
+    kv = [prefix + int(x) for x in rng.integers(0, suffix_hi + 1, size=R)]
+    b = assemble("decode_shared_prefix", hq, hkv, page_size, [1] * R, kv, [MASK_CAUSAL] * R, [None] * R, rng, seed)
+    npre = prefix // page_size
+    groups = []
+    for g in range(num_groups):
+        first = g * members
+        for r in range(first + 1, first + members):
+            b.block_table[r, :npre] = b.block_table[first, :npre]
+        groups.append((first, members, prefix))
+    return b, groups
+
+
 def custom(name: str, hq: int, hkv: int, page_size: int, requests, seed: int = 0,
            permute_pages: bool = True, spare_frac: float = 0.10) -> Batch:
     """`requests` is a list of (q_len, kv_len, kind, parents-or-None) tuples."""

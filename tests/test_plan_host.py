@@ -34,7 +34,7 @@ def test_library_exports_every_declared_symbol():
 def test_struct_sizes_match_header():
     assert ctypes.sizeof(xb.xy_attn_task) == 32
     assert ctypes.sizeof(xb.xy_attn_request) == 16
-    assert ctypes.sizeof(xb.xy_attn_merge_unit) == 24
+    assert ctypes.sizeof(xb.xy_attn_merge_unit) == 40
     assert ctypes.sizeof(xb.xy_attn_config) == 14 * 4 + 8
 
 
@@ -296,3 +296,54 @@ def test_task_table_cache_reuses_equal_decompositions_bit_exactly():
     assert c.plan_cache(0) == (4, 2)
     c.plan_batch(b0)
     assert c.plan_cache() == (4, 2)
+
+
+def test_shared_prefix_groups_cover_every_key_once_and_reject_bad_groups():
+    """A shared-prefix group turns the members' first `prefix` keys into tiles of one virtual
+    request (read once) and leaves each member a task for its own keys; together they cover every
+    (member, kv head, key tile) exactly once, and each member gets one merge unit with both
+    families of partials."""
+    b, groups = W.shared_prefix_decode(seed=3, num_groups=3, members=20, prefix=1024, suffix_hi=700,
+                                       hq=8, hkv=2, page_size=64)
+    c = host_ctx(8, 2, 64, max_requests=256)
+    info = c.plan_batch(b, groups=groups)
+    tasks, merges = c.get_tasks(), c.get_merge_units()
+    R, G = b.num_requests, 4
+    assert info.useful_flops == W.useful_flops(b)
+    for gi, (first, n, prefix) in enumerate(groups):
+        vt = tasks[tasks["req"] == R + gi]
+        assert len(vt) and np.all(vt["part"] >= 0) and np.all(vt["kt_hi"] <= prefix // 128)
+        for g in range(2):
+            for m in range(n):
+                r = first + m
+                need = -(-(int(b.kv_len[r]) + 1) // 128)
+                cover = np.zeros(need, np.int32)
+                for t in vt[(vt["kv_head"] == g) & (vt["tok0"] <= m) & (m < vt["tok0"] + vt["ntok"])]:
+                    cover[t["kt_lo"]: t["kt_hi"]] += 1
+                own = tasks[(tasks["req"] == r) & (tasks["kv_head"] == g)]
+                assert len(own) >= 1 and np.all(own["part"] >= 0) and own["kt_lo"].min() == prefix // 128
+                for t in own:
+                    cover[t["kt_lo"]: t["kt_hi"]] += 1
+                assert np.all(cover == 1), (r, g)
+                mu = merges[(merges["req"] == r) & (merges["kv_head"] == g)]
+                assert len(mu) == 1 and mu["nsplit"][0] == len(own) and mu["nsplit1"][0] >= 1
+                assert mu["stride1"][0] % G == 0
+    # the queue is still a permutation; partial rows are disjoint
+    assert sorted(c.get_queue().tolist()) == list(range(len(tasks)))
+    used = np.zeros(int(info.partial_rows), np.int32)
+    for t in tasks[tasks["part"] >= 0]:
+        used[t["part"]: t["part"] + t["ntok"] * G] += 1
+    assert np.all(used == 1)
+    # bad groups
+    def code(gs):
+        with pytest.raises(xb.XYAttnError) as e:
+            c.plan_batch(b, groups=gs)
+        return e.value.code
+    assert code([(0, 20, 1000)]) == xb.XY_ERR_INVALID_ARG         # prefix not a multiple of 128
+    assert code([(0, 20, 1024), (10, 5, 1024)]) == xb.XY_ERR_INVALID_ARG  # overlap
+    assert code([(50, 20, 1024)]) == xb.XY_ERR_INVALID_ARG        # range beyond the batch
+    assert code([(0, 20, 4096)]) == xb.XY_ERR_INVALID_ARG         # prefix longer than a member's kv_len
+    pb = W.custom("p", 8, 2, 64, [(5, 2000, 0, None), (1, 2000, 0, None)], seed=1)
+    with pytest.raises(xb.XYAttnError) as e:
+        c.plan_batch(pb, groups=[(0, 2, 1024)])                   # a prefill request in a group
+    assert e.value.code == xb.XY_ERR_INVALID_ARG
