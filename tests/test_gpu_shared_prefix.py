@@ -52,3 +52,43 @@ def test_groups_beside_other_requests_and_member_without_suffix():
     O_ref, LSE_ref = oracle.attention(b, t, H.SCALE)
     H.check_against_oracle(O, LSE, O_ref, LSE_ref, "mixed groups")
     ctx.close()
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_random_groups(seed):
+    """Random mixes: several groups of random size and prefix length between ungrouped prefill,
+    decode and verify requests; random head ratio, page size and worker count."""
+    rng = np.random.default_rng(1000 + seed)
+    hkv = int(rng.choice([1, 2, 4]))
+    G = int(rng.choice([1, 2, 4, 8]))
+    page = int(rng.choice([16, 32, 64, 128]))
+    reqs, groups = [], []
+    for _ in range(int(rng.integers(1, 4))):
+        for _ in range(int(rng.integers(0, 3))):  # ungrouped requests before the group
+            k = rng.random()
+            if k < 0.4:
+                reqs.append((1, int(rng.integers(1, 900)), 0, None))
+            elif k < 0.7:
+                reqs.append((int(rng.integers(2, 90)), int(rng.integers(0, 500)), 0, None))
+            else:
+                n = int(rng.integers(2, 20))
+                reqs.append((n, int(rng.integers(0, 500)), 1, W.random_tree(rng, n, 5)))
+        n = int(rng.integers(1, 45))
+        prefix = 128 * int(rng.integers(1, 9))
+        groups.append((len(reqs), n, prefix))
+        for _ in range(n):
+            reqs.append((1, prefix + int(rng.integers(0, 400)), 0, None))
+    b = W.custom("rgroups%d" % seed, hkv * G, hkv, page, reqs, seed=seed)
+    for first, n, prefix in groups:
+        npre = prefix // page
+        for r in range(first + 1, first + n):
+            b.block_table[r, :npre] = b.block_table[first, :npre]
+    t = W.make_tensors(b)
+    ctx = H.make_ctx(b, num_workers=int(rng.choice([1, 5, 148])), max_requests=512)
+    ctx.plan_batch(b, groups=groups)
+    O_ref, LSE_ref = oracle.attention(b, t, H.SCALE)
+    O, LSE = H.run_gpu(b, t, ctx=ctx)
+    H.check_against_oracle(O, LSE, O_ref, LSE_ref, "random groups %d" % seed)
+    O2, LSE2 = H.run_gpu(b, t, ctx=ctx)
+    assert np.array_equal(O, O2) and np.array_equal(LSE, LSE2)
+    ctx.close()
