@@ -418,11 +418,14 @@ __device__ __forceinline__ uint32_t stream_task(const RunArgs& a, const TaskView
   {
     const int xl = lane >> 2, xh = xl + 8;
     float* mine = xch + warp * (16 * kHeadDim);
+    // only the task's rows are merged below: padding rows (most of the 16 in a decode step) are
+    // not written
+    const bool has_lo = xl < tv.rows, has_hi = xh < tv.rows;
 #pragma unroll
     for (int n = 0; n < 16; ++n) {
       const int col = n * 8 + 2 * (lane & 3);
-      *reinterpret_cast<float2*>(mine + xl * kHeadDim + col) = make_float2(w.o[n][0], w.o[n][1]);
-      *reinterpret_cast<float2*>(mine + xh * kHeadDim + col) = make_float2(w.o[n][2], w.o[n][3]);
+      if (has_lo) *reinterpret_cast<float2*>(mine + xl * kHeadDim + col) = make_float2(w.o[n][0], w.o[n][1]);
+      if (has_hi) *reinterpret_cast<float2*>(mine + xh * kHeadDim + col) = make_float2(w.o[n][2], w.o[n][3]);
     }
     if ((lane & 3) == 0) {
       ml[(warp * 16 + xl) * 2 + 0] = w.m_lo;
