@@ -244,7 +244,8 @@ def measure_stream(kernel, dev, peaks, chunks=48, budget=4096, reserved=512, ses
     verify a token tree instead; the chunk former cuts fixed-budget chunks, every chunk is planned
     (Task-Table cache on) and run.  K/V pool and Q are random and resident; the block table maps
     every session onto random pages of one pool (contents do not matter for timing).  Reports the
-    host time of chunk forming and planning and the device time of attention per chunk."""
+    host time of chunk forming and planning (the C calls, chunk handed from one to the other as
+    the request array) and the device time of attention per chunk."""
     import torch
 
     from paper_2412_18106_b200 import binding as xb
@@ -282,18 +283,14 @@ def measure_stream(kernel, dev, peaks, chunks=48, budget=4096, reserved=512, ses
     e0.record()
     while done < chunks and sch.pending() != (0, 0):
         t0 = time.perf_counter()
-        chunk = sch.next_chunk()
+        n, reqs_raw, ents_raw, par_raw, npar = sch.next_chunk_raw()
         t1 = time.perf_counter()
-        ql = [e["q_len"] for e in chunk]
-        kl = [e["kv_len"] for e in chunk]
-        mk = [1 if e["parents"] is not None else 0 for e in chunk]
-        par, off = [], []
-        for e in chunk:
-            off.append(len(par) if e["parents"] is not None else -1)
-            par += e["parents"] or []
-        t2 = time.perf_counter()
-        info = ctx.plan(ql, kl, mk, off, np.asarray(par, np.int32) if par else None)
+        info = ctx.plan_raw(reqs_raw, n, par_raw, npar)
         t3 = time.perf_counter()
+        t2 = t1
+        chunk = [dict(id=int(ents_raw[k].id), kind=int(ents_raw[k].kind), last=bool(ents_raw[k].last),
+                      q_len=int(reqs_raw[k].q_len), kv_len=int(reqs_raw[k].kv_len)) for k in range(n)]
+        ql = [e["q_len"] for e in chunk]
         rows = torch.tensor([e["id"] for e in chunk], dtype=torch.long)
         bt_dev[: len(chunk)].copy_(bt_all[rows], non_blocking=False)
         T = int(sum(ql))

@@ -189,6 +189,14 @@ class XYAttn:
                                           int(par.size), _stream_ptr(stream), ctypes.byref(self.info)))
         return self.info
 
+    def plan_raw(self, reqs, num_reqs: int, parents: Optional[np.ndarray], num_parents: int,
+                 stream=None) -> xy_attn_plan_info:
+        """xy_attn_plan on an xy_attn_request array as the chunk former returns it."""
+        par_ptr = ctypes.c_void_p(parents.ctypes.data) if (parents is not None and num_parents) else ctypes.c_void_p(0)
+        self._check(self.lib.xy_attn_plan(self._ctx, ctypes.cast(reqs, ctypes.c_void_p), int(num_reqs), par_ptr,
+                                          int(num_parents), _stream_ptr(stream), ctypes.byref(self.info)))
+        return self.info
+
     def plan_shared(self, q_len, kv_len, mask_kind, parent_off, parents, groups, stream=None) -> xy_attn_plan_info:
         """xy_attn_plan_shared: `groups` is a list of (first_req, num_reqs, prefix_tokens)."""
         R = len(q_len)

@@ -90,6 +90,17 @@ class XYSched:
         self._check(self.lib.xy_sched_pending(self._s, ctypes.byref(p), ctypes.byref(d)))
         return int(p.value), int(d.value)
 
+    def next_chunk_raw(self):
+        """The next chunk without Python objects per entry: (n, requests, entries, parents,
+        num_parents) where requests is the xy_attn_request array xy_attn_plan takes as it is
+        (valid until the next call)."""
+        npar = ctypes.c_int32(0)
+        n = self._check(self.lib.xy_sched_next_chunk(
+            self._s, ctypes.cast(self._reqs, ctypes.c_void_p), ctypes.cast(self._entries, ctypes.c_void_p),
+            self.cfg.max_requests, ctypes.c_void_p(self._parents.ctypes.data), int(self._parents.size),
+            ctypes.byref(npar)))
+        return n, self._reqs, self._entries, self._parents, int(npar.value)
+
     def next_chunk(self) -> List[dict]:
         """The next chunk as a list of dicts (id, kind, q_len, kv_len, last, parents)."""
         npar = ctypes.c_int32(0)
