@@ -223,6 +223,27 @@ int xy_attn_append_kv(xy_attn_ctx* ctx, const void* qkv, int64_t qkv_token_strid
 int xy_attn_merge(const float* o_part, const float* lse_part, int32_t num_splits, int64_t rows,
                   int32_t head_dim, void* o, float* lse, void* stream);
 
+/* Context sharded over devices (one long request's keys split across GPUs; the cross-device
+ * form of the Update stage, Section 4.2.1).  Device k holds the keys [bounds[k], bounds[k+1]) of
+ * the request in its own paged cache and runs xy_attn_run on them as a decode request whose
+ * kv_len is the slice length minus one (the last key of the slice stands where the new token
+ * would: every key of the slice is visible to the single query row); that yields the slice's
+ * normalised O_k (bf16) and LSE_k.  After one all-gather of (O_k, LSE_k) into local memory every
+ * device merges:  LSE = ln sum_k exp(LSE_k),  O = sum_k exp(LSE_k - LSE) O_k.
+ *
+ * xy_attn_shard_context: HOST arithmetic only.  Splits total_tokens (cached + new, >= 1) into
+ *   num_shards contiguous slices whose starts are multiples of page_size; page counts differ by
+ *   at most one, the ragged tail (and so the position the new token is appended at) lies in the
+ *   last slice.  bounds HOST int64 [num_shards + 1], written.  XY_ERR_INVALID_ARG when the
+ *   context has fewer pages than shards.
+ * xy_attn_merge_shards: o_shards DEVICE bf16 [num_shards, rows, D] and lse_shards DEVICE fp32
+ *   [num_shards, rows] in LOCAL memory (the all-gather's output; rows = tokens x q heads);
+ *   o DEVICE bf16 [rows, D], lse DEVICE fp32 [rows], written.  A shard with LSE_k = -inf is
+ *   ignored and its O_k not read.  Needs no context; asynchronous on `stream`. */
+int xy_attn_shard_context(int64_t total_tokens, int32_t page_size, int32_t num_shards, int64_t* bounds);
+int xy_attn_merge_shards(const void* o_shards, const float* lse_shards, int32_t num_shards, int64_t rows,
+                         int32_t head_dim, void* o, float* lse, void* stream);
+
 /* Allocation-free decode attention.  The paper has no counterpart for this call: it exists
  * for callers that cannot allocate device memory where they need attention - a serving loop
  * whose memory pool is already handed out in full, a plugin that is given only a stream and

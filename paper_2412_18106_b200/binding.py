@@ -81,7 +81,7 @@ EXPORTS = (
     "xy_attn_last_launches", "xy_attn_last_error", "xy_attn_device_status",
     "xy_attn_set_timing", "xy_attn_get_timing", "xy_attn_debug_trace", "xy_attn_decode_static",
     "xy_attn_append_kv", "xy_attn_worker_times", "xy_attn_get_queue", "xy_attn_plan_cache",
-    "xy_attn_plan_shared",
+    "xy_attn_plan_shared", "xy_attn_shard_context", "xy_attn_merge_shards",
 )
 
 _lib = None
@@ -105,6 +105,8 @@ def load() -> ctypes.CDLL:
     L.xy_attn_run.argtypes = [vp, vp, i64, vp, vp, i64, i64, i64, i64, vp, i32, vp, ctypes.c_float,
                               vp, i64, vp, vp]
     L.xy_attn_merge.argtypes = [vp, vp, i32, i64, i32, vp, vp, vp]
+    L.xy_attn_merge_shards.argtypes = [vp, vp, i32, i64, i32, vp, vp, vp]
+    L.xy_attn_shard_context.argtypes = [i64, i32, i32, ctypes.POINTER(i64)]
     L.xy_attn_append_kv.argtypes = [vp, vp, i64, vp, vp, i64, i64, i64, i64, vp, i32, vp]
     L.xy_attn_debug_gather.argtypes = [vp, i32, i32, vp, vp, i64, i64, i64, vp, i32, vp, vp, vp]
     for name in ("xy_attn_get_tasks", "xy_attn_get_worker_offsets", "xy_attn_get_merge_units",
@@ -343,6 +345,32 @@ def xy_attn_merge(o_part: torch.Tensor, lse_part: torch.Tensor, o: torch.Tensor,
                          lse.data_ptr(), _stream_ptr(stream))
     if rc != XY_OK:
         raise XYAttnError(rc, "xy_attn_merge failed")
+
+
+def xy_attn_shard_context(total_tokens: int, page_size: int, num_shards: int) -> np.ndarray:
+    """Page-aligned contiguous slices of a context for num_shards devices: int64 [num_shards + 1]."""
+    L = load()
+    bounds = (ctypes.c_int64 * (num_shards + 1))()
+    rc = L.xy_attn_shard_context(int(total_tokens), int(page_size), int(num_shards), bounds)
+    if rc != XY_OK:
+        raise XYAttnError(rc, "xy_attn_shard_context: %d tokens of page size %d do not split %d ways"
+                          % (total_tokens, page_size, num_shards))
+    return np.array(bounds[:], dtype=np.int64)
+
+
+def xy_attn_merge_shards(o_shards: torch.Tensor, lse_shards: torch.Tensor, o: torch.Tensor,
+                         lse: torch.Tensor, stream=None) -> None:
+    """Merge of per-device results: o_shards bf16 [S, rows, D], lse_shards fp32 [S, rows], both in
+    local device memory -> o bf16 [rows, D], lse fp32 [rows]."""
+    L = load()
+    assert o_shards.is_cuda and o_shards.dtype == torch.bfloat16 and o_shards.is_contiguous()
+    assert lse_shards.is_cuda and lse_shards.dtype == torch.float32 and lse_shards.is_contiguous()
+    S, rows, D = o_shards.shape
+    assert lse_shards.shape == (S, rows) and o.is_contiguous() and lse.is_contiguous()
+    rc = L.xy_attn_merge_shards(o_shards.data_ptr(), lse_shards.data_ptr(), S, rows, D, o.data_ptr(),
+                                lse.data_ptr(), _stream_ptr(stream))
+    if rc != XY_OK:
+        raise XYAttnError(rc, "xy_attn_merge_shards failed")
 
 
 XY_ATTN_STATIC_MAX_ROWS = 8192

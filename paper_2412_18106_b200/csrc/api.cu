@@ -423,6 +423,33 @@ int xy_attn_merge(const float* o_part, const float* lse_part, int32_t num_splits
   return e == cudaSuccess ? XY_OK : XY_ERR_CUDA;
 }
 
+int xy_attn_merge_shards(const void* o_shards, const float* lse_shards, int32_t num_shards, int64_t rows,
+                         int32_t head_dim, void* o, float* lse, void* stream) {
+  if (head_dim != kHeadDim) return XY_ERR_UNSUPPORTED;
+  if (num_shards < 1 || rows < 0) return XY_ERR_INVALID_ARG;
+  if (rows == 0) return XY_OK;
+  if (!o_shards || !lse_shards || !o || !lse) return XY_ERR_INVALID_ARG;
+  cudaError_t e = launch_merge_shards(static_cast<const uint16_t*>(o_shards), lse_shards, num_shards, rows,
+                                      static_cast<uint16_t*>(o), lse, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? XY_OK : XY_ERR_CUDA;
+}
+
+int xy_attn_shard_context(int64_t total_tokens, int32_t page_size, int32_t num_shards, int64_t* bounds) {
+  if (bounds == nullptr || num_shards < 1 || total_tokens < 1 || page_size < 1) return XY_ERR_INVALID_ARG;
+  const int64_t pages = (total_tokens + page_size - 1) / page_size;
+  if (pages < num_shards) return XY_ERR_INVALID_ARG;  // every shard must hold at least one token
+  // pages dealt as evenly as whole pages allow; the earlier shards take the extra ones so that
+  // the last shard, which holds the ragged tail and receives the appends, is never the largest
+  const int64_t base = pages / num_shards, extra = pages % num_shards;
+  int64_t page = 0;
+  for (int32_t k = 0; k < num_shards; ++k) {
+    bounds[k] = page * page_size;
+    page += base + (k < extra ? 1 : 0);
+  }
+  bounds[num_shards] = total_tokens;
+  return XY_OK;
+}
+
 int xy_attn_debug_gather(xy_attn_ctx* ctx, int32_t req, int32_t kv_head, const void* k_pool,
                          const void* v_pool, int64_t page_stride, int64_t head_stride,
                          int64_t token_stride, const int32_t* block_table,

@@ -192,6 +192,61 @@ __global__ void __launch_bounds__(128) merge_plain_kernel(const float* o_part, c
   if (lane == 0) lse_out[x] = lse;
 }
 
+// Merge of per-device results when the context of a request is sharded over devices: every
+// shard ran attention over its own slice of the keys and produced a normalised bf16 O_c and
+// LSE_c; the merge is the same Update formula (Section 4.2.1).  One warp per row; lane c holds
+// LSE_c when there are at most 32 shards; each lane owns four output columns.
+__global__ void __launch_bounds__(128) merge_shards_kernel(const uint16_t* o_shards, const float* lse_shards,
+                                                          int num_shards, int64_t rows, uint16_t* o,
+                                                          float* lse_out) {
+  const int lane = threadIdx.x & 31;
+  const int64_t x = static_cast<int64_t>(blockIdx.x) * 4 + (threadIdx.x >> 5);
+  if (x >= rows) return;
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  float lse;
+  auto add = [&](int c, float w) {
+    const uint2 v = *reinterpret_cast<const uint2*>(o_shards + (static_cast<int64_t>(c) * rows + x) * kHeadDim + lane * 4);
+    acc[0] += w * __uint_as_float(v.x << 16);
+    acc[1] += w * __uint_as_float(v.x & 0xffff0000u);
+    acc[2] += w * __uint_as_float(v.y << 16);
+    acc[3] += w * __uint_as_float(v.y & 0xffff0000u);
+  };
+  if (num_shards <= 32) {
+    const float lc = lane < num_shards ? lse_shards[static_cast<int64_t>(lane) * rows + x] : -INFINITY;
+    float mx = lc;
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, s));
+    const float e = lc != -INFINITY ? __expf(lc - mx) : 0.f;
+    float z = e;
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) z += __shfl_xor_sync(0xffffffffu, z, s);
+    lse = mx + logf(z);
+    const float w_mine = z > 0.f ? e / z : 0.f;
+    for (int c = 0; c < num_shards; ++c) {
+      const float w = __shfl_sync(0xffffffffu, w_mine, c);
+      if (w != 0.f) add(c, w);  // an empty shard (LSE_c = -inf) is not read
+    }
+  } else {
+    float mx = -INFINITY;
+    for (int c = 0; c < num_shards; ++c) mx = fmaxf(mx, lse_shards[static_cast<int64_t>(c) * rows + x]);
+    float z = 0.f;
+    for (int c = 0; c < num_shards; ++c) {
+      const float lc = lse_shards[static_cast<int64_t>(c) * rows + x];
+      if (lc != -INFINITY) z += __expf(lc - mx);
+    }
+    lse = mx + logf(z);
+    for (int c = 0; c < num_shards; ++c) {
+      const float lc = lse_shards[static_cast<int64_t>(c) * rows + x];
+      if (lc != -INFINITY) add(c, __expf(lc - lse));
+    }
+  }
+  uint2 packed;
+  packed.x = float_to_bf16_bits(acc[0]) | (static_cast<uint32_t>(float_to_bf16_bits(acc[1])) << 16);
+  packed.y = float_to_bf16_bits(acc[2]) | (static_cast<uint32_t>(float_to_bf16_bits(acc[3])) << 16);
+  *reinterpret_cast<uint2*>(o + x * kHeadDim + lane * 4) = packed;
+  if (lane == 0) lse_out[x] = lse;
+}
+
 // Step a5 in isolation: copy the rows a request sees, in logical order (Section 4.1.1).
 __global__ void gather_kernel(const uint16_t* k_pool, const uint16_t* v_pool, int64_t page_stride,
                               int64_t head_stride, int64_t token_stride, const int32_t* bt,
@@ -271,6 +326,14 @@ cudaError_t launch_merge_plain(const float* o_part, const float* lse_part, int n
   if (rows == 0) return cudaSuccess;
   const unsigned blocks = static_cast<unsigned>((rows + 3) / 4);
   merge_plain_kernel<<<blocks, 128, 0, s>>>(o_part, lse_part, num_splits, rows, o, lse);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_merge_shards(const uint16_t* o_shards, const float* lse_shards, int num_shards,
+                                int64_t rows, uint16_t* o, float* lse, cudaStream_t s) {
+  if (rows == 0) return cudaSuccess;
+  const unsigned blocks = static_cast<unsigned>((rows + 3) / 4);
+  merge_shards_kernel<<<blocks, 128, 0, s>>>(o_shards, lse_shards, num_shards, rows, o, lse);
   return cudaGetLastError();
 }
 

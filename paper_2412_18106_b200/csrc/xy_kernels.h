@@ -23,6 +23,8 @@ cudaError_t launch_meta(const RunArgs& a, int num_workers, int64_t num_pages, bo
 cudaError_t launch_merge_units(const MergeArgs& a, int num_units, int max_rows, cudaStream_t s);
 cudaError_t launch_merge_plain(const float* o_part, const float* lse_part, int num_splits,
                                int64_t rows, uint16_t* o, float* lse, cudaStream_t s);
+cudaError_t launch_merge_shards(const uint16_t* o_shards, const float* lse_shards, int num_shards,
+                                int64_t rows, uint16_t* o, float* lse, cudaStream_t s);
 cudaError_t launch_append_kv(const uint16_t* qkv, int64_t qkv_token_stride, uint16_t* k_pool, uint16_t* v_pool,
                              int64_t page_stride, int64_t head_stride, int64_t token_stride,
                              const int32_t* block_table, int bt_stride, const ReqInfo* reqs, int num_reqs,

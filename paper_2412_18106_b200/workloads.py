@@ -284,6 +284,26 @@ def custom(name: str, hq: int, hkv: int, page_size: int, requests, seed: int = 0
                     spare_frac=spare_frac, permute_pages=permute_pages)
 
 
+def context_shard(batch: Batch, bounds, k: int) -> Batch:
+    """Shard k of a decode batch whose contexts are split over devices.  `bounds[r]` holds the
+    slice starts of request r's kv_len + 1 tokens (page-aligned, one more entry than shards).  The
+    shard is a decode batch over the same pools: request r keeps the pages of its slice, and its
+    kv_len is the slice length minus one, so that the single query row sees the whole slice."""
+    assert np.all(batch.q_len == 1)
+    B = batch.page_size
+    lo = np.array([int(bd[k]) for bd in bounds], dtype=np.int64)
+    hi = np.array([int(bd[k + 1]) for bd in bounds], dtype=np.int64)
+    assert np.all(lo % B == 0) and np.all(hi > lo)
+    need = (hi - lo + B - 1) // B
+    bt = np.full((batch.num_requests, int(need.max())), -1, dtype=np.int32)
+    for r in range(batch.num_requests):
+        p0 = int(lo[r]) // B
+        bt[r, : int(need[r])] = batch.block_table[r, p0 : p0 + int(need[r])]
+    return Batch("%s_shard%d" % (batch.name, k), batch.num_q_heads, batch.num_kv_heads, batch.head_dim, B,
+                 batch.q_len.copy(), (hi - lo - 1).astype(np.int32), batch.mask_kind.copy(),
+                 batch.parent_off.copy(), batch.parents.copy(), bt, batch.num_pages, batch.seed)
+
+
 def _randn_bf16(shape, gen: torch.Generator, chunk_elems: int = 1 << 26) -> torch.Tensor:
     """N(0,1) drawn in fp32 and rounded to bf16, produced in chunks to bound memory."""
     total = int(np.prod(shape)) if len(shape) else 1
