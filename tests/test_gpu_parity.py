@@ -260,3 +260,20 @@ def test_many_task_kind_transitions_per_worker(workers):
             first = (O, LSE)
         assert np.array_equal(O, first[0]) and np.array_equal(LSE, first[1])
     ctx.close()
+
+
+def test_maximum_sizes_one_million_token_context_and_largest_tree():
+    """The largest shapes the path is meant for: a decode and a 64-node verify tree (the largest
+    tree a context accepts by default) on contexts of about a million and 300 thousand tokens,
+    next to a fresh one-token prefill; the long rows are split over every worker and merged."""
+    rng = np.random.default_rng(99)
+    reqs = [(1, 1_000_003, 0, None), (64, 300_001, 1, W.random_tree(rng, 64, 8)), (1, 0, 0, None)]
+    b = W.custom("max_sizes", 8, 2, 128, reqs, seed=99, spare_frac=0.01)
+    ctx = H.make_ctx(b)
+    info = ctx.plan_batch(b)
+    assert info.num_merge_units > 0
+    t = W.make_tensors(b)
+    O, LSE = H.run_gpu(b, t, ctx=ctx)
+    ctx.close()
+    O_ref, LSE_ref = oracle.attention(b, t, H.SCALE)
+    H.check_against_oracle(O, LSE, O_ref, LSE_ref, "max_sizes")
