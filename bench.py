@@ -417,6 +417,50 @@ def measure_shared_prefix(kernel, dev, peaks, steps=20):
     return out
 
 
+def measure_long_decode(kernel, dev, peaks, steps=20):
+    """Long-context decode: 4 requests with 128k - 512k cached tokens, 32/8 heads, page 128.  Every
+    (request, kv head) row is cut into up to 32 key ranges handled by different workers and the
+    partials are merged by the second kernel.  The pools are random and generated on the device
+    (contents do not matter for timing); the roofline counts every cached K/V byte once."""
+    import torch
+
+    from paper_2412_18106_b200 import binding as xb
+    from paper_2412_18106_b200 import workloads as W
+    batch = W.long_context_decode(seed=0)
+    g = torch.Generator(device=dev).manual_seed(0)
+    shape = (batch.num_pages, batch.num_kv_heads, batch.page_size, batch.head_dim)
+    k_pool = torch.empty(shape, dtype=torch.bfloat16, device=dev)
+    v_pool = torch.empty(shape, dtype=torch.bfloat16, device=dev)
+    step_pages = 2048
+    for pool in (k_pool, v_pool):
+        for p0 in range(0, batch.num_pages, step_pages):
+            n = min(step_pages, batch.num_pages - p0)
+            pool[p0: p0 + n] = torch.randn((n,) + shape[1:], device=dev, generator=g).to(torch.bfloat16)
+    q = torch.randn((batch.total_q, batch.num_q_heads, batch.head_dim), device=dev, generator=g).to(torch.bfloat16)
+    bt = torch.from_numpy(np.where(batch.block_table < 0, 0, batch.block_table).astype(np.int32)).to(dev)
+    o = torch.empty((batch.total_q, batch.num_q_heads, batch.head_dim), dtype=torch.bfloat16, device=dev)
+    lse = torch.empty((batch.total_q, batch.num_q_heads), dtype=torch.float32, device=dev)
+    ctx = xb.XYAttn(batch.num_q_heads, batch.num_kv_heads, batch.page_size, device=dev.index, kernel=kernel,
+                    max_requests=256, max_q_tokens=1 << 15, max_pages_per_req=batch.block_table.shape[1])
+    info = ctx.plan_batch(batch)
+    for _ in range(3):
+        ctx.run(q, k_pool, v_pool, bt, SCALE, o, lse)
+    torch.cuda.synchronize()
+    ctx.set_timing(True)
+    for _ in range(steps):
+        ctx.run(q, k_pool, v_pool, bt, SCALE, o, lse)
+    attn_ms, merge_ms, runs = ctx.get_timing()
+    assert ctx.device_status() == 0
+    ctx.close()
+    assert torch.isfinite(o.float()).all() and torch.isfinite(lse).all()
+    alg = float(W.algorithmic_bytes(batch))
+    k_ms, m_ms = attn_ms / runs, merge_ms / runs
+    return {"requests": batch.num_requests, "kv_tokens": [int(x) for x in batch.kv_len], "tasks": info.num_tasks,
+            "merge_units": info.num_merge_units, "kernel_ms": k_ms, "merge_ms": m_ms,
+            "kv_gbs": float(info.kv_bytes) / (k_ms * 1e-3) / 1e9, "bound": "hbm",
+            "roofline_frac_measured": alg / (peaks["hbm_gbs"] * 1e9) / (k_ms * 1e-3), "steps": steps}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -671,6 +715,11 @@ def main():
             others["decode_shared_prefix"] = measure_shared_prefix(kernel, dev, peaks)
         except Exception as e:
             others["decode_shared_prefix"] = {"error": repr(e)}
+        try:
+            torch.cuda.empty_cache()
+            others["long_context_decode"] = measure_long_decode(kernel, dev, peaks)
+        except Exception as e:
+            others["long_context_decode"] = {"error": repr(e)}
         try:
             torch.cuda.empty_cache()
             others["smoothgemm"] = measure_gemm(dev, peaks)

@@ -272,6 +272,16 @@ def shared_prefix_decode(seed: int = 0, num_groups: int = 4, members: int = 32, 
     return b, groups
 
 
+def long_context_decode(seed: int = 0, num_requests: int = 4, kv_lo: int = 131072, kv_hi: int = 524288,
+                        hq: int = 32, hkv: int = 8, page_size: int = 128) -> Batch:
+    """Few decode requests on very long contexts (log-uniform lengths): every (request, kv head)
+    row is split over many workers and merged (the split-KV path)."""
+    rng = np.random.default_rng(seed)
+    kv = [_log_uniform_int(rng, kv_lo, kv_hi) for _ in range(num_requests)]
+    return assemble("long_context_decode", hq, hkv, page_size, [1] * num_requests, kv,
+                    [MASK_CAUSAL] * num_requests, [None] * num_requests, rng, seed, spare_frac=0.01)
+
+
 def custom(name: str, hq: int, hkv: int, page_size: int, requests, seed: int = 0,
            permute_pages: bool = True, spare_frac: float = 0.10) -> Batch:
     """`requests` is a list of (q_len, kv_len, kind, parents-or-None) tuples."""
