@@ -934,6 +934,9 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
         const bool exists = X * 128 < tv.rows;
         const bool valid = x < tv.rows;
         if (!exists) continue;
+        // A warp whose 32 rows all lie past the tile's last row has nothing to compute: it only
+        // keeps step with the hand-offs (its rows of Q are zero, so are its rows of S, P and O).
+        const bool warp_active = X * 128 + (warp & 3) * 32 < tv.rows;
         const int nX = ds.n[X];
         const int i_row = tv.t.tok0 + min(x, tv.rows - 1) / G;
         if (nX == 0) {  // a KV split that lies wholly above this sub-tile's causal frontier
@@ -987,6 +990,14 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
             dead = true;
           }
           ph_s ^= 1u;
+          if (!warp_active) {
+            __syncwarp();
+            if (lane == 0) {
+              mbar_arrive(smem_u32(&ub->p_full[X][0]));
+              mbar_arrive(smem_u32(&ub->p_full[X][1]));
+            }
+            continue;
+          }
           tc_fence_after();
           uint32_t sr[128];
           tmem_ld_32x32b_x32(t_s, &sr[0]);
@@ -1123,7 +1134,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
           // (its MMAs have completed; 16-byte chunks XOR-swizzled by row so that neither side has
           // bank conflicts) and leave as row-contiguous 256-byte stores, two rows per instruction.
           uint8_t* stage = gen_base + X * kTileBytes;
-          {
+          if (warp_active) {
             uint32_t orow[128];  // the whole row with one wait: four loads in flight together
             tmem_ld_32x32b_x32(t_o, &orow[0]);
             tmem_ld_32x32b_x32(t_o + 32, &orow[32]);
@@ -1141,7 +1152,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
             }
           }
           __syncwarp();
-          {
+          if (warp_active) {  // a warp stores only rows it staged itself
             const int ch = lane & 15;
             int rr = (warp & 3) * 32 + (lane >> 4);  // row of the sub-tile this lane stores first
             const int xs = X * 128 + rr;
@@ -1165,7 +1176,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
             }
           }
           named_bar_sync(2 + X, 128);  // staging reads done before the next task's Q lands here
-        } else {
+        } else if (warp_active) {
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
             uint32_t orow[32];
