@@ -170,6 +170,22 @@ int xy_attn_plan_shared(xy_attn_ctx* ctx, const xy_attn_request* reqs /*HOST*/, 
                         const xy_attn_prefix_group* groups /*HOST*/, int32_t num_groups, void* stream,
                         xy_attn_plan_info* info /*HOST, nullable*/);
 
+/* Finds shared-prefix groups from the block tables (what a radix-tree prefix cache leaves behind:
+ * requests that matched the same cached prefix point at the same pages, Section 4.1.1).  HOST
+ * arithmetic only; needs no context.  Scans the requests in order; a group is a maximal run of
+ * consecutive decode requests (q_len 1, XY_MASK_CAUSAL) that each share at least
+ * max(min_prefix_tokens, 128) leading tokens with the run's first request — same page ids in
+ * block_table (HOST int32 [num_reqs, block_table_stride], entries < 0 never match), counted in
+ * whole 128-token tiles inside both histories; the group's prefix_tokens is the smallest such
+ * overlap.  Runs shorter than min_members (>= 2) are left ungrouped.  Every group written
+ * satisfies the rules of xy_attn_prefix_group.  groups HOST [capacity], *num_groups written.
+ * Returns XY_OK, XY_ERR_INVALID_ARG (null pointer, bad page_size or min_members) or
+ * XY_ERR_CAPACITY (more groups than capacity; the first `capacity` are written). */
+int xy_attn_find_prefix_groups(const xy_attn_request* reqs /*HOST*/, int32_t num_reqs,
+                               const int32_t* block_table /*HOST*/, int32_t block_table_stride,
+                               int32_t page_size, int32_t min_members, int32_t min_prefix_tokens,
+                               xy_attn_prefix_group* groups /*HOST*/, int32_t capacity, int32_t* num_groups);
+
 /* Task-Table cache (Section 3.3: the Task-Table is what the kernels consume; Section 3.3.2 keeps
  * pre-built Task-Tables for recurring shapes).  xy_attn_plan keeps the Task-Tables of the last
  * `capacity` distinct decompositions (default 8).  A plan whose decomposition — per request, kv

@@ -82,6 +82,7 @@ EXPORTS = (
     "xy_attn_set_timing", "xy_attn_get_timing", "xy_attn_debug_trace", "xy_attn_decode_static",
     "xy_attn_append_kv", "xy_attn_worker_times", "xy_attn_get_queue", "xy_attn_plan_cache",
     "xy_attn_plan_shared", "xy_attn_shard_context", "xy_attn_merge_shards",
+    "xy_attn_find_prefix_groups",
 )
 
 _lib = None
@@ -106,6 +107,7 @@ def load() -> ctypes.CDLL:
                               vp, i64, vp, vp]
     L.xy_attn_merge.argtypes = [vp, vp, i32, i64, i32, vp, vp, vp]
     L.xy_attn_merge_shards.argtypes = [vp, vp, i32, i64, i32, vp, vp, vp]
+    L.xy_attn_find_prefix_groups.argtypes = [vp, i32, vp, i32, i32, i32, i32, vp, i32, ctypes.POINTER(i32)]
     L.xy_attn_shard_context.argtypes = [i64, i32, i32, ctypes.POINTER(i64)]
     L.xy_attn_append_kv.argtypes = [vp, vp, i64, vp, vp, i64, i64, i64, i64, vp, i32, vp]
     L.xy_attn_debug_gather.argtypes = [vp, i32, i32, vp, vp, i64, i64, i64, vp, i32, vp, vp, vp]
@@ -216,6 +218,12 @@ class XYAttn:
         return self.info
 
     def plan_batch(self, batch, stream=None, groups=None) -> xy_attn_plan_info:
+        """`groups`: None, a list of (first_req, num_reqs, prefix_tokens), or "auto" to read the
+        shared-prefix groups off the batch's block table."""
+        if isinstance(groups, str):
+            assert groups == "auto"
+            groups = xy_attn_find_prefix_groups(batch.q_len, batch.kv_len, batch.mask_kind, batch.block_table,
+                                                batch.page_size)
         if groups:
             return self.plan_shared(batch.q_len, batch.kv_len, batch.mask_kind, batch.parent_off, batch.parents,
                                     groups, stream)
@@ -345,6 +353,26 @@ def xy_attn_merge(o_part: torch.Tensor, lse_part: torch.Tensor, o: torch.Tensor,
                          lse.data_ptr(), _stream_ptr(stream))
     if rc != XY_OK:
         raise XYAttnError(rc, "xy_attn_merge failed")
+
+
+def xy_attn_find_prefix_groups(q_len, kv_len, mask_kind, block_table: np.ndarray, page_size: int,
+                               min_members: int = 2, min_prefix_tokens: int = 128):
+    """Shared-prefix groups read off the block tables: list of (first_req, num_reqs, prefix_tokens)."""
+    L = load()
+    R = len(q_len)
+    reqs = (xy_attn_request * max(R, 1))()
+    for r in range(R):
+        reqs[r] = xy_attn_request(int(q_len[r]), int(kv_len[r]), int(mask_kind[r]), -1)
+    bt = np.ascontiguousarray(block_table, dtype=np.int32)
+    assert bt.ndim == 2 and bt.shape[0] == R
+    gs = (xy_attn_prefix_group * max(R // 2, 1))()
+    n = ctypes.c_int32(0)
+    rc = L.xy_attn_find_prefix_groups(ctypes.cast(reqs, ctypes.c_void_p), R, ctypes.c_void_p(bt.ctypes.data),
+                                      bt.shape[1], int(page_size), int(min_members), int(min_prefix_tokens),
+                                      ctypes.cast(gs, ctypes.c_void_p), max(R // 2, 1), ctypes.byref(n))
+    if rc != XY_OK:
+        raise XYAttnError(rc, "xy_attn_find_prefix_groups failed")
+    return [(gs[k].first_req, gs[k].num_reqs, gs[k].prefix_tokens) for k in range(n.value)]
 
 
 def xy_attn_shard_context(total_tokens: int, page_size: int, num_shards: int) -> np.ndarray:

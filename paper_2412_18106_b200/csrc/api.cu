@@ -423,6 +423,55 @@ int xy_attn_merge(const float* o_part, const float* lse_part, int32_t num_splits
   return e == cudaSuccess ? XY_OK : XY_ERR_CUDA;
 }
 
+int xy_attn_find_prefix_groups(const xy_attn_request* reqs, int32_t num_reqs, const int32_t* block_table,
+                               int32_t block_table_stride, int32_t page_size, int32_t min_members,
+                               int32_t min_prefix_tokens, xy_attn_prefix_group* groups, int32_t capacity,
+                               int32_t* num_groups) {
+  if (num_groups == nullptr) return XY_ERR_INVALID_ARG;
+  *num_groups = 0;
+  if (num_reqs < 0 || capacity < 0 || (num_reqs > 0 && (reqs == nullptr || block_table == nullptr)) ||
+      (capacity > 0 && groups == nullptr) || page_size < 1 || page_size > kKeyTile ||
+      (page_size & (page_size - 1)) != 0 || block_table_stride < 0 || min_members < 2)
+    return XY_ERR_INVALID_ARG;
+  const int32_t floor_tokens = std::max(min_prefix_tokens, kKeyTile);
+  auto is_decode = [&](int32_t r) { return reqs[r].q_len == 1 && reqs[r].mask_kind == XY_MASK_CAUSAL; };
+  // tokens of the longest common run of leading page ids of requests a and b, counted in whole
+  // 128-token tiles that lie inside both histories
+  auto common_tokens = [&](int32_t a, int32_t b, int32_t limit) -> int32_t {
+    const int32_t tokens = std::min(std::min(reqs[a].kv_len, reqs[b].kv_len), limit) / kKeyTile * kKeyTile;
+    const int32_t pages = std::min(tokens / page_size, block_table_stride);
+    const int32_t* ra = block_table + static_cast<int64_t>(a) * block_table_stride;
+    const int32_t* rb = block_table + static_cast<int64_t>(b) * block_table_stride;
+    int32_t p = 0;
+    while (p < pages && ra[p] == rb[p] && ra[p] >= 0) ++p;
+    return static_cast<int32_t>(static_cast<int64_t>(p) * page_size / kKeyTile * kKeyTile);
+  };
+  int32_t r = 0;
+  while (r < num_reqs) {
+    if (!is_decode(r) || reqs[r].kv_len < floor_tokens) {
+      ++r;
+      continue;
+    }
+    int32_t prefix = reqs[r].kv_len / kKeyTile * kKeyTile;
+    int32_t end = r + 1;
+    while (end < num_reqs && is_decode(end)) {
+      const int32_t c = common_tokens(r, end, prefix);
+      if (c < floor_tokens) break;
+      prefix = c;
+      ++end;
+    }
+    if (end - r >= min_members) {
+      if (*num_groups >= capacity) return XY_ERR_CAPACITY;
+      groups[*num_groups] = xy_attn_prefix_group{r, end - r, prefix};
+      ++*num_groups;
+      r = end;
+    } else {
+      ++r;
+    }
+  }
+  return XY_OK;
+}
+
 int xy_attn_merge_shards(const void* o_shards, const float* lse_shards, int32_t num_shards, int64_t rows,
                          int32_t head_dim, void* o, float* lse, void* stream) {
   if (head_dim != kHeadDim) return XY_ERR_UNSUPPORTED;

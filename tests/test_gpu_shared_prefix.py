@@ -92,3 +92,19 @@ def test_random_groups(seed):
     O2, LSE2 = H.run_gpu(b, t, ctx=ctx)
     assert np.array_equal(O, O2) and np.array_equal(LSE, LSE2)
     ctx.close()
+
+
+def test_groups_found_from_the_block_table():
+    """groups="auto": the groups are read off the block table, the plan uses them, the result is
+    the oracle's."""
+    b, groups = W.shared_prefix_decode(seed=21, num_groups=3, members=24, prefix=1024, suffix_hi=400, hq=16, hkv=4,
+                                       page_size=64)
+    t = W.make_tensors(b)
+    ctx = H.make_ctx(b, max_requests=512)
+    plain_tasks = ctx.plan_batch(b).num_tasks
+    info = ctx.plan_batch(b, groups="auto")
+    assert info.num_tasks != plain_tasks and info.num_merge_units >= 3 * 24
+    O, LSE = H.run_gpu(b, t, ctx=ctx)
+    O_ref, LSE_ref = oracle.attention(b, t, H.SCALE)
+    H.check_against_oracle(O, LSE, O_ref, LSE_ref, "auto groups")
+    ctx.close()
