@@ -1076,14 +1076,14 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
             const float alpha = (m_cand == -INFINITY) ? 1.f : ex2(m_ref - m_cand);
             l *= alpha;
             m_ref = m_cand;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-              uint32_t orow[32];
-              tmem_ld_32x32b_x32(t_o + c * 32, orow);
+#pragma unroll 1
+            for (int c = 0; c < 8; ++c) {  // rare path: small chunks, the 128 scores stay live
+              uint32_t orow[16];
+              tmem_ld_32x32b_x16(t_o + c * 16, orow);
               tmem_wait_ld();
 #pragma unroll
-              for (int k = 0; k < 32; ++k) orow[k] = __float_as_uint(__uint_as_float(orow[k]) * alpha);
-              tmem_st_32x32b_x32(t_o + c * 32, orow);
+              for (int k = 0; k < 16; ++k) orow[k] = __float_as_uint(__uint_as_float(orow[k]) * alpha);
+              tmem_st_32x32b_x16(t_o + c * 16, orow);
             }
           }
           tr(24);
