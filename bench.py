@@ -190,7 +190,7 @@ def run_reference(args):
 
 # DRAM bytes (read + write) of one launch of the attention meta-kernel, from the ncu captures
 # summarised under profiles/ (same workload, seed 0); None where no capture was taken.
-NCU_TRAFFIC_BYTES = {"full_mix": 6.04e9, "splitfuse_mix": 1.670e9, "verify_trees": 2.348e9, "decode_only": 0.593e9}
+NCU_TRAFFIC_BYTES = {"full_mix": 6.00e9, "splitfuse_mix": 1.667e9, "verify_trees": 2.507e9, "decode_only": 0.594e9}
 
 
 def measure_other(name, kernel, dev, peaks, steps=20, warmup=3):
