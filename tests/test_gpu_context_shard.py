@@ -85,3 +85,44 @@ def test_merge_shards_kernel_matches_oracle_merge():
         assert np.isfinite(got).all()
         assert np.abs(got - O_ref).max() <= 2e-2
         assert np.all(np.abs(lse.cpu().numpy() - L_ref) <= 1e-3 * np.maximum(1, np.abs(L_ref)))
+
+
+_NCCL_ONE_RANK = r"""
+import os, sys
+import numpy as np
+import torch
+import torch.distributed as dist
+sys.path.insert(0, sys.argv[1])
+os.environ["NCCL_NVLS_ENABLE"] = "0"
+torch.cuda.set_device(0)
+dist.init_process_group("nccl", init_method="tcp://127.0.0.1:%s" % sys.argv[2], rank=0, world_size=1,
+                        device_id=torch.device("cuda", 0))
+from paper_2412_18106_b200 import context_shard as cs
+g = torch.Generator(device="cuda").manual_seed(5)
+o_local = torch.randn((7, 8, 128), device="cuda", generator=g).to(torch.bfloat16)
+l_local = torch.randn((7, 8), device="cuda", generator=g)
+o, lse = cs.gather_and_merge(o_local, l_local)
+torch.cuda.synchronize()
+# one rank: weight 1 for its only shard, so the merge returns the bits it was given
+assert torch.equal(o.view(torch.int16), o_local.view(torch.int16))
+assert torch.allclose(lse, l_local, rtol=0, atol=1e-6)
+dist.destroy_process_group()
+print("one-rank nccl ok")
+"""
+
+
+def test_gather_and_merge_over_nccl_with_one_rank():
+    """The CUDA side of the exchange (NCCL all-gather into local memory, then the merge kernel) with
+    a process group of one rank; the two-rank exchange itself runs on CPU ranks (gloo)."""
+    import os
+    import socket
+    import subprocess
+    import sys
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, "-c", _NCCL_ONE_RANK, root, str(port)], capture_output=True, text=True,
+                       timeout=300)
+    assert r.returncode == 0 and "one-rank nccl ok" in r.stdout, r.stdout[-2000:] + r.stderr[-2000:]
