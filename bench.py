@@ -658,9 +658,10 @@ def main():
                            "(copies of neighbouring steps overlap the kernels); the cached history is "
                            "device-resident state; CUDA events around all steps, the last one after a device synchronize"}
 
+    if world > 1:  # every collective is behind us: all ranks leave the group together
+        dist.barrier()
+        dist.destroy_process_group()
     if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
         return 0
 
     peaks = measured_peaks()
@@ -686,7 +687,7 @@ def main():
     roof["frac_of_nominal_roofline"] = roof["t_roof_us_nominal"] / (attn_ms_avg * 1e3)
 
     cpu = None
-    if not args.no_cpu_baseline:
+    if not args.no_cpu_baseline and world == 1:  # the oracle is timed at N = 1 only
         r = time_oracle_sample(batch, tensors, 12.0)
         cpu = {"value": r["tflops"], "unit": "TFLOP/s", "cores": r["cores"], "kind": "oracle",
                "sample": "%d random output rows (request, head, token) of the workload, %.1f s; %s"
@@ -742,8 +743,6 @@ def main():
         "other_workloads": others,
     }
     print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
     return 0
 
 
