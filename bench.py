@@ -190,7 +190,8 @@ def run_reference(args):
 
 # DRAM bytes (read + write) of one launch of the attention meta-kernel, from the ncu captures
 # summarised under profiles/ (same workload, seed 0); None where no capture was taken.
-NCU_TRAFFIC_BYTES = {"full_mix": 6.00e9, "splitfuse_mix": 1.667e9, "verify_trees": 2.507e9, "decode_only": 0.594e9}
+NCU_TRAFFIC_BYTES = {"full_mix": 6.00e9, "splitfuse_mix": 1.667e9, "verify_trees": 2.507e9, "decode_only": 0.594e9,
+                     "long_context_decode": 3.202e9}
 
 
 def measure_other(name, kernel, dev, peaks, steps=20, warmup=3):
@@ -469,7 +470,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="full_mix",
                     choices=["decode_only", "splitfuse_mix", "verify_trees", "full_mix", "tiny_hybrid",
-                             "prefill_prefix"])
+                             "prefill_prefix", "long_context_decode"])
     ap.add_argument("--kernel", default="auto", choices=["auto", "reference", "mma"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")

@@ -282,6 +282,9 @@ def long_context_decode(seed: int = 0, num_requests: int = 4, kv_lo: int = 13107
                     [MASK_CAUSAL] * num_requests, [None] * num_requests, rng, seed, spare_frac=0.01)
 
 
+CONFIGS["long_context_decode"] = long_context_decode
+
+
 def custom(name: str, hq: int, hkv: int, page_size: int, requests, seed: int = 0,
            permute_pages: bool = True, spare_frac: float = 0.10) -> Batch:
     """`requests` is a list of (q_len, kv_len, kind, parents-or-None) tuples."""

@@ -28,7 +28,7 @@ def sample_rows(batch, rng, n_random):
     return np.array(req, np.int32), np.array(head, np.int32), np.array(row, np.int32)
 
 
-@pytest.mark.parametrize("name", ["decode_only", "splitfuse_mix", "verify_trees", "full_mix"])
+@pytest.mark.parametrize("name", ["decode_only", "splitfuse_mix", "verify_trees", "full_mix", "long_context_decode"])
 def test_full_size_sampled_parity(name):
     batch = W.CONFIGS[name](seed=0)
     tensors = W.make_tensors(batch)
