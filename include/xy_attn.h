@@ -82,7 +82,8 @@ typedef struct {
   int32_t kernel;            /* XY_KERNEL_* */
   int32_t plan_mode;         /* XY_PLAN_* */
   int32_t tile_tokens;       /* XY_PLAN_PAPER only: tileSize in tokens (0 = 128 / (Hq/Hkv)) */
-  int32_t max_splits;        /* upper bound on KV splits of one tile unit (0 = 32) */
+  int32_t max_splits;        /* upper bound on KV splits of one tile unit (0 = 32, or up to 128 when so few
+                              * streaming units exist that 32 splits each would leave workers idle) */
   int64_t workspace_bytes;   /* split-KV workspace (fp32 partial O and LSE); 0 = 256 MiB */
 } xy_attn_config;
 

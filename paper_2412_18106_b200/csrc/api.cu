@@ -341,10 +341,12 @@ int xy_attn_run(xy_attn_ctx* ctx, const void* q, int64_t q_token_stride, const v
     m.lse = lse;
     m.num_q_heads = cfg.num_q_heads;
     m.num_kv_heads = cfg.num_kv_heads;
-    int max_rows = 1;
-    for (const xy_attn_merge_unit& mu : p.merges)
+    int max_rows = 1, max_parts = 1;
+    for (const xy_attn_merge_unit& mu : p.merges) {
       max_rows = std::max(max_rows, mu.ntok * (cfg.num_q_heads / cfg.num_kv_heads));
-    XY_CUDA(ctx, launch_merge_units(m, static_cast<int>(p.merges.size()), max_rows, s));
+      max_parts = std::max(max_parts, mu.nsplit + mu.nsplit1);
+    }
+    XY_CUDA(ctx, launch_merge_units(m, static_cast<int>(p.merges.size()), max_rows, max_parts, s));
     ctx->last_launches += 1;
   }
   if (timed) {

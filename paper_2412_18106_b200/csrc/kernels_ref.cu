@@ -90,10 +90,15 @@ __global__ void __launch_bounds__(128) ref_attention_kernel(RunArgs a) {
 }
 
 // Cross-task form of the Update stage (Section 4.2.1): combine the partials of every tile
-// unit whose KV range was split.  One warp per packed row (a unit has at most 256): lane c holds
-// LSE_c of split c, the maximum and the sum go through warp shuffles, and the weights
-// exp(LSE_c - LSE) are broadcast while the lanes accumulate four output columns each.
+// unit whose KV range was split.  One warp per packed row (a unit has at most 256): lane l holds
+// LSE_c of splits l, l + 32, ..., the maximum and the sum go through warp shuffles, and the
+// weights exp(LSE_c - LSE) are broadcast while the lanes accumulate four output columns each,
+// eight partial rows per round so that their loads are in flight together.
 constexpr int kMergeBlocksPerUnit = 64;  // x 4 warps = 256 rows
+constexpr int kMergeLaneParts = 8;     // partials per lane on the shuffle path: up to 256 per row
+// kWide: some unit has more than 32 partials per row (a single long context cut for every
+// worker); that path holds eight partial rows in registers and is kept out of the common kernel.
+template <bool kWide>
 __global__ void __launch_bounds__(128) merge_units_kernel(MergeArgs a) {
   const xy_attn_merge_unit u = a.units[blockIdx.x];
   const int G = a.num_q_heads / a.num_kv_heads;
@@ -112,6 +117,7 @@ __global__ void __launch_bounds__(128) merge_units_kernel(MergeArgs a) {
                           : static_cast<int64_t>(u.part1) + static_cast<int64_t>(c - u.nsplit) * u.stride1 + x;
     };
     if (nparts <= 32) {
+      // the common case: lane c holds LSE_c; the partial rows are read four at a time
       const float lc = lane < nparts ? a.lse_part[part_row(lane)] : -INFINITY;
       float mx = lc;
 #pragma unroll
@@ -122,14 +128,73 @@ __global__ void __launch_bounds__(128) merge_units_kernel(MergeArgs a) {
       for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
       lse = mx + logf(z);
       const float w_mine = z > 0.f ? e / z : 0.f;
-      for (int c = 0; c < nparts; ++c) {
-        const float w = __shfl_sync(0xffffffffu, w_mine, c);
-        if (w == 0.f) continue;  // empty split (LSE_c = -inf): its O_c is not read
-        const float4 v = *reinterpret_cast<const float4*>(a.o_part + part_row(c) * kHeadDim + lane * 4);
-        acc.x += w * v.x;
-        acc.y += w * v.y;
-        acc.z += w * v.z;
-        acc.w += w * v.w;
+      for (int c0 = 0; c0 < nparts; c0 += 4) {
+        float w[4];
+        float4 v[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const int c = c0 + q;
+          w[q] = __shfl_sync(0xffffffffu, w_mine, c & 31);
+          if (c >= nparts) w[q] = 0.f;
+          // an empty split (LSE_c = -inf, weight 0) is not read
+          v[q] = w[q] != 0.f ? *reinterpret_cast<const float4*>(a.o_part + part_row(c) * kHeadDim + lane * 4)
+                             : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          acc.x += w[q] * v[q].x;
+          acc.y += w[q] * v[q].y;
+          acc.z += w[q] * v[q].z;
+          acc.w += w[q] * v[q].w;
+        }
+      }
+    } else if (kWide && nparts <= 32 * kMergeLaneParts) {
+      // lane l holds LSE_c of parts l, l + 32, ...; maximum and sum go through shuffles; the
+      // partial rows are then read eight at a time (independent loads in flight together)
+      float lc[kMergeLaneParts], mx = -INFINITY;
+#pragma unroll
+      for (int k = 0; k < kMergeLaneParts; ++k) {
+        const int c = k * 32 + lane;
+        lc[k] = c < nparts ? a.lse_part[part_row(c)] : -INFINITY;
+        mx = fmaxf(mx, lc[k]);
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      float z = 0.f;
+#pragma unroll
+      for (int k = 0; k < kMergeLaneParts; ++k) {
+        lc[k] = lc[k] != -INFINITY ? __expf(lc[k] - mx) : 0.f;
+        z += lc[k];
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
+      lse = mx + logf(z);
+      const float rz = z > 0.f ? 1.f / z : 0.f;
+#pragma unroll
+      for (int k = 0; k < kMergeLaneParts; ++k) {
+        if (k * 32 >= nparts) break;
+        const float w_mine = lc[k] * rz;
+        for (int j = 0; j < 32 && k * 32 + j < nparts; j += 8) {
+          float w[8];
+          float4 v[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            const int c = k * 32 + j + e;
+            w[e] = __shfl_sync(0xffffffffu, w_mine, (j + e) & 31);
+            // an empty split (LSE_c = -inf, weight 0) is not read
+            v[e] = (c < nparts && w[e] != 0.f)
+                       ? *reinterpret_cast<const float4*>(a.o_part + part_row(c) * kHeadDim + lane * 4)
+                       : make_float4(0.f, 0.f, 0.f, 0.f);
+            if (c >= nparts) w[e] = 0.f;
+          }
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            acc.x += w[e] * v[e].x;
+            acc.y += w[e] * v[e].y;
+            acc.z += w[e] * v[e].z;
+            acc.w += w[e] * v[e].w;
+          }
+        }
       }
     } else {
       float mx = -INFINITY;
@@ -312,12 +377,15 @@ cudaError_t launch_reference(const RunArgs& a, int num_workers, cudaStream_t s) 
   return cudaGetLastError();
 }
 
-cudaError_t launch_merge_units(const MergeArgs& a, int num_units, int max_rows, cudaStream_t s) {
+cudaError_t launch_merge_units(const MergeArgs& a, int num_units, int max_rows, int max_parts, cudaStream_t s) {
   if (num_units == 0) return cudaSuccess;
   // one warp per row of the largest unit (four rows per block), at most kMergeBlocksPerUnit blocks
   int by = (max_rows + 3) / 4;
   by = by < 1 ? 1 : (by > kMergeBlocksPerUnit ? kMergeBlocksPerUnit : by);
-  merge_units_kernel<<<dim3(num_units, by), 128, 0, s>>>(a);
+  if (max_parts > 32)
+    merge_units_kernel<true><<<dim3(num_units, by), 128, 0, s>>>(a);
+  else
+    merge_units_kernel<false><<<dim3(num_units, by), 128, 0, s>>>(a);
   return cudaGetLastError();
 }
 

@@ -276,7 +276,15 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
   }
 
   // KV splits: cap the cost of one task at a fraction of the mean per-worker load.
-  const int max_splits = cfg.max_splits > 0 ? cfg.max_splits : 32;
+  // Default bound on the splits of one unit: 32, or, when the batch has only a few streaming
+  // units (a single long-context decode), enough for one task per worker.
+  int max_splits = cfg.max_splits;
+  if (max_splits <= 0) {
+    int n_stream = 0;
+    for (const Unit& u : units) n_stream += u.kind == 1 ? 1 : 0;
+    max_splits = 32;
+    if (n_stream > 0) max_splits = std::max(32, std::min(128, ceil_div(num_workers, n_stream)));
+  }
   double total_cost = 0.0;
   for (const Unit& u : units) total_cost += kTaskFixedUs + u.visit_cost * (u.nkt - u.kt0);
   float cap = static_cast<float>(total_cost / std::max(1, num_workers) * kTaskCapFraction);

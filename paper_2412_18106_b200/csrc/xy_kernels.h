@@ -20,7 +20,7 @@ struct MergeArgs {
 
 cudaError_t launch_reference(const RunArgs& a, int num_workers, cudaStream_t s);
 cudaError_t launch_meta(const RunArgs& a, int num_workers, int64_t num_pages, bool umma, cudaStream_t s);
-cudaError_t launch_merge_units(const MergeArgs& a, int num_units, int max_rows, cudaStream_t s);
+cudaError_t launch_merge_units(const MergeArgs& a, int num_units, int max_rows, int max_parts, cudaStream_t s);
 cudaError_t launch_merge_plain(const float* o_part, const float* lse_part, int num_splits,
                                int64_t rows, uint16_t* o, float* lse, cudaStream_t s);
 cudaError_t launch_merge_shards(const uint16_t* o_shards, const float* lse_shards, int num_shards,

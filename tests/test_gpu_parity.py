@@ -277,3 +277,21 @@ def test_maximum_sizes_one_million_token_context_and_largest_tree():
     ctx.close()
     O_ref, LSE_ref = oracle.attention(b, t, H.SCALE)
     H.check_against_oracle(O, LSE, O_ref, LSE_ref, "max_sizes")
+
+
+@pytest.mark.parametrize("hq,hkv,kv", [(8, 1, 400_000), (8, 2, 1_000_003)])
+def test_single_long_context_is_cut_for_every_worker(hq, hkv, kv):
+    """One decode request on a very long context: the default bound on splits grows so that every
+    worker gets a key range (more than 32 partials per row: the wide merge kernel)."""
+    b = W.custom("one_long", hq, hkv, 128, [(1, kv, 0, None)], seed=5, spare_frac=0.01)
+    ctx = H.make_ctx(b)
+    info = ctx.plan_batch(b)
+    mu = ctx.get_merge_units()
+    assert int(mu["nsplit"].max()) > 32 and 100 <= info.num_tasks <= 148
+    t = W.make_tensors(b)
+    O, LSE = H.run_gpu(b, t, ctx=ctx)
+    O2, LSE2 = H.run_gpu(b, t, ctx=ctx)
+    ctx.close()
+    assert np.array_equal(O, O2) and np.array_equal(LSE, LSE2)
+    O_ref, LSE_ref = oracle.attention(b, t, H.SCALE)
+    H.check_against_oracle(O, LSE, O_ref, LSE_ref, "one long context")

@@ -228,6 +228,21 @@ def test_splits_appear_for_long_decode_and_respect_max_splits():
     coverage_check(b, c, info)
 
 
+def test_default_split_bound_grows_when_few_streaming_units_exist():
+    # two units (one request, two kv heads) on 148 workers: 74 splits each, one task per worker
+    b = W.custom("one_long", 8, 2, 128, [(1, 1_000_000, 0, None)], seed=2)
+    c = host_ctx(8, 2, 128, num_workers=148, max_pages_per_req=8192)
+    info = c.plan_batch(b)
+    assert info.num_tasks == 148 and int(c.get_merge_units()["nsplit"].max()) == 74
+    coverage_check(b, c, info)
+    # many units: the bound stays at 32
+    b = W.custom("many", 8, 2, 128, [(1, 300_000, 0, None)] * 8 + [(1, 1_000_000, 0, None)], seed=2)
+    c = host_ctx(8, 2, 128, num_workers=148, max_pages_per_req=8192)
+    info = c.plan_batch(b)
+    assert int(c.get_merge_units()["nsplit"].max()) <= 32
+    coverage_check(b, c, info)
+
+
 def test_paper_mode_equals_python_task_table_and_fig3b():
     q_len, kv_len = [300, 1, 16, 1], [0, 700, 900, 350]
     hq, hkv, C, tile = 6, 6, 4, 128
