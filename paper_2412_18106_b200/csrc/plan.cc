@@ -433,7 +433,8 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
       }
       std::vector<size_t> idx(head);
       std::iota(idx.begin(), idx.end(), size_t{0});
-      std::vector<size_t> first_pos(static_cast<size_t>(num_reqs) * cfg.num_kv_heads, SIZE_MAX);
+      // keyed by every Token-Table entry, the virtual requests of shared-prefix groups included
+      std::vector<size_t> first_pos(out->reqs.size() * static_cast<size_t>(cfg.num_kv_heads), SIZE_MAX);
       for (size_t i = 0; i < head; ++i)
         if (first_pos[group_of[i]] == SIZE_MAX) first_pos[group_of[i]] = i;
       std::stable_sort(idx.begin(), idx.end(),

@@ -362,3 +362,23 @@ def test_shared_prefix_groups_cover_every_key_once_and_reject_bad_groups():
     with pytest.raises(xb.XYAttnError) as e:
         c.plan_batch(pb, groups=[(0, 2, 1024)])                   # a prefill request in a group
     assert e.value.code == xb.XY_ERR_INVALID_ARG
+
+
+def test_queue_keeps_sibling_dense_tiles_of_group_requests_together():
+    """The dense tiles of a shared-prefix group's virtual request (request index >= num_reqs) are
+    regrouped like every other dense tile: in the queue, all but the last tenth of the dense tasks
+    of one (request, kv head) follow each other without another key in between."""
+    b, groups = W.shared_prefix_decode(seed=1, num_groups=2, members=32, prefix=8192, suffix_hi=512,
+                                       hq=32, hkv=8, page_size=128)
+    c = host_ctx(32, 8, 128, max_requests=256)
+    c.plan_batch(b, groups=groups)
+    tasks, queue = c.get_tasks(), c.get_queue()
+    dense = [int(q) for q in queue if tasks[int(q)]["kind"] == 0]
+    assert len(dense) > 20 and max(int(tasks[q]["req"]) for q in dense) >= b.num_requests
+    head = dense[: len(dense) - len(dense) // 10]
+    keys = [(int(tasks[q]["req"]), int(tasks[q]["kv_head"])) for q in head]
+    closed = set()
+    for k, key in enumerate(keys):
+        if k and key != keys[k - 1]:
+            closed.add(keys[k - 1])
+        assert key not in closed, "tiles of %r are not adjacent in the queue" % (key,)
