@@ -273,7 +273,9 @@ int xy_attn_merge_shards(const void* o_shards, const float* lse_shards, int32_t 
  * that loads the library holds until the process exits.
  *   q, k_pool, v_pool, block_table, o, lse: as for xy_attn_run (token r of q / o / lse is request r)
  *   kv_len      DEVICE int32 [num_reqs]: cached tokens before the new one
- *   max_kv_len  HOST value, >= every kv_len[r]; sets the number of 2048-key chunks
+ *   max_kv_len  HOST value, >= every kv_len[r]; sets the number of 2048-key chunks.  A request
+ *               whose kv_len[r] exceeds it reads nothing beyond max_kv_len + 1 keys and gets NaN
+ *               in its rows of o and lse (never a silently truncated context)
  * Limit: num_reqs * num_q_heads * ceil((max_kv_len + 1) / 2048) <= XY_ATTN_STATIC_MAX_ROWS;
  * beyond it the call returns XY_ERR_CAPACITY (and prints one line to stderr) without launching.
  * The first call on each device looks up the scratch's device address; make that first call
@@ -331,14 +333,38 @@ int xy_attn_set_timing(xy_attn_ctx* ctx, int32_t enable);
 int xy_attn_get_timing(xy_attn_ctx* ctx, float* attention_ms /*HOST*/, float* merge_ms /*HOST*/,
                        int32_t* runs /*HOST*/);
 
+/* Validation aid (the stand-in for a memory checker on the paged gather, Section 4.1.1).  Checks a
+ * HOST copy of the block table against the current plan: every request must find
+ * ceil((kv_len + q_len) / B) entries in its row (<= block_table_stride) and each of them must lie
+ * in [0, num_pages).  Host arithmetic only; works on a host-only context.  Returns XY_OK,
+ * XY_ERR_NOT_PLANNED, or XY_ERR_INVALID_ARG with the offending request and entry in
+ * xy_attn_last_error.  A context created while the environment variable XY_ATTN_DEBUG=1 is set
+ * runs this check inside every xy_attn_run (it copies the device block table to the host first,
+ * which synchronises the stream) and launches nothing when it fails. */
+int xy_attn_debug_check_block_table(xy_attn_ctx* ctx, const int32_t* block_table /*HOST*/,
+                                    int32_t block_table_stride, int64_t num_pages);
+
+/* Failure-path test hook for the bounded waits of the attention kernel (every wait on a barrier
+ * or a turn counter gives up after a limit and records XY_ERR_DEVICE_TIMEOUT, Section 4.2.1's
+ * pipelines being chains of such hand-offs).  wait_limit_polls > 0 replaces the limit (0 restores
+ * the default of 2^22 polls); skip_fill >= 0 makes the producer of every worker leave out its
+ * skip_fill-th K/V stage fill of the following runs (-1: none), so that the readers of that stage
+ * never see it filled and their waits run out.  Nothing faults and nothing spins without bound:
+ * the kernel returns, frees its tensor memory, and the status shows the timeout; O and LSE of
+ * such a run are unspecified.  The next run on the context starts from a clean status word. */
+int xy_attn_debug_inject(xy_attn_ctx* ctx, int32_t wait_limit_polls, int32_t skip_fill);
+
 /* Number of kernel launches the last xy_attn_run enqueued. */
 int xy_attn_last_launches(const xy_attn_ctx* ctx);
 
 /* Message of the last error on this context (never null). */
 const char* xy_attn_last_error(const xy_attn_ctx* ctx);
 
-/* Synchronises the device and reads the status word the kernels write:
- * XY_OK, or XY_ERR_DEVICE_TIMEOUT when a bounded wait inside a kernel gave up. */
+/* Synchronises the device, reads the status the kernels recorded and clears it: XY_OK, or
+ * XY_ERR_DEVICE_TIMEOUT when a bounded wait inside a kernel gave up in any run since the last
+ * call.  A run whose status is not XY_OK has unspecified O and LSE.  The context stays usable:
+ * every xy_attn_run starts from a clean status word, so the run after a timeout is an ordinary
+ * run (the record of the failure is kept until this function reports it). */
 int xy_attn_device_status(xy_attn_ctx* ctx, int32_t* status_out /*HOST*/);
 
 #ifdef __cplusplus

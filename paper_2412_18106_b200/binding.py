@@ -82,7 +82,7 @@ EXPORTS = (
     "xy_attn_set_timing", "xy_attn_get_timing", "xy_attn_debug_trace", "xy_attn_decode_static",
     "xy_attn_append_kv", "xy_attn_worker_times", "xy_attn_get_queue", "xy_attn_plan_cache",
     "xy_attn_plan_shared", "xy_attn_shard_context", "xy_attn_merge_shards",
-    "xy_attn_find_prefix_groups",
+    "xy_attn_find_prefix_groups", "xy_attn_debug_check_block_table", "xy_attn_debug_inject",
 )
 
 _lib = None
@@ -122,6 +122,8 @@ def load() -> ctypes.CDLL:
     L.xy_attn_plan_cache.argtypes = [vp, i32, ctypes.POINTER(i64), ctypes.POINTER(i64)]
     L.xy_attn_decode_static.argtypes = [vp, i64, vp, vp, i64, i64, i64, vp, i32, vp, i32, i32, i32, i32, i32,
                                         ctypes.c_float, vp, i64, vp, vp]
+    L.xy_attn_debug_check_block_table.argtypes = [vp, vp, i32, i64]
+    L.xy_attn_debug_inject.argtypes = [vp, i32, i32]
     L.xy_attn_last_launches.argtypes = [vp]
     L.xy_attn_last_error.argtypes = [vp]
     L.xy_attn_last_error.restype = ctypes.c_char_p
@@ -331,6 +333,16 @@ class XYAttn:
         self.lib.xy_attn_debug_trace(self._ctx, ctypes.c_void_p(out.ctypes.data), n)
         return out.reshape(4, -1)
 
+    def debug_check_block_table(self, block_table: np.ndarray, num_pages: int) -> None:
+        """xy_attn_debug_check_block_table on a HOST int32 [R, stride] array; raises on a bad entry."""
+        bt = np.ascontiguousarray(block_table, dtype=np.int32)
+        assert bt.ndim == 2
+        self._check(self.lib.xy_attn_debug_check_block_table(self._ctx, ctypes.c_void_p(bt.ctypes.data),
+                                                             bt.shape[1], int(num_pages)))
+
+    def debug_inject(self, wait_limit_polls: int = 0, skip_fill: int = -1) -> None:
+        self._check(self.lib.xy_attn_debug_inject(self._ctx, int(wait_limit_polls), int(skip_fill)))
+
     def last_launches(self) -> int:
         return int(self.lib.xy_attn_last_launches(self._ctx))
 
@@ -415,6 +427,13 @@ def xy_attn_decode_static(q, k_pool, v_pool, block_table, kv_len, max_kv_len: in
     for t in (q, k_pool, v_pool, block_table, kv_len, o, lse):
         if not t.is_cuda:
             raise XYAttnError(XY_ERR_INVALID_ARG, "xy_attn_decode_static needs CUDA tensors")
+    if not (q.dtype == o.dtype == k_pool.dtype == v_pool.dtype == torch.bfloat16 and lse.dtype == torch.float32
+            and kv_len.dtype == torch.int32 and block_table.dtype == torch.int32):
+        raise XYAttnError(XY_ERR_INVALID_ARG, "xy_attn_decode_static: q, o and the pools must be bf16, lse fp32, "
+                                              "kv_len and block_table int32")
+    assert q.stride(2) == 1 and q.stride(1) == 128 and o.stride(2) == 1 and o.stride(1) == 128
+    assert lse.is_contiguous() and kv_len.is_contiguous() and block_table.stride(1) == 1
+    assert k_pool.stride() == v_pool.stride() and k_pool.stride(3) == 1
     return int(L.xy_attn_decode_static(
         q.data_ptr(), q.stride(0), k_pool.data_ptr(), v_pool.data_ptr(), k_pool.stride(0), k_pool.stride(1),
         k_pool.stride(2), block_table.data_ptr(), block_table.stride(0), kv_len.data_ptr(), q.shape[0],

@@ -40,6 +40,11 @@ struct xy_attn_ctx {
   unsigned long long* d_trace = nullptr;
   unsigned long long* d_worker_times = nullptr;
   int last_launches = 0;
+  MetaLaunchCache launch_cache;     // tensor maps of the last pools seen, kernel attributes set once
+  uint32_t dbg_wait_limit = 0;      // 0: default
+  int32_t dbg_skip_fill = -1;       // -1: none
+  bool debug_validate = false;      // XY_ATTN_DEBUG=1 at create: block tables are range-checked before launch
+  std::vector<int32_t> dbg_bt;      // host copy of the block table for that check
   bool timing = false;
   std::vector<cudaEvent_t> events;  // three per timed run: before attention, after it, after merge
   int timed_runs = 0;
@@ -158,6 +163,8 @@ int xy_attn_create(const xy_attn_config* cfg, xy_attn_ctx** out) {
     alloc(reinterpret_cast<void**>(&c->d_status), 256);
     alloc(reinterpret_cast<void**>(&c->d_worker_times), sizeof(unsigned long long) * 4 * c->num_workers);
     if (e == cudaSuccess) e = cudaMemset(c->d_status, 0, 256);
+    const char* dbg = getenv("XY_ATTN_DEBUG");
+    c->debug_validate = dbg != nullptr && dbg[0] == '1';
     const char* tr = getenv("XY_ATTN_TRACE");
     if (tr != nullptr && tr[0] == '1') {
       alloc(reinterpret_cast<void**>(&c->d_trace), sizeof(unsigned long long) * kTraceRoles * kTraceLen);
@@ -248,6 +255,34 @@ int xy_attn_plan_shared(xy_attn_ctx* ctx, const xy_attn_request* reqs, int32_t n
   return XY_OK;
 }
 
+int xy_attn_debug_check_block_table(xy_attn_ctx* ctx, const int32_t* block_table, int32_t block_table_stride,
+                                    int64_t num_pages) {
+  if (ctx == nullptr) return XY_ERR_INVALID_ARG;
+  if (!ctx->planned) return set_err(ctx, XY_ERR_NOT_PLANNED, "block-table check before xy_attn_plan");
+  if (block_table == nullptr || block_table_stride < 1 || num_pages < 1)
+    return set_err(ctx, XY_ERR_INVALID_ARG, "null block table, bad stride or num_pages");
+  char buf[200];
+  const int B = ctx->cfg.page_size;
+  for (size_t r = 0; r < ctx->plan.reqs.size(); ++r) {
+    const ReqInfo& rq = ctx->plan.reqs[r];
+    const int64_t need = (static_cast<int64_t>(rq.kv_len) + rq.q_len + B - 1) / B;
+    if (need > block_table_stride) {
+      snprintf(buf, sizeof buf, "request %zu needs %lld block-table entries, the row has %d", r,
+               static_cast<long long>(need), block_table_stride);
+      return set_err(ctx, XY_ERR_INVALID_ARG, buf);
+    }
+    const int32_t* row = block_table + static_cast<int64_t>(rq.bt_row) * block_table_stride;
+    for (int64_t p = 0; p < need; ++p) {
+      if (row[p] < 0 || row[p] >= num_pages) {
+        snprintf(buf, sizeof buf, "block table of request %zu, entry %lld: page %d outside [0, %lld)", r,
+                 static_cast<long long>(p), row[p], static_cast<long long>(num_pages));
+        return set_err(ctx, XY_ERR_INVALID_ARG, buf);
+      }
+    }
+  }
+  return XY_OK;
+}
+
 int xy_attn_run(xy_attn_ctx* ctx, const void* q, int64_t q_token_stride, const void* k_pool,
                 const void* v_pool, int64_t num_pages, int64_t page_stride, int64_t head_stride,
                 int64_t token_stride, const int32_t* block_table, int32_t block_table_stride,
@@ -277,6 +312,19 @@ int xy_attn_run(xy_attn_ctx* ctx, const void* q, int64_t q_token_stride, const v
 
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   XY_CUDA(ctx, cudaSetDevice(cfg.device));
+  if (ctx->debug_validate) {
+    // Validation build of the call (XY_ATTN_DEBUG=1 at create): the block table is brought to the
+    // host (this synchronises the stream and allocates host memory - a debugging aid, not the
+    // serving path) and every entry a planned request uses is range-checked before anything runs.
+    int32_t max_row = 0;
+    for (const ReqInfo& rq : p.reqs) max_row = std::max(max_row, rq.bt_row);
+    ctx->dbg_bt.resize(static_cast<size_t>(max_row + 1) * block_table_stride);
+    XY_CUDA(ctx, cudaStreamSynchronize(s));
+    XY_CUDA(ctx, cudaMemcpy(ctx->dbg_bt.data(), block_table, ctx->dbg_bt.size() * sizeof(int32_t),
+                            cudaMemcpyDeviceToHost));
+    const int rc = xy_attn_debug_check_block_table(ctx, ctx->dbg_bt.data(), block_table_stride, num_pages);
+    if (rc != XY_OK) return rc;
+  }
   RunArgs a{};
   a.q = static_cast<const uint16_t*>(q);
   a.q_token_stride = q_token_stride;
@@ -305,12 +353,16 @@ int xy_attn_run(xy_attn_ctx* ctx, const void* q, int64_t q_token_stride, const v
   a.page_size = cfg.page_size;
   a.page_shift = ctx->page_shift;
   a.queue = ctx->d_queue;
-  a.queue_head = ctx->d_status + 16;  // second cache line of the status block
+  a.queue_head = ctx->d_status + kStatusQueueHead;  // second cache line of the status block
   a.num_tasks = static_cast<int32_t>(p.tasks.size());
   // Balanced plans are dealt dynamically by the meta-kernel; paper-mode plans keep the static
   // Task-Table (each worker walks its own list), as does the reference kernel.
   a.dynamic = (cfg.plan_mode == XY_PLAN_BALANCED && cfg.kernel != XY_KERNEL_REFERENCE) ? 1 : 0;
-  if (a.dynamic) XY_CUDA(ctx, cudaMemsetAsync(a.queue_head, 0, sizeof(int32_t), s));
+  a.wait_limit = ctx->dbg_wait_limit ? ctx->dbg_wait_limit : (1u << 22);
+  a.debug_skip_fill = ctx->dbg_skip_fill;
+  // Every run starts with a clean status word and queue head (one memset covers both): a run
+  // after a device-side timeout is an ordinary run.  The sticky record (status[1]) is kept.
+  XY_CUDA(ctx, cudaMemsetAsync(a.status, 0, 17 * sizeof(int32_t), s));
 
   const bool timed = ctx->timing && ctx->timed_runs < kMaxTimedRuns;
   if (timed) {
@@ -325,7 +377,8 @@ int xy_attn_run(xy_attn_ctx* ctx, const void* q, int64_t q_token_stride, const v
   if (cfg.kernel == XY_KERNEL_REFERENCE) {
     XY_CUDA(ctx, launch_reference(a, ctx->num_workers, s));
   } else {
-    XY_CUDA(ctx, launch_meta(a, ctx->num_workers, num_pages, cfg.kernel == XY_KERNEL_AUTO && p.info.num_dense_tasks > 0, s));
+    XY_CUDA(ctx, launch_meta(a, ctx->num_workers, num_pages, cfg.kernel == XY_KERNEL_AUTO && p.info.num_dense_tasks > 0,
+                             &ctx->launch_cache, s));
   }
   ctx->last_launches += 1;
   if (timed) XY_CUDA(ctx, cudaEventRecord(ctx->events[3 * ctx->timed_runs + 1], s));
@@ -573,6 +626,13 @@ int xy_attn_debug_trace(xy_attn_ctx* ctx, uint64_t* out, int32_t cap) {
   return n;
 }
 
+int xy_attn_debug_inject(xy_attn_ctx* ctx, int32_t wait_limit_polls, int32_t skip_fill) {
+  if (ctx == nullptr || wait_limit_polls < 0 || skip_fill < -1) return XY_ERR_INVALID_ARG;
+  ctx->dbg_wait_limit = static_cast<uint32_t>(wait_limit_polls);
+  ctx->dbg_skip_fill = skip_fill;
+  return XY_OK;
+}
+
 int xy_attn_last_launches(const xy_attn_ctx* ctx) { return ctx ? ctx->last_launches : XY_ERR_INVALID_ARG; }
 
 const char* xy_attn_last_error(const xy_attn_ctx* ctx) { return ctx ? ctx->err.c_str() : "null context"; }
@@ -582,9 +642,16 @@ int xy_attn_device_status(xy_attn_ctx* ctx, int32_t* status_out) {
   if (ctx->host_only) return set_err(ctx, XY_ERR_UNSUPPORTED, "host-only context");
   XY_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
   XY_CUDA(ctx, cudaDeviceSynchronize());
-  int32_t st = 0;
-  XY_CUDA(ctx, cudaMemcpy(&st, ctx->d_status, sizeof st, cudaMemcpyDeviceToHost));
-  *status_out = st;
+  // word 0 is the last run's status (cleared by every run), word kStatusSticky the record of
+  // every failure since the last call of this function: report it and clear both.
+  int32_t st[kStatusSticky + 1];
+  XY_CUDA(ctx, cudaMemcpy(st, ctx->d_status, sizeof st, cudaMemcpyDeviceToHost));
+  const int32_t seen = st[kStatusSticky] != 0 ? st[kStatusSticky] : st[0];
+  if (seen != 0) {
+    XY_CUDA(ctx, cudaMemset(ctx->d_status, 0, sizeof(int32_t)));
+    XY_CUDA(ctx, cudaMemset(ctx->d_status + kStatusSticky, 0, sizeof(int32_t)));
+  }
+  *status_out = seen;
   return XY_OK;
 }
 

@@ -50,11 +50,15 @@ __global__ void decode_static_partial_kernel(const uint16_t* q, int64_t q_token_
                                              const uint16_t* v_pool, int64_t page_stride, int64_t head_stride,
                                              int64_t token_stride, const int32_t* block_table, int bt_stride,
                                              const int32_t* kv_len, int G, int Hq, int page_size, int page_shift,
-                                             float sm_scale, int num_chunks, float* scratch_o, float* scratch_lse) {
+                                             float sm_scale, int num_chunks, int max_kv_len, float* scratch_o,
+                                             float* scratch_lse) {
   const int chunk = blockIdx.x, g = blockIdx.y, r = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int head = g * G + warp;
-  const int L = kv_len[r] + 1;  // cached tokens plus the new one, whose K/V is already in the cache
+  // cached tokens plus the new one, whose K/V is already in the cache; never beyond what the
+  // caller's max_kv_len sized the chunks (and its block-table rows) for: a request that breaks
+  // the bound gets NaN from the merge kernel instead of a silently truncated context
+  const int L = min(kv_len[r], max_kv_len) + 1;
   const int j_lo = chunk * kChunkKeys, j_hi = min(L, j_lo + kChunkKeys);
   const uint16_t* qp = q + static_cast<int64_t>(r) * q_token_stride + head * kD + lane * 4;
   float qv[4];
@@ -86,10 +90,18 @@ __global__ void decode_static_partial_kernel(const uint16_t* q, int64_t q_token_
 
 // One warp per (request, q head): merge its chunks.
 __global__ void decode_static_merge_kernel(const float* scratch_o, const float* scratch_lse, int num_chunks,
-                                           int64_t rows, int Hq, uint16_t* o, int64_t o_token_stride, float* lse) {
+                                           int64_t rows, int Hq, const int32_t* kv_len, int max_kv_len, uint16_t* o,
+                                           int64_t o_token_stride, float* lse) {
   const int64_t x = static_cast<int64_t>(blockIdx.x) * 4 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (x >= rows) return;
+  if (kv_len[x / Hq] > max_kv_len) {  // the caller's bound does not hold for this request: say so loudly
+    uint16_t* bad = o + (x / Hq) * o_token_stride + (x % Hq) * kD + lane * 4;
+#pragma unroll
+    for (int d = 0; d < 4; ++d) bad[d] = 0x7FC0u;  // bf16 NaN
+    if (lane == 0) lse[x] = __int_as_float(0x7FC00000);
+    return;
+  }
   const float* lc = scratch_lse + x * num_chunks;
   float mx = -INFINITY;
   for (int c = 0; c < num_chunks; ++c) mx = fmaxf(mx, lc[c]);
@@ -129,13 +141,14 @@ extern "C" int xy_attn_decode_static(const void* q, int64_t q_token_stride, cons
   if (q_token_stride < static_cast<int64_t>(num_q_heads) * kD || o_token_stride < static_cast<int64_t>(num_q_heads) * kD ||
       token_stride < kD || block_table_stride < 1 || !(sm_scale > 0.f))
     return XY_ERR_INVALID_ARG;
-  const int num_chunks = (max_kv_len + 1 + kChunkKeys - 1) / kChunkKeys;
+  const int64_t num_chunks64 = (static_cast<int64_t>(max_kv_len) + 1 + kChunkKeys - 1) / kChunkKeys;
   const int64_t rows = static_cast<int64_t>(num_reqs) * num_q_heads;
+  const int num_chunks = static_cast<int>(num_chunks64 > XY_ATTN_STATIC_MAX_ROWS ? XY_ATTN_STATIC_MAX_ROWS + 1 : num_chunks64);
   if (rows * num_chunks > XY_ATTN_STATIC_MAX_ROWS) {
     fprintf(stderr,
             "xy_attn_decode_static: num_reqs * num_q_heads * ceil((max_kv_len + 1) / %d) = %lld exceeds the static "
             "scratch of %d partial rows\n",
-            kChunkKeys, static_cast<long long>(rows * num_chunks), XY_ATTN_STATIC_MAX_ROWS);
+            kChunkKeys, static_cast<long long>(rows * num_chunks64), XY_ATTN_STATIC_MAX_ROWS);
     return XY_ERR_CAPACITY;
   }
   // Set-up, once per device, with that device current: the device address of the scratch.
@@ -161,10 +174,11 @@ extern "C" int xy_attn_decode_static(const void* q, int64_t q_token_stride, cons
   decode_static_partial_kernel<<<grid, 32 * G, 0, s>>>(
       static_cast<const uint16_t*>(q), q_token_stride, static_cast<const uint16_t*>(k_pool),
       static_cast<const uint16_t*>(v_pool), page_stride, head_stride, token_stride, block_table, block_table_stride,
-      kv_len, G, num_q_heads, page_size, page_shift, sm_scale, num_chunks, scratch_o, scratch_lse);
+      kv_len, G, num_q_heads, page_size, page_shift, sm_scale, num_chunks, max_kv_len, scratch_o, scratch_lse);
   if (cudaGetLastError() != cudaSuccess) return XY_ERR_CUDA;
   decode_static_merge_kernel<<<static_cast<unsigned>((rows + 3) / 4), 128, 0, s>>>(
-      scratch_o, scratch_lse, num_chunks, rows, num_q_heads, static_cast<uint16_t*>(o), o_token_stride, lse);
+      scratch_o, scratch_lse, num_chunks, rows, num_q_heads, kv_len, max_kv_len, static_cast<uint16_t*>(o),
+      o_token_stride, lse);
   if (cudaGetLastError() != cudaSuccess) return XY_ERR_CUDA;
   return XY_OK;
 }

@@ -332,8 +332,11 @@ struct Tracer {
 #endif
 };
 
+// Word 0 of the status block is this run's (cleared at every launch, polled by every wait); the
+// sticky word is what xy_attn_device_status reads and clears.
 __device__ __forceinline__ void report_timeout(const RunArgs& a) {
   atomicExch(a.status, XY_ERR_DEVICE_TIMEOUT);
+  atomicExch(a.status + kStatusSticky, XY_ERR_DEVICE_TIMEOUT);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -376,7 +379,7 @@ __device__ __forceinline__ uint32_t stream_task(const RunArgs& a, const TaskView
     long long c_prev = clock64();
     ph[5] += 1;
 #endif
-    if (!dead && !mbar_wait(smem_u32(&bars->full[pipe.stage]), pipe.phase, a.status)) {
+    if (!dead && !mbar_wait(smem_u32(&bars->full[pipe.stage]), pipe.phase, a.status, a.wait_limit)) {
       report_timeout(a);
       dead = true;
     }
@@ -391,7 +394,7 @@ __device__ __forceinline__ uint32_t stream_task(const RunArgs& a, const TaskView
       w.softmax(a, tv.rq, s, p, col0, i_lo, i_hi, need_mask, scale_log2, lane);
     }
     XY_PH(2)
-    if (!dead && !mbar_wait(smem_u32(&bars->full[pipe.stage]), pipe.phase, a.status)) {
+    if (!dead && !mbar_wait(smem_u32(&bars->full[pipe.stage]), pipe.phase, a.status, a.wait_limit)) {
       report_timeout(a);
       dead = true;
     }
@@ -470,18 +473,6 @@ constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kTmemS = 0, kTmemO = 256;
 constexpr float kRescaleThreshold = 8.0f;  // log2 units: rescale O only when the row max grows by > 2^8
 
-// Shared-memory matrix descriptor, 128-byte swizzle, 8-row groups 1024 B apart.
-//   K-major operand (Q, K): rows are MN, 64 elements (128 B) per row; LBO unused.
-//   MN-major operand (V):   rows are K (keys), the second 64-element half of N is LBO bytes away.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes) {
-  uint64_t d = 0;
-  d |= static_cast<uint64_t>((addr >> 4) & 0x3FFFu);
-  d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFFu) << 16;
-  d |= static_cast<uint64_t>((1024u >> 4) & 0x3FFFu) << 32;
-  d |= 1ull << 46;  // descriptor version for sm_100
-  d |= 2ull << 61;  // SWIZZLE_128B
-  return d;
-}
 // Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 128.
 constexpr uint32_t kIdescBase = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 constexpr uint32_t kIdescQK = kIdescBase;              // A, B K-major
@@ -522,15 +513,12 @@ struct __align__(8) UmmaBarriers {
   uint64_t s_full[2];  // MMA -> consumers: S = Q K^T of the next KV tile is in TMEM
   uint64_t p_full[2][2];  // consumers -> MMA: [sub-tile][half] 64 keys of P are in TMEM (O rescaled if need be)
   uint64_t o_done[2];  // MMA -> consumers: the task's last P V has completed
+  uint64_t drained[2];  // every MMA an issuer has issued has completed (waited for once, before exit)
   uint32_t tmem_base;
   volatile uint32_t turn;  // index of the next MMA group allowed onto the tensor pipe
 };
 
-// Corner-mask words of one row covering columns [jp0, jp0 + 128) of the speculative corner.
-struct TreeWords {
-  uint64_t w[3];
-  int wbase;
-};
+static_assert(sizeof(UmmaBarriers) <= 128, "the shared-memory layout reserves 128 bytes for UmmaBarriers");
 
 template <bool kUmma>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -569,6 +557,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
       mbar_init(smem_u32(&ub->p_full[X][0]), 4);
       mbar_init(smem_u32(&ub->p_full[X][1]), 4);
       mbar_init(smem_u32(&ub->o_done[X]), 1);
+      mbar_init(smem_u32(&ub->drained[X]), 1);
     }
     fence_mbar_init();
   }
@@ -591,8 +580,8 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
   auto next_task = [&](bool whole_warp) -> int {  // whole_warp: called by all 32 lanes (else by one)
     if (!dynamic) return seq_static < t_end ? seq_static++ : -1;
     const uint32_t slot = n_read % kTaskRing;
-    if (!feed_dead && !mbar_wait(smem_u32(&tq->full[slot]), (n_read / kTaskRing) & 1u, a.status)) {
-      atomicExch(a.status, XY_ERR_DEVICE_TIMEOUT);
+    if (!feed_dead && !mbar_wait(smem_u32(&tq->full[slot]), (n_read / kTaskRing) & 1u, a.status, a.wait_limit)) {
+      report_timeout(a);
       feed_dead = true;
     }
     const int ti = feed_dead ? -1 : tq->ti[slot];
@@ -619,21 +608,29 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
       // Who read each stage last (bit set: the tcgen05 path) and the parity to wait for on each
       // of the two empty barriers of a stage; a stage that was never filled needs no wait.
       uint32_t used = 0, last_umma = 0, ph_cons = 0, ph_umma = 0;
+      uint32_t fill_par = 0;  // per stage: parity of the `full` phase its latest fill completes
       Tracer tr;
       tr.init(a, 3, true);
       const int ppt = kKeyTile >> a.page_shift;  // pages per 128-key tile
       const uint32_t page_bytes = static_cast<uint32_t>(a.page_size) * 128u;
       const uint64_t pol_stream = make_l2_policy_evict_first(), pol_keep = make_l2_policy_evict_last();
       // Fill one stage (the K or the V tile) once its previous reader has released it.
+      int n_fill = 0;
       auto fill = [&](int op, bool by_umma, int kv_head, int kt, const int32_t* bt, int npages, int page0) {
+        // Failure-path test hook (xy_attn_debug_inject): this worker leaves out one fill, so the
+        // stage's `full` barrier never completes and the readers' bounded waits run out.
+        if (n_fill++ == a.debug_skip_fill) {
+          pipe.advance();
+          return;
+        }
         const uint32_t bit = 1u << pipe.stage;
         if (used & bit) {
           bool ok;
           if (last_umma & bit) {
-            ok = mbar_wait(smem_u32(&bars->empty_umma[pipe.stage]), (ph_umma >> pipe.stage) & 1u, a.status);
+            ok = mbar_wait(smem_u32(&bars->empty_umma[pipe.stage]), (ph_umma >> pipe.stage) & 1u, a.status, a.wait_limit);
             ph_umma ^= bit;
           } else {
-            ok = mbar_wait(smem_u32(&bars->empty[pipe.stage]), (ph_cons >> pipe.stage) & 1u, a.status);
+            ok = mbar_wait(smem_u32(&bars->empty[pipe.stage]), (ph_cons >> pipe.stage) & 1u, a.status, a.wait_limit);
             ph_cons ^= bit;
           }
           if (!ok) {
@@ -642,6 +639,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
             return;
           }
         }
+        if (used & bit) fill_par ^= bit;
         used |= bit;
         last_umma = by_umma ? (last_umma | bit) : (last_umma & ~bit);
         tr(1 + op);
@@ -687,7 +685,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
         if (k < a.num_tasks) ti = __ldg(a.queue + k);
         const uint32_t slot = n_pub % kTaskRing;
         if (n_pub >= kTaskRing &&
-            !mbar_wait(smem_u32(&tq->empty[slot]), ((n_pub / kTaskRing) - 1u) & 1u, a.status)) {
+            !mbar_wait(smem_u32(&tq->empty[slot]), ((n_pub / kTaskRing) - 1u) & 1u, a.status, a.wait_limit)) {
           report_timeout(a);
           dead = true;
         }
@@ -738,6 +736,11 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
         fill(0, cur.by_umma, cur.kv_head, cur.kt, cur.bt, cur.npages, cur.page);
         if (!dead) fill(1, cur.by_umma, cur.kv_head, cur.kt, cur.bt, cur.npages, cur.page);
       }
+      // No bulk copy of this CTA may still be in flight when it exits: the latest fill of every
+      // stage has landed once its `full` phase completes (immediate on the normal path, where the
+      // readers have long consumed it; a bounded wait after a failure).
+      for (int s = 0; s < kStages; ++s)
+        if (used & (1u << s)) mbar_wait(smem_u32(&bars->full[s]), (fill_par >> s) & 1u, a.status, 1u << 16);
     } else if (kUmma && (warp == kConsumerWarps + 1 || warp == kConsumerWarps + 2) && lane == 0) {
       // ================================ tcgen05 MMA issuers =============================
       // One issuing thread per sub-tile (on different schedulers), each walking its own chain
@@ -750,7 +753,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
       Tracer tr;
       tr.init(a, 2, X == 0);
       auto wait_or_die = [&](uint32_t bar, uint32_t parity) {
-        if (!dead && !mbar_wait(bar, parity, a.status)) {
+        if (!dead && !mbar_wait(bar, parity, a.status, a.wait_limit)) {
           report_timeout(a);
           dead = true;
         }
@@ -818,7 +821,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
       auto take_turn = [&](uint32_t g) {
         if (dead) return;
         for (uint32_t spin = 0; ub->turn != g; ++spin) {
-          if (spin > (1u << 22) || ((spin & 4095u) == 4095u && *reinterpret_cast<const volatile int32_t*>(a.status) != 0)) {
+          if (spin > a.wait_limit || ((spin & 4095u) == 4095u && *reinterpret_cast<const volatile int32_t*>(a.status) != 0)) {
             report_timeout(a);
             dead = true;
             return;
@@ -884,6 +887,11 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
           tr(16);
         }
       }
+      // Tensor memory is freed after the final barrier: no MMA of this thread may still be in
+      // flight then.  On the normal path they completed long ago (immediate); after a failure
+      // this is a bounded wait.
+      umma_commit(smem_u32(&ub->drained[X]));
+      mbar_wait(smem_u32(&ub->drained[X]), 0u, a.status, 1u << 16);
     }
   } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsConsumer));
@@ -985,7 +993,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
         for (int j = 0; j < nX; ++j) {
           const int col0 = (tv.t.kt_lo + j) * kKeyTile;
           tr(20);
-          if (!dead && !mbar_wait(smem_u32(&ub->s_full[X]), ph_s, a.status)) {
+          if (!dead && !mbar_wait(smem_u32(&ub->s_full[X]), ph_s, a.status, a.wait_limit)) {
             report_timeout(a);
             dead = true;
           }
@@ -1120,7 +1128,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
           tr(26);
         }
         // ---- epilogue: O / l -> global
-        if (!dead && !mbar_wait(smem_u32(&ub->o_done[X]), ph_o, a.status)) {
+        if (!dead && !mbar_wait(smem_u32(&ub->o_done[X]), ph_o, a.status, a.wait_limit)) {
           report_timeout(a);
           dead = true;
         }
@@ -1232,7 +1240,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
           const bool work = active && col0 <= h + i_max;  // mask-aware skip (Section 4.2.2)
           float s[16][4];
           uint32_t p[8][4];
-          if (!dead && !mbar_wait(smem_u32(&bars->full[pipe.stage]), pipe.phase, a.status)) {
+          if (!dead && !mbar_wait(smem_u32(&bars->full[pipe.stage]), pipe.phase, a.status, a.wait_limit)) {
             report_timeout(a);
             dead = true;
           }
@@ -1244,7 +1252,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
             const bool need_mask = tree ? (col0 + kKeyTile > h) : (col0 + kKeyTile > h + i_min + 1);
             w.softmax(a, tv.rq, s, p, col0, i_lo, i_hi, need_mask, scale_log2, lane);
           }
-          if (!dead && !mbar_wait(smem_u32(&bars->full[pipe.stage]), pipe.phase, a.status)) {
+          if (!dead && !mbar_wait(smem_u32(&bars->full[pipe.stage]), pipe.phase, a.status, a.wait_limit)) {
             report_timeout(a);
             dead = true;
           }
@@ -1337,18 +1345,40 @@ bool encode_pool_map(CUtensorMap* m, const void* pool, int64_t num_pages, int nu
 
 }  // namespace
 
-cudaError_t launch_meta(const RunArgs& a, int num_workers, int64_t num_pages, bool umma, cudaStream_t s) {
+cudaError_t launch_meta(const RunArgs& a, int num_workers, int64_t num_pages, bool umma, MetaLaunchCache* cache,
+                        cudaStream_t s) {
+  static_assert(sizeof(CUtensorMap) == 128, "MetaLaunchCache holds a tensor map in 128 bytes");
   auto kernel = umma ? meta_attention_kernel<true> : meta_attention_kernel<false>;
-  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTotal);
-  if (e != cudaSuccess) return e;
-  CUtensorMap k_map, v_map;
-  if (!encode_pool_map(&k_map, a.k_pool, num_pages, a.num_kv_heads, a.page_size, a.page_stride, a.head_stride,
-                       a.token_stride) ||
-      !encode_pool_map(&v_map, a.v_pool, num_pages, a.num_kv_heads, a.page_size, a.page_stride, a.head_stride,
-                       a.token_stride))
-    return cudaErrorInvalidValue;
+  if (!cache->attr_set[umma ? 1 : 0]) {
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTotal);
+    if (e != cudaSuccess) return e;
+    cache->attr_set[umma ? 1 : 0] = true;
+  }
+  CUtensorMap* k_map = reinterpret_cast<CUtensorMap*>(cache->maps[0]);
+  CUtensorMap* v_map = reinterpret_cast<CUtensorMap*>(cache->maps[1]);
+  const bool same = cache->valid && cache->k_pool == a.k_pool && cache->v_pool == a.v_pool &&
+                    cache->num_pages == num_pages && cache->page_stride == a.page_stride &&
+                    cache->head_stride == a.head_stride && cache->token_stride == a.token_stride &&
+                    cache->num_kv_heads == a.num_kv_heads && cache->page_size == a.page_size;
+  if (!same) {
+    cache->valid = false;
+    if (!encode_pool_map(k_map, a.k_pool, num_pages, a.num_kv_heads, a.page_size, a.page_stride, a.head_stride,
+                         a.token_stride) ||
+        !encode_pool_map(v_map, a.v_pool, num_pages, a.num_kv_heads, a.page_size, a.page_stride, a.head_stride,
+                         a.token_stride))
+      return cudaErrorInvalidValue;
+    cache->k_pool = a.k_pool;
+    cache->v_pool = a.v_pool;
+    cache->num_pages = num_pages;
+    cache->page_stride = a.page_stride;
+    cache->head_stride = a.head_stride;
+    cache->token_stride = a.token_stride;
+    cache->num_kv_heads = a.num_kv_heads;
+    cache->page_size = a.page_size;
+    cache->valid = true;
+  }
   MetaParams P{a};
-  kernel<<<num_workers, kThreads, kSmemTotal, s>>>(P, k_map, v_map);
+  kernel<<<num_workers, kThreads, kSmemTotal, s>>>(P, *k_map, *v_map);
   return cudaGetLastError();
 }
 

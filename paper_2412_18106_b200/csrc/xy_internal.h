@@ -12,6 +12,11 @@ namespace xy {
 constexpr int kHeadDim = 128;
 constexpr int kKeyTile = 128;      // keys per KV tile (one MMA N extent)
 constexpr int kStreamRowsMax = 16;
+// Words of the 256-byte status block: [0] the current run's status, polled by every bounded wait
+// and cleared when a run starts; the queue head of dynamic dealing (its own cache line); the
+// sticky record of failures that xy_attn_device_status reports and clears.
+constexpr int kStatusQueueHead = 16;
+constexpr int kStatusSticky = 32;
 constexpr int kTraceRoles = 4;      // sub-tile A, sub-tile B, MMA issuer, producer (worker 0 only)
 constexpr int kTraceLen = 2048;    // records per role and run
 
@@ -97,7 +102,7 @@ struct RunArgs {
   const int32_t* worker_off;
   float* o_part;
   float* lse_part;
-  int32_t* status;
+  int32_t* status;                   // the context's status block, see kStatus*
   unsigned long long* worker_times;  // [2 * workers]: globaltimer at entry and exit of each worker
   unsigned long long* trace;  // null unless tracing: kTraceRoles x kTraceLen (tag << 48 | cycle) records
   int32_t num_q_heads, num_kv_heads, page_size, page_shift;
@@ -105,6 +110,10 @@ struct RunArgs {
   const int32_t* queue;
   int32_t* queue_head;
   int32_t num_tasks, dynamic;
+  // bounded waits give up after this many polls; test hook: the producer of every worker leaves
+  // out its debug_skip_fill-th stage fill (-1: none)
+  uint32_t wait_limit;
+  int32_t debug_skip_fill;
 };
 
 }  // namespace xy

@@ -18,8 +18,22 @@ struct MergeArgs {
   int32_t num_q_heads, num_kv_heads;
 };
 
+// What launch_meta keeps between calls: the two TMA tensor maps (128 opaque bytes each) of the
+// pools it saw last, keyed by everything they were encoded from, and whether the kernels'
+// shared-memory attribute has been set.
+struct MetaLaunchCache {
+  alignas(64) unsigned char maps[2][128];
+  const void* k_pool = nullptr;
+  const void* v_pool = nullptr;
+  int64_t num_pages = 0, page_stride = 0, head_stride = 0, token_stride = 0;
+  int32_t num_kv_heads = 0, page_size = 0;
+  bool valid = false;
+  bool attr_set[2] = {false, false};
+};
+
 cudaError_t launch_reference(const RunArgs& a, int num_workers, cudaStream_t s);
-cudaError_t launch_meta(const RunArgs& a, int num_workers, int64_t num_pages, bool umma, cudaStream_t s);
+cudaError_t launch_meta(const RunArgs& a, int num_workers, int64_t num_pages, bool umma, MetaLaunchCache* cache,
+                        cudaStream_t s);
 cudaError_t launch_merge_units(const MergeArgs& a, int num_units, int max_rows, int max_parts, cudaStream_t s);
 cudaError_t launch_merge_plain(const float* o_part, const float* lse_part, int num_splits,
                                int64_t rows, uint16_t* o, float* lse, cudaStream_t s);

@@ -365,6 +365,41 @@ def make_tensors(batch: Batch, seed: Optional[int] = None, fused_qkv: bool = Fal
     return Tensors(q=q, k_pool=k_pool, v_pool=v_pool, qkv=qkv)
 
 
+def set_tile_onehot_v(batch: Batch, tensors: Tensors, tile: int = 128) -> None:
+    """Probe input (in place): the V row of logical key j of every request becomes the unit
+    vector e_d with d = (j // tile) mod D.  Each output element is then the probability mass of
+    every D-th key tile, so one key tile that is lost, doubled or attributed to the wrong
+    request moves an element by that tile's whole mass.  Pure data placement through the block
+    table (requests that share pages keep the same logical positions, so they agree)."""
+    B, D = batch.page_size, batch.head_dim
+    for r in range(batch.num_requests):
+        L = int(batch.q_len[r]) + int(batch.kv_len[r])
+        npg = (L + B - 1) // B
+        pages = torch.from_numpy(batch.block_table[r, :npg].astype(np.int64))
+        j = torch.arange(npg * B, dtype=torch.int64).view(npg, B)
+        d = (j // tile) % D
+        rows = torch.zeros((npg, B, D), dtype=torch.bfloat16)
+        rows.scatter_(2, d.unsqueeze(-1), 1.0)
+        tensors.v_pool[pages] = rows.unsqueeze(1).expand(npg, batch.num_kv_heads, B, D)
+
+
+def set_dominant_keys(batch: Batch, tensors: Tensors, positions, q_value: float = 4.0, k_value: float = 8.0) -> None:
+    """Probe input (in place): every query row of request r becomes the constant vector q_value
+    and the K row at logical position positions[r] (all kv heads) the constant vector k_value, so
+    that this key's score exceeds every other by hundreds and its probability is exactly 1 in any
+    fp32 softmax: the output row must then be that key's V row, bit for bit.  positions[r] must be
+    visible to every row of the request (inside the history, or the first new token of a causal request)."""
+    B = batch.page_size
+    qs = batch.q_start
+    for r in range(batch.num_requests):
+        j = int(positions[r])
+        h = int(batch.kv_len[r])
+        assert 0 <= j < h or (j == h and (int(batch.mask_kind[r]) == MASK_CAUSAL or int(batch.q_len[r]) == 1))
+        tensors.q[int(qs[r]) : int(qs[r + 1])] = q_value
+        page = int(batch.block_table[r, j // B])
+        tensors.k_pool[page, :, j % B, :] = k_value
+
+
 def pairs_per_request(batch: Batch) -> np.ndarray:
     """Allowed (query row, key) pairs per request and q head: n h + n (n+1) / 2 for
     a causal request, n h + sum of node depths for a tree request.  Pure counting,

@@ -277,6 +277,16 @@ def test_maximum_sizes_one_million_token_context_and_largest_tree():
     ctx.close()
     O_ref, LSE_ref = oracle.attention(b, t, H.SCALE)
     H.check_against_oracle(O, LSE, O_ref, LSE_ref, "max_sizes")
+    # the comparison can see 128 lost keys even here: the same batch with kv_len - 128 (a valid
+    # run on the same pool) must fail it
+    reqs2 = [(1, 1_000_003 - 128, 0, None), (64, 300_001 - 128, 1, b.tree_parents(1)), (1, 0, 0, None)]
+    b2 = W.custom("max_sizes_short", 8, 2, 128, reqs2, seed=99, spare_frac=0.01)
+    b2.block_table, b2.num_pages = b.block_table, b.num_pages
+    O_m, LSE_m = H.run_gpu(b2, t)
+    with pytest.raises(AssertionError):
+        H.check_against_oracle(O_m[:1], LSE_m[:1], O_ref[:1], LSE_ref[:1], "mutant, million-token row")
+    with pytest.raises(AssertionError):
+        H.check_against_oracle(O_m[1:65], LSE_m[1:65], O_ref[1:65], LSE_ref[1:65], "mutant, tree rows")
 
 
 @pytest.mark.parametrize("hq,hkv,kv", [(8, 1, 400_000), (8, 2, 1_000_003)])

@@ -382,3 +382,37 @@ def test_queue_keeps_sibling_dense_tiles_of_group_requests_together():
         if k and key != keys[k - 1]:
             closed.add(keys[k - 1])
         assert key not in closed, "tiles of %r are not adjacent in the queue" % (key,)
+
+
+def test_debug_block_table_check_on_the_host():
+    """The validation aid: a host copy of the block table is checked against the plan, every entry
+    a request uses must lie in [0, num_pages) and fit the row; unused entries (-1) are ignored."""
+    b = W.config1_tiny()
+    c = host_ctx(8, 2, 16)
+    with pytest.raises(xb.XYAttnError) as e:
+        c.debug_check_block_table(b.block_table, b.num_pages)
+    assert e.value.code == xb.XY_ERR_NOT_PLANNED
+    c.plan_batch(b)
+    c.debug_check_block_table(b.block_table, b.num_pages)   # rows carry -1 beyond what a request uses
+    need = -(-(int(b.kv_len[2]) + int(b.q_len[2])) // 16)
+    for bad in (-1, b.num_pages, 2 ** 31 - 1):
+        bt = b.block_table.copy()
+        bt[2, need - 1] = bad
+        with pytest.raises(xb.XYAttnError) as e:
+            c.debug_check_block_table(bt, b.num_pages)
+        assert e.value.code == xb.XY_ERR_INVALID_ARG and "request 2" in str(e.value)
+        bt[2, need - 1] = b.block_table[2, need - 1]
+        bt[2, need:] = bad                                   # beyond the request's last page: not read
+        c.debug_check_block_table(bt, b.num_pages)
+    with pytest.raises(xb.XYAttnError) as e:                 # a row too short for the longest request
+        c.debug_check_block_table(b.block_table[:, : need - 1], b.num_pages)
+    assert e.value.code == xb.XY_ERR_INVALID_ARG
+    # groups: the virtual request reads the first member's row
+    gb, groups = W.shared_prefix_decode(seed=3, num_groups=2, members=8, prefix=256, suffix_hi=100, hq=8, hkv=2,
+                                        page_size=64)
+    g = host_ctx(8, 2, 64)
+    g.plan_batch(gb, groups=groups)
+    g.debug_check_block_table(gb.block_table, gb.num_pages)
+    with pytest.raises(xb.XYAttnError):
+        g.debug_inject(-1, 0)
+    g.debug_inject(0, -1)
