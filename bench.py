@@ -109,25 +109,66 @@ def dist_env():
     return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
 
 
+def row_pairs(batch):
+    """Allowed keys of every new-token row (pure counting): kv_len + i + 1 under the causal
+    mask, kv_len + depth(i) under a tree mask (depth counts the node itself)."""
+    out = []
+    for r in range(batch.num_requests):
+        n, h = int(batch.q_len[r]), int(batch.kv_len[r])
+        par = batch.tree_parents(r)
+        if par is None:
+            out.append(h + 1 + np.arange(n, dtype=np.int64))
+        else:
+            depth = np.zeros(n, dtype=np.int64)
+            for i in range(n):
+                depth[i] = 1 if par[i] < 0 else depth[par[i]] + 1
+            out.append(h + depth)
+    return np.concatenate(out) if out else np.zeros(0, np.int64)
+
+
 def pick_sample(batch, rng, target_pairs):
-    """Rows (request, head, row) drawn in proportion to nothing in particular: uniform over
-    all (token, head) rows, until the allowed pairs reach `target_pairs`."""
+    """Rows (request, head, row) drawn uniformly over all (token, head) rows until their allowed
+    (row, key) pairs reach `target_pairs`; returns the exact pair count of the sample."""
     T, Hq = batch.total_q, batch.num_q_heads
     q_start = batch.q_start
     req_of_tok = np.repeat(np.arange(batch.num_requests), batch.q_len)
+    per_row = row_pairs(batch)
     order = rng.permutation(T * Hq)
     req, head, row, pairs = [], [], [], 0
     for x in order:
         t, a = divmod(int(x), Hq)
         r = int(req_of_tok[t])
-        i = t - int(q_start[r])
         req.append(r)
         head.append(a)
-        row.append(i)
-        pairs += int(batch.kv_len[r]) + i + 1
+        row.append(t - int(q_start[r]))
+        pairs += int(per_row[t])
         if pairs >= target_pairs:
             break
     return np.array(req, np.int32), np.array(head, np.int32), np.array(row, np.int32), pairs
+
+
+def host_cpu():
+    """Core count and model string of the host the oracle is timed on."""
+    model = "unknown"
+    try:
+        for line in open("/proc/cpuinfo"):
+            if line.lower().startswith("model name"):
+                model = line.split(":", 1)[1].strip()
+                break
+    except OSError:
+        pass
+    return {"nproc": os.cpu_count(), "model": model}
+
+
+def time_oracle_full(batch, tensors):
+    """The oracle over the whole workload, once (minutes on the large configurations)."""
+    import oracle
+    t0 = time.perf_counter()
+    oracle.attention(batch, tensors, SCALE)
+    dt = time.perf_counter() - t0
+    pairs = int(row_pairs(batch).sum()) * batch.num_q_heads
+    return {"tflops": 4.0 * batch.head_dim * pairs / dt / 1e12, "seconds": dt, "rows": batch.total_q * batch.num_q_heads,
+            "pairs": pairs, "cores": oracle.num_threads()}
 
 
 def time_oracle_sample(batch, tensors, seconds_target=12.0):
@@ -150,7 +191,7 @@ def time_oracle_sample(batch, tensors, seconds_target=12.0):
 
 
 def tree_pairs_note():
-    return "pairs counted as kv_len + row + 1 per sampled row (causal bound; tree rows see fewer)"
+    return "pairs counted exactly per sampled row (kv_len + row + 1 causal, kv_len + depth for tree rows)"
 
 
 def run_reference(args):
@@ -177,9 +218,8 @@ def run_reference(args):
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": 1e3 * secs / max(1, args.steps), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": args.workload, "num_requests": batch.num_requests,
-                   "total_q_tokens": batch.total_q},
-        "cpu_baseline": {"value": v, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
+        "config": workload_config(args.workload, batch),
+        "cpu_baseline": {"value": v, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "host": host_cpu(),
                          "sample": "%d random output rows (request, head, token) of the workload per step; %s"
                                    % (rows, tree_pairs_note())},
         "e2e": {"value": v, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -189,9 +229,59 @@ def run_reference(args):
 
 
 # DRAM bytes (read + write) of one launch of the attention meta-kernel, from the ncu captures
-# summarised under profiles/ (same workload, seed 0); None where no capture was taken.
-NCU_TRAFFIC_BYTES = {"full_mix": 6.00e9, "splitfuse_mix": 1.667e9, "verify_trees": 2.507e9, "decode_only": 0.594e9,
-                     "long_context_decode": 3.202e9}
+# summarised under profiles/ (same workload, seed 0), each stamped with the commit of the kernel
+# that was captured and the date; a kernel change that may move traffic needs a new capture.
+NCU_TRAFFIC = {
+    "full_mix": {"bytes": 6.00e9, "commit": "29136c8", "date": "2026-11-24", "summary": "profiles/launch_list_full_mix.md"},
+    "splitfuse_mix": {"bytes": 1.667e9, "commit": "29136c8", "date": "2026-11-24",
+                      "summary": "profiles/meta_attention_splitfuse_mix.md"},
+    "verify_trees": {"bytes": 2.507e9, "commit": "29136c8", "date": "2026-11-24",
+                     "summary": "profiles/meta_attention_verify_trees.md"},
+    "decode_only": {"bytes": 0.594e9, "commit": "29136c8", "date": "2026-11-24",
+                    "summary": "profiles/meta_attention_decode_only.md"},
+    "long_context_decode": {"bytes": 3.202e9, "commit": "29136c8", "date": "2026-11-24",
+                            "summary": "profiles/meta_attention_long_context_decode.md"},
+}
+
+
+def ncu_traffic(name):
+    e = NCU_TRAFFIC.get(name)
+    return (e["bytes"], "ncu capture of commit %s, %s (%s)" % (e["commit"], e["date"], e["summary"])) if e else (None, None)
+
+
+def workload_config(name, batch):
+    """The `config` object both arms print for a workload (same keys, so the two lines compare)."""
+    return {"workload": name, "num_requests": batch.num_requests, "total_q_tokens": batch.total_q,
+            "q_heads": batch.num_q_heads, "kv_heads": batch.num_kv_heads, "page_size": batch.page_size,
+            "kv_tokens": int((batch.q_len + batch.kv_len).sum())}
+
+
+def roofline_entry(flops, alg_bytes, kernel_ms, merge_ms, peaks, clocks):
+    """Everything needed to recompute a configuration's roofline fraction: the algorithmic work,
+    the measured kernel time and the fraction against every candidate peak.  The headline `frac`
+    uses the measured peak that matches the clocks seen during the timed region: the burst bf16
+    figure when the median SM clock stayed within 10 % of the maximum, else the sustained one (HBM
+    bound: the measured copy bandwidth either way)."""
+    t = kernel_ms * 1e-3
+    sm, mx = (clocks or {}).get("sm_mhz"), (clocks or {}).get("sm_max_mhz")
+    at_max = bool(sm and mx and sm >= 0.9 * mx)
+    tf_peak = peaks["bf16_tflops"] if at_max else peaks["bf16_tflops_sustained"]
+    t_flop, t_byte = flops / (tf_peak * 1e12), alg_bytes / (peaks["hbm_gbs"] * 1e9)
+    tensor = t_flop >= t_byte
+    e = {"bound": "tensor" if tensor else "hbm",
+         "achieved": flops / t / 1e12 if tensor else alg_bytes / t / 1e9,
+         "peak": tf_peak if tensor else peaks["hbm_gbs"], "unit": "TFLOP/s" if tensor else "GB/s"}
+    e["frac"] = e["achieved"] / e["peak"]
+    e["peak_source"] = "%s (%s)" % (peaks["source"], ("burst bf16: median SM clock within 10%% of max" if at_max else
+                                                     "sustained bf16: SM clock below 0.9 max") if tensor else "copy")
+    e["kernel_ms"], e["merge_ms"] = kernel_ms, merge_ms
+    e["kernel_mcycles"] = kernel_ms * 1e-3 * sm if sm else None   # duration x median SM MHz
+    e["algorithmic_flops"], e["algorithmic_bytes"] = flops, alg_bytes
+    roof = lambda tf, gb: max(flops / (tf * 1e12), alg_bytes / (gb * 1e9))
+    e["frac_burst"] = roof(peaks["bf16_tflops"], peaks["hbm_gbs"]) / t
+    e["frac_sustained"] = roof(peaks["bf16_tflops_sustained"], peaks["hbm_gbs"]) / t
+    e["frac_nominal"] = roof(NOMINAL_TFLOPS, NOMINAL_GBS) / t
+    return e
 
 
 def measure_other(name, kernel, dev, peaks, steps=20, warmup=3):
@@ -212,31 +302,35 @@ def measure_other(name, kernel, dev, peaks, steps=20, warmup=3):
     bt = torch.from_numpy(np.where(batch.block_table < 0, 0, batch.block_table).astype(np.int32)).to(dev)
     o = torch.empty((batch.total_q, batch.num_q_heads, batch.head_dim), dtype=torch.bfloat16, device=dev)
     lse = torch.empty((batch.total_q, batch.num_q_heads), dtype=torch.float32, device=dev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
     for _ in range(warmup):
         ctx.run(q, k_pool, v_pool, bt, SCALE, o, lse)
+    e1.record()
     torch.cuda.synchronize()
+    # enough steps for the clock sampler to see the timed region (about 0.4 s), at most 4000
+    steps = int(min(4000, max(steps, 400.0 / max(e0.elapsed_time(e1) / warmup, 1e-3))))
+    sampler = ClockSampler(dev.index)
+    sampler.start()
+    time.sleep(0.25)
     ctx.set_timing(True)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(steps):
         ctx.run(q, k_pool, v_pool, bt, SCALE, o, lse)
     e1.record()
     torch.cuda.synchronize()
+    clocks = sampler.stop()
     ms = e0.elapsed_time(e1) / steps
     attn_ms, merge_ms, runs = ctx.get_timing()
     assert ctx.device_status() == 0
     ctx.close()
     flops, alg = float(info.useful_flops), float(W.algorithmic_bytes(batch))
-    t_flop = flops / (peaks["bf16_tflops_sustained"] * 1e12)
-    t_byte = alg / (peaks["hbm_gbs"] * 1e9)
-    k_ms = attn_ms / max(1, runs)
-    return {"ms_per_step": ms, "tflops": flops / (ms * 1e-3) / 1e12,
-            "kv_gbs": float(info.kv_bytes) / (ms * 1e-3) / 1e9,
-            "bound": "tensor" if t_flop >= t_byte else "hbm",
-            "kernel_ms": k_ms, "merge_ms": merge_ms / max(1, runs),
-            "roofline_frac_measured": max(t_flop, t_byte) / (k_ms * 1e-3),
-            "roofline_frac_nominal": max(flops / (NOMINAL_TFLOPS * 1e12), alg / (NOMINAL_GBS * 1e9)) / (k_ms * 1e-3),
-            "steps": steps}
+    e = roofline_entry(flops, alg, attn_ms / max(1, runs), merge_ms / max(1, runs), peaks, clocks)
+    e.update({"ms_per_step": ms, "tflops": flops / (ms * 1e-3) / 1e12, "kv_gbs": float(info.kv_bytes) / (ms * 1e-3) / 1e9,
+              "steps": steps, "tasks": info.num_tasks, "merge_units": info.num_merge_units,
+              "clocks": {k: clocks.get(k) for k in ("sm_mhz", "sm_max_mhz", "reasons")}})
+    e["traffic"], e["traffic_source"] = ncu_traffic(name)
+    return e
 
 
 def measure_stream(kernel, dev, peaks, chunks=48, budget=4096, reserved=512, sessions=96, seed=0):
@@ -453,13 +547,46 @@ def measure_long_decode(kernel, dev, peaks, steps=20):
     attn_ms, merge_ms, runs = ctx.get_timing()
     assert ctx.device_status() == 0
     ctx.close()
-    assert torch.isfinite(o.float()).all() and torch.isfinite(lse).all()
+    # Every output row against the plain SIMT kernel (independent device code, same inputs), with
+    # bounds that scale with the signal: two bf16 roundings of O apart, fp32 LSE.
+    ref = xb.XYAttn(batch.num_q_heads, batch.num_kv_heads, batch.page_size, device=dev.index,
+                    kernel=xb.XY_KERNEL_REFERENCE, max_requests=256, max_q_tokens=1 << 15,
+                    max_pages_per_req=batch.block_table.shape[1])
+    ref.plan_batch(batch)
+    o_r, lse_r = torch.empty_like(o), torch.empty_like(lse)
+    ref.run(q, k_pool, v_pool, bt, SCALE, o_r, lse_r)
+    torch.cuda.synchronize()
+    ref.close()
+    err = (o.float() - o_r.float()).norm(dim=-1)
+    row_rel = float((err / (o_r.float().norm(dim=-1) + 1e-4 * 2 ** 6)).max())
+    lse_rel = float(((lse - lse_r).abs() / lse_r.abs().clamp(min=1.0)).max())
+    assert row_rel <= 2.0 ** -6 and lse_rel <= 4e-5, ("long-context decode disagrees with the SIMT kernel", row_rel, lse_rel)
     alg = float(W.algorithmic_bytes(batch))
     k_ms, m_ms = attn_ms / runs, merge_ms / runs
     return {"requests": batch.num_requests, "kv_tokens": [int(x) for x in batch.kv_len], "tasks": info.num_tasks,
             "merge_units": info.num_merge_units, "kernel_ms": k_ms, "merge_ms": m_ms,
             "kv_gbs": float(info.kv_bytes) / (k_ms * 1e-3) / 1e9, "bound": "hbm",
-            "roofline_frac_measured": alg / (peaks["hbm_gbs"] * 1e9) / (k_ms * 1e-3), "steps": steps}
+            "roofline_frac_measured": alg / (peaks["hbm_gbs"] * 1e9) / (k_ms * 1e-3), "steps": steps,
+            "check": {"against": "SIMT kernel, every row", "o_row_rel_max": row_rel, "lse_rel_max": lse_rel}}
+
+
+def self_launch(n):
+    """`--gpus N` without a launcher: start N ranks of this script, one process per GPU, with the
+    rendezvous variables torch.distributed reads; rank 0 prints the line.  NCCL's communicator log
+    (which transport and algorithms it picked) goes to stderr."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    procs = []
+    for r in range(n):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1",
+                   MASTER_PORT=str(port))
+        env.setdefault("NCCL_DEBUG", "INFO")
+        env.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__)] + sys.argv[1:], env=env,
+                                      stdout=None if r == 0 else subprocess.DEVNULL))
+    return max(p.wait() for p in procs)
 
 
 def main():
@@ -473,12 +600,16 @@ def main():
                              "prefill_prefix", "long_context_decode"])
     ap.add_argument("--kernel", default="auto", choices=["auto", "reference", "mma"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-full", action="store_true",
+                    help="time the oracle on the whole workload once instead of a bounded sample (minutes)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-others", action="store_true",
                     help="skip the short extra measurements of the other benchmark configurations")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        return self_launch(args.gpus)
 
     import torch
     import torch.distributed as dist
@@ -667,32 +798,21 @@ def main():
 
     peaks = measured_peaks()
     attn_ms_avg = attn_ms / max(1, runs)
-    t_flop = flops / (peaks["bf16_tflops_sustained"] * 1e12)
-    t_byte = alg_bytes / (peaks["hbm_gbs"] * 1e9)
-    if t_flop >= t_byte:
-        roof = {"bound": "tensor", "achieved": flops / (attn_ms_avg * 1e-3) / 1e12,
-                "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s"}
-    else:
-        roof = {"bound": "hbm", "achieved": alg_bytes / (attn_ms_avg * 1e-3) / 1e9,
-                "peak": peaks["hbm_gbs"], "unit": "GB/s"}
-    roof["frac"] = roof["achieved"] / roof["peak"]
-    roof["traffic"] = NCU_TRAFFIC_BYTES.get(args.workload)
-    roof["peak_source"] = peaks["source"] + (" (sustained bf16)" if roof["bound"] == "tensor" else " (copy)")
+    roof = roofline_entry(flops, alg_bytes, attn_ms_avg, merge_ms / max(1, runs), peaks, clocks)
+    roof["traffic"], roof["traffic_source"] = ncu_traffic(args.workload)
     roof["kernel"] = "attention meta-kernel"
-    roof["kernel_ms"] = attn_ms_avg
-    roof["merge_ms"] = merge_ms / max(1, runs)
-    roof["algorithmic_flops"] = flops
-    roof["algorithmic_bytes"] = alg_bytes
-    roof["t_roof_us_measured"] = 1e6 * max(t_flop, t_byte)
-    roof["t_roof_us_nominal"] = 1e6 * max(flops / (NOMINAL_TFLOPS * 1e12), alg_bytes / (NOMINAL_GBS * 1e9))
-    roof["frac_of_nominal_roofline"] = roof["t_roof_us_nominal"] / (attn_ms_avg * 1e3)
+    roof["workload"] = args.workload
 
     cpu = None
     if not args.no_cpu_baseline and world == 1:  # the oracle is timed at N = 1 only
-        r = time_oracle_sample(batch, tensors, 12.0)
-        cpu = {"value": r["tflops"], "unit": "TFLOP/s", "cores": r["cores"], "kind": "oracle",
-               "sample": "%d random output rows (request, head, token) of the workload, %.1f s; %s"
-                         % (r["rows"], r["seconds"], tree_pairs_note())}
+        if args.cpu_full:
+            r = time_oracle_full(batch, tensors)
+            what = "the whole workload once (%d output rows), %.1f s" % (r["rows"], r["seconds"])
+        else:
+            r = time_oracle_sample(batch, tensors, 12.0)
+            what = "%d random output rows (request, head, token) of the workload, %.1f s" % (r["rows"], r["seconds"])
+        cpu = {"value": r["tflops"], "unit": "TFLOP/s", "cores": r["cores"], "kind": "oracle", "host": host_cpu(),
+               "sample": "%s; %s" % (what, tree_pairs_note())}
 
     pool_gb = 2 * k_pool.numel() * 2 / 1e9
     others = None
@@ -700,13 +820,16 @@ def main():
         others = {}
         del q, qkv, k_pool, v_pool, o, lse, tensors
         torch.cuda.empty_cache()
+        per_config = {}
         for name in ("decode_only", "splitfuse_mix", "verify_trees", "full_mix"):
             if name == args.workload:
+                per_config[name] = "this line's primary workload: see the keys of `roofline` itself"
                 continue
             try:
-                others[name] = measure_other(name, kernel, dev, peaks)
+                per_config[name] = measure_other(name, kernel, dev, peaks)
             except Exception as e:  # report, never hide the primary line
-                others[name] = {"error": repr(e)}
+                per_config[name] = {"error": repr(e)}
+        roof["per_config"] = per_config
         try:
             torch.cuda.empty_cache()
             others["serving_stream"] = measure_stream(kernel, dev, peaks)
@@ -733,18 +856,27 @@ def main():
         "kv_gbs": kv_gbs, "n_gpus": world, "steps": args.steps, "warmup": warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": args.workload, "num_requests": batch.num_requests,
-                   "total_q_tokens": batch.total_q, "q_heads": batch.num_q_heads,
-                   "kv_heads": batch.num_kv_heads, "page_size": batch.page_size,
-                   "kv_tokens": int((batch.q_len + batch.kv_len).sum()), "kernel": args.kernel,
-                   "tasks": info.num_tasks, "merge_units": info.num_merge_units,
-                   "plan_us": plan_us, "l2": "KV pool (%.2f GB) exceeds L2; no flush" % pool_gb,
-                   "parallelism": "replicas x%d (requests sharded, no collective)" % world},
-        "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
-        "other_workloads": others,
+        "config": dict(workload_config(args.workload, batch), kernel=args.kernel, tasks=info.num_tasks,
+                       merge_units=info.num_merge_units, plan_us=plan_us,
+                       l2="KV pool (%.2f GB) exceeds L2; no flush" % pool_gb,
+                       parallelism="replicas x%d (requests sharded, no collective)" % world),
+        "other_workloads": others, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
+        "roofline": roof,
     }
-    print(json.dumps(line))
+    print(json.dumps(compact(line)))
     return 0
+
+
+def compact(x):
+    """Floats to five significant digits: the line stays short enough that its tail still holds
+    every configuration."""
+    if isinstance(x, float):
+        return float("%.5g" % x) if math.isfinite(x) else None
+    if isinstance(x, dict):
+        return {k: compact(v) for k, v in x.items()}
+    if isinstance(x, (list, tuple)):
+        return [compact(v) for v in x]
+    return x
 
 
 if __name__ == "__main__":

@@ -305,3 +305,30 @@ def test_single_long_context_is_cut_for_every_worker(hq, hkv, kv):
     assert np.array_equal(O, O2) and np.array_equal(LSE, LSE2)
     O_ref, LSE_ref = oracle.attention(b, t, H.SCALE)
     H.check_against_oracle(O, LSE, O_ref, LSE_ref, "one long context")
+
+
+@pytest.mark.parametrize("world", [2, 4])
+def test_kv_head_split_runs_on_strided_views_of_the_full_tensors(world):
+    """The tensor-parallel style sharding on one device: shard k runs the unchanged xy_attn_run
+    on kv heads [k Hkv/N, (k+1) Hkv/N) - strided views of the full pools, of Q and of O, no copies,
+    no exchange - and the shards' outputs together are the oracle's result for the whole batch."""
+    rng = np.random.default_rng(world)
+    reqs = [(90, 200, 0, None), (1, 3000, 0, None), (17, 450, 1, W.random_tree(rng, 17, 5)), (1, 0, 0, None)]
+    b = W.custom("headsplit", 16, 4, 64, reqs, seed=world)
+    t = W.make_tensors(b)
+    d = H.DeviceBatch(b, t)
+    hkv, g = 4 // world, 4
+    ctx = xb.XYAttn(hkv * g, hkv, 64, max_q_tokens=1 << 15, max_pages_per_req=1024)
+    ctx.plan_batch(b)   # the plan depends on the requests only: one plan serves every shard
+    for k in range(world):
+        hs = slice(k * hkv * g, (k + 1) * hkv * g)
+        lse_k = torch.full((b.total_q, hkv * g), float("nan"), dtype=torch.float32, device="cuda")
+        ctx.run(d.q[:, hs], d.k_pool[:, k * hkv: (k + 1) * hkv], d.v_pool[:, k * hkv: (k + 1) * hkv], d.block_table,
+                H.SCALE, d.o[:, hs], lse_k)
+        d.lse[:, hs] = lse_k
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    ctx.close()
+    O_ref, LSE_ref = oracle.attention(b, t, H.SCALE)
+    H.check_against_oracle(d.o.float().cpu().numpy().astype(np.float64), d.lse.cpu().numpy().astype(np.float64),
+                           O_ref, LSE_ref, "kv-head split")
