@@ -41,7 +41,6 @@ struct xy_attn_ctx {
   unsigned long long* d_worker_times = nullptr;
   int last_launches = 0;
   MetaLaunchCache launch_cache;     // tensor maps of the last pools seen, kernel attributes set once
-  uint32_t dbg_wait_limit = 0;      // 0: default
   int32_t dbg_skip_fill = -1;       // -1: none
   bool debug_validate = false;      // XY_ATTN_DEBUG=1 at create: block tables are range-checked before launch
   std::vector<int32_t> dbg_bt;      // host copy of the block table for that check
@@ -163,6 +162,9 @@ int xy_attn_create(const xy_attn_config* cfg, xy_attn_ctx** out) {
     alloc(reinterpret_cast<void**>(&c->d_status), 256);
     alloc(reinterpret_cast<void**>(&c->d_worker_times), sizeof(unsigned long long) * 4 * c->num_workers);
     if (e == cudaSuccess) e = cudaMemset(c->d_status, 0, 256);
+    const int32_t default_limit = 1 << 22;
+    if (e == cudaSuccess)
+      e = cudaMemcpy(c->d_status + kStatusWaitLimit, &default_limit, sizeof default_limit, cudaMemcpyHostToDevice);
     const char* dbg = getenv("XY_ATTN_DEBUG");
     c->debug_validate = dbg != nullptr && dbg[0] == '1';
     const char* tr = getenv("XY_ATTN_TRACE");
@@ -358,7 +360,6 @@ int xy_attn_run(xy_attn_ctx* ctx, const void* q, int64_t q_token_stride, const v
   // Balanced plans are dealt dynamically by the meta-kernel; paper-mode plans keep the static
   // Task-Table (each worker walks its own list), as does the reference kernel.
   a.dynamic = (cfg.plan_mode == XY_PLAN_BALANCED && cfg.kernel != XY_KERNEL_REFERENCE) ? 1 : 0;
-  a.wait_limit = ctx->dbg_wait_limit ? ctx->dbg_wait_limit : (1u << 22);
   a.debug_skip_fill = ctx->dbg_skip_fill;
   // Every run starts with a clean status word and queue head (one memset covers both): a run
   // after a device-side timeout is an ordinary run.  The sticky record (status[1]) is kept.
@@ -628,8 +629,14 @@ int xy_attn_debug_trace(xy_attn_ctx* ctx, uint64_t* out, int32_t cap) {
 
 int xy_attn_debug_inject(xy_attn_ctx* ctx, int32_t wait_limit_polls, int32_t skip_fill) {
   if (ctx == nullptr || wait_limit_polls < 0 || skip_fill < -1) return XY_ERR_INVALID_ARG;
-  ctx->dbg_wait_limit = static_cast<uint32_t>(wait_limit_polls);
   ctx->dbg_skip_fill = skip_fill;
+  if (!ctx->host_only) {
+    // the limit lives in the status block, where the kernels' waits look it up on their slow path
+    const int32_t limit = wait_limit_polls > 0 ? wait_limit_polls : (1 << 22);
+    XY_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+    XY_CUDA(ctx, cudaDeviceSynchronize());
+    XY_CUDA(ctx, cudaMemcpy(ctx->d_status + kStatusWaitLimit, &limit, sizeof limit, cudaMemcpyHostToDevice));
+  }
   return XY_OK;
 }
 

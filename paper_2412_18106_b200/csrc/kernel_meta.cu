@@ -379,7 +379,7 @@ __device__ __forceinline__ uint32_t stream_task(const RunArgs& a, const TaskView
     long long c_prev = clock64();
     ph[5] += 1;
 #endif
-    if (!dead && !mbar_wait(smem_u32(&bars->full[pipe.stage]), pipe.phase, a.status, a.wait_limit)) {
+    if (!dead && !mbar_wait_block(smem_u32(&bars->full[pipe.stage]), pipe.phase, a.status)) {
       report_timeout(a);
       dead = true;
     }
@@ -394,7 +394,7 @@ __device__ __forceinline__ uint32_t stream_task(const RunArgs& a, const TaskView
       w.softmax(a, tv.rq, s, p, col0, i_lo, i_hi, need_mask, scale_log2, lane);
     }
     XY_PH(2)
-    if (!dead && !mbar_wait(smem_u32(&bars->full[pipe.stage]), pipe.phase, a.status, a.wait_limit)) {
+    if (!dead && !mbar_wait_block(smem_u32(&bars->full[pipe.stage]), pipe.phase, a.status)) {
       report_timeout(a);
       dead = true;
     }
@@ -518,6 +518,7 @@ struct __align__(8) UmmaBarriers {
   volatile uint32_t turn;  // index of the next MMA group allowed onto the tensor pipe
 };
 
+static_assert(kStatusWaitLimit == kStatusWaitLimitWord, "one word, two names");
 static_assert(sizeof(UmmaBarriers) <= 128, "the shared-memory layout reserves 128 bytes for UmmaBarriers");
 
 template <bool kUmma>
@@ -580,7 +581,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
   auto next_task = [&](bool whole_warp) -> int {  // whole_warp: called by all 32 lanes (else by one)
     if (!dynamic) return seq_static < t_end ? seq_static++ : -1;
     const uint32_t slot = n_read % kTaskRing;
-    if (!feed_dead && !mbar_wait(smem_u32(&tq->full[slot]), (n_read / kTaskRing) & 1u, a.status, a.wait_limit)) {
+    if (!feed_dead && !mbar_wait_block(smem_u32(&tq->full[slot]), (n_read / kTaskRing) & 1u, a.status)) {
       report_timeout(a);
       feed_dead = true;
     }
@@ -627,10 +628,10 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
         if (used & bit) {
           bool ok;
           if (last_umma & bit) {
-            ok = mbar_wait(smem_u32(&bars->empty_umma[pipe.stage]), (ph_umma >> pipe.stage) & 1u, a.status, a.wait_limit);
+            ok = mbar_wait_block(smem_u32(&bars->empty_umma[pipe.stage]), (ph_umma >> pipe.stage) & 1u, a.status);
             ph_umma ^= bit;
           } else {
-            ok = mbar_wait(smem_u32(&bars->empty[pipe.stage]), (ph_cons >> pipe.stage) & 1u, a.status, a.wait_limit);
+            ok = mbar_wait_block(smem_u32(&bars->empty[pipe.stage]), (ph_cons >> pipe.stage) & 1u, a.status);
             ph_cons ^= bit;
           }
           if (!ok) {
@@ -685,7 +686,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
         if (k < a.num_tasks) ti = __ldg(a.queue + k);
         const uint32_t slot = n_pub % kTaskRing;
         if (n_pub >= kTaskRing &&
-            !mbar_wait(smem_u32(&tq->empty[slot]), ((n_pub / kTaskRing) - 1u) & 1u, a.status, a.wait_limit)) {
+            !mbar_wait_block(smem_u32(&tq->empty[slot]), ((n_pub / kTaskRing) - 1u) & 1u, a.status)) {
           report_timeout(a);
           dead = true;
         }
@@ -740,7 +741,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
       // stage has landed once its `full` phase completes (immediate on the normal path, where the
       // readers have long consumed it; a bounded wait after a failure).
       for (int s = 0; s < kStages; ++s)
-        if (used & (1u << s)) mbar_wait(smem_u32(&bars->full[s]), (fill_par >> s) & 1u, a.status, 1u << 16);
+        if (used & (1u << s)) mbar_wait_block(smem_u32(&bars->full[s]), (fill_par >> s) & 1u, a.status);
     } else if (kUmma && (warp == kConsumerWarps + 1 || warp == kConsumerWarps + 2) && lane == 0) {
       // ================================ tcgen05 MMA issuers =============================
       // One issuing thread per sub-tile (on different schedulers), each walking its own chain
@@ -753,7 +754,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
       Tracer tr;
       tr.init(a, 2, X == 0);
       auto wait_or_die = [&](uint32_t bar, uint32_t parity) {
-        if (!dead && !mbar_wait(bar, parity, a.status, a.wait_limit)) {
+        if (!dead && !mbar_wait_block(bar, parity, a.status)) {
           report_timeout(a);
           dead = true;
         }
@@ -821,7 +822,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
       auto take_turn = [&](uint32_t g) {
         if (dead) return;
         for (uint32_t spin = 0; ub->turn != g; ++spin) {
-          if (spin > a.wait_limit || ((spin & 4095u) == 4095u && *reinterpret_cast<const volatile int32_t*>(a.status) != 0)) {
+          if (spin > (1u << 22) || ((spin & 4095u) == 4095u && wait_should_give_up(a.status, spin))) {
             report_timeout(a);
             dead = true;
             return;
@@ -891,7 +892,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
       // flight then.  On the normal path they completed long ago (immediate); after a failure
       // this is a bounded wait.
       umma_commit(smem_u32(&ub->drained[X]));
-      mbar_wait(smem_u32(&ub->drained[X]), 0u, a.status, 1u << 16);
+      mbar_wait_block(smem_u32(&ub->drained[X]), 0u, a.status);
     }
   } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsConsumer));
@@ -993,7 +994,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
         for (int j = 0; j < nX; ++j) {
           const int col0 = (tv.t.kt_lo + j) * kKeyTile;
           tr(20);
-          if (!dead && !mbar_wait(smem_u32(&ub->s_full[X]), ph_s, a.status, a.wait_limit)) {
+          if (!dead && !mbar_wait_block(smem_u32(&ub->s_full[X]), ph_s, a.status)) {
             report_timeout(a);
             dead = true;
           }
@@ -1128,7 +1129,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
           tr(26);
         }
         // ---- epilogue: O / l -> global
-        if (!dead && !mbar_wait(smem_u32(&ub->o_done[X]), ph_o, a.status, a.wait_limit)) {
+        if (!dead && !mbar_wait_block(smem_u32(&ub->o_done[X]), ph_o, a.status)) {
           report_timeout(a);
           dead = true;
         }
@@ -1240,7 +1241,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
           const bool work = active && col0 <= h + i_max;  // mask-aware skip (Section 4.2.2)
           float s[16][4];
           uint32_t p[8][4];
-          if (!dead && !mbar_wait(smem_u32(&bars->full[pipe.stage]), pipe.phase, a.status, a.wait_limit)) {
+          if (!dead && !mbar_wait_block(smem_u32(&bars->full[pipe.stage]), pipe.phase, a.status)) {
             report_timeout(a);
             dead = true;
           }
@@ -1252,7 +1253,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
             const bool need_mask = tree ? (col0 + kKeyTile > h) : (col0 + kKeyTile > h + i_min + 1);
             w.softmax(a, tv.rq, s, p, col0, i_lo, i_hi, need_mask, scale_log2, lane);
           }
-          if (!dead && !mbar_wait(smem_u32(&bars->full[pipe.stage]), pipe.phase, a.status, a.wait_limit)) {
+          if (!dead && !mbar_wait_block(smem_u32(&bars->full[pipe.stage]), pipe.phase, a.status)) {
             report_timeout(a);
             dead = true;
           }

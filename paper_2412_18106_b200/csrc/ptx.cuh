@@ -39,14 +39,27 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait: gives up after `limit` polls and reports it; never spins forever.  Once any
-// thread of the grid has recorded a failure in `*status`, every other wait gives up within
-// a few thousand polls, so a broken pipeline drains quickly instead of timing out everywhere.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const volatile int32_t* status,
-                                          uint32_t limit = (1u << 22)) {
-  for (uint32_t i = 0; i < limit; ++i) {
+// Bounded waits: never spin forever.  Every 4096 polls they look at the status word the launch
+// was given: non-zero once any thread of the grid has recorded a failure, so that a broken
+// pipeline drains within a few thousand polls instead of timing out everywhere.  The hot loop
+// itself tests nothing but the barrier.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const volatile int32_t* status) {
+  for (uint32_t i = 0; i < (1u << 22); ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 4095u) == 4095u && *status != 0) return false;
+  }
+  return false;
+}
+// The same for kernels whose status is a block of words: word kStatusWaitLimitWord holds the
+// number of polls after which a wait gives up (2^22 by default; a test hook lowers it).
+constexpr int kStatusWaitLimitWord = 33;
+__device__ __forceinline__ bool wait_should_give_up(const volatile int32_t* status, uint32_t polls) {
+  return status[0] != 0 || polls >= static_cast<uint32_t>(status[kStatusWaitLimitWord]);
+}
+__device__ __forceinline__ bool mbar_wait_block(uint32_t bar, uint32_t parity, const volatile int32_t* status) {
+  for (uint32_t i = 0; i < (1u << 22); ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 4095u) == 4095u && wait_should_give_up(status, i)) return false;
   }
   return false;
 }

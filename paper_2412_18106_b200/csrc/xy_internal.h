@@ -17,6 +17,7 @@ constexpr int kStreamRowsMax = 16;
 // sticky record of failures that xy_attn_device_status reports and clears.
 constexpr int kStatusQueueHead = 16;
 constexpr int kStatusSticky = 32;
+constexpr int kStatusWaitLimit = 33;  // polls after which a bounded wait gives up (ptx.cuh reads the same word)
 constexpr int kTraceRoles = 4;      // sub-tile A, sub-tile B, MMA issuer, producer (worker 0 only)
 constexpr int kTraceLen = 2048;    // records per role and run
 
@@ -110,9 +111,7 @@ struct RunArgs {
   const int32_t* queue;
   int32_t* queue_head;
   int32_t num_tasks, dynamic;
-  // bounded waits give up after this many polls; test hook: the producer of every worker leaves
-  // out its debug_skip_fill-th stage fill (-1: none)
-  uint32_t wait_limit;
+  // test hook: the producer of every worker leaves out its debug_skip_fill-th stage fill (-1: none)
   int32_t debug_skip_fill;
 };
 

@@ -22,7 +22,7 @@ LSE_REL = 1e-3
 # row; 2^-7 = 7.8e-3 leaves a factor of five.  LSE: fp32 arithmetic in the log2 domain, observed
 # error below 2e-6 of max(1, |ref|); the bound is ten times that.
 O_ROW_REL = 2.0 ** -7
-O_ROW_ABS = 1e-4
+O_ROW_ABS = 1e-5
 LSE_REL_TIGHT = 2e-5
 
 # Largest values seen by check_against_oracle in this process (written out by conftest at exit).
@@ -84,17 +84,18 @@ def check_against_oracle(O, LSE, O_ref, LSE_ref, what="", tight=True):
     row_ref = np.sqrt((O_ref ** 2).sum(axis=-1))
     row_rel = float((row_err / (row_ref + O_ROW_ABS / O_ROW_REL)).max()) if row_err.size else 0.0
     lse_rel = float((dL / scale_l).max()) if dL.size else 0.0
-    OBSERVED["o_max_abs"] = max(OBSERVED["o_max_abs"], float(dO.max()))
-    OBSERVED["o_mean_abs"] = max(OBSERVED["o_mean_abs"], float(dO.mean()))
-    OBSERVED["o_row_rel"] = max(OBSERVED["o_row_rel"], row_rel)
-    OBSERVED["lse_rel"] = max(OBSERVED["lse_rel"], lse_rel)
-    OBSERVED["checks"] += 1
     if tight:
         bad = row_err > O_ROW_REL * row_ref + O_ROW_ABS
         assert not bad.any(), "%s: %d rows beyond the row-relative bound, worst ||dO|| = %g against ||O_ref|| = %g" % (
             what, int(bad.sum()), float(row_err[bad].max()), float(row_ref[bad][np.argmax(row_err[bad])]))
         assert np.all(dL <= LSE_REL_TIGHT * scale_l), "%s: LSE off by %g relative (tight bound %g)" % (
             what, lse_rel, LSE_REL_TIGHT)
+        # largest errors among the comparisons that passed
+        OBSERVED["o_max_abs"] = max(OBSERVED["o_max_abs"], float(dO.max()))
+        OBSERVED["o_mean_abs"] = max(OBSERVED["o_mean_abs"], float(dO.mean()))
+        OBSERVED["o_row_rel"] = max(OBSERVED["o_row_rel"], row_rel)
+        OBSERVED["lse_rel"] = max(OBSERVED["lse_rel"], lse_rel)
+        OBSERVED["checks"] += 1
     return float(dO.max()), float(dO.mean()), lse_rel
 
 
