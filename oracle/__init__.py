@@ -176,3 +176,48 @@ def append_kv(batch, qkv: torch.Tensor, k_pool: torch.Tensor, v_pool: torch.Tens
         ctypes.c_int64(qkv.stride(0)), _ptr(_u16(k_pool)), _ptr(_u16(v_pool)), ctypes.c_int64(k_pool.stride(0)),
         ctypes.c_int64(k_pool.stride(1)), ctypes.c_int64(k_pool.stride(2)), _ptr(bt), ctypes.c_int32(bt.shape[1]))
     assert rc == 0
+
+
+def e4m3_table() -> np.ndarray:
+    """The oracle's decode of all 256 e4m3 bytes (fp64; NaN at 0x7F and 0xFF)."""
+    out = np.zeros(256, dtype=np.float64)
+    assert lib().oracle_e4m3_table(_ptr(out)) == 0
+    return out
+
+
+def attention_fp8(batch, tensors, sm_scale: float, rows=None):
+    """fp8 KV-cache variant: tensors.k_pool / v_pool are uint8 e4m3 pools [P, Hkv, B, D] and
+    tensors.k_scale / v_scale fp32 [P, Hkv]; the attended values are decode(byte) * scale.
+    Whole batch -> (O [T, Hq, D], LSE [T, Hq]); with rows = (req, head, row) -> sampled outputs."""
+    k8, v8 = tensors.k_pool, tensors.v_pool
+    assert k8.dtype == torch.uint8 and v8.dtype == torch.uint8 and k8.stride() == v8.stride() and k8.stride(3) == 1
+    ks = np.ascontiguousarray(tensors.k_scale.numpy() if isinstance(tensors.k_scale, torch.Tensor) else tensors.k_scale,
+                              dtype=np.float32)
+    vs = np.ascontiguousarray(tensors.v_scale.numpy() if isinstance(tensors.v_scale, torch.Tensor) else tensors.v_scale,
+                              dtype=np.float32)
+    assert ks.shape == (k8.shape[0], batch.num_kv_heads) and vs.shape == ks.shape
+    q = tensors.q
+    assert q.stride(2) == 1 and q.stride(1) == batch.head_dim
+    ql, kl, mk, po = _i32(batch.q_len), _i32(batch.kv_len), _i32(batch.mask_kind), _i32(batch.parent_off)
+    pa = _i32(batch.parents) if batch.parents.size else np.zeros(1, np.int32)
+    bt = _i32(batch.block_table)
+    args = [ctypes.c_int(batch.num_requests), ctypes.c_int(batch.num_q_heads), ctypes.c_int(batch.num_kv_heads),
+            ctypes.c_int(batch.head_dim), ctypes.c_int(batch.page_size), _ptr(ql), _ptr(kl), _ptr(mk), _ptr(po), _ptr(pa),
+            _ptr(_u16(q)), ctypes.c_int64(q.stride(0)), ctypes.c_void_p(0), ctypes.c_void_p(0),
+            ctypes.c_int64(k8.stride(0)), ctypes.c_int64(k8.stride(1)), ctypes.c_int64(k8.stride(2)),
+            _ptr(bt), ctypes.c_int32(bt.shape[1]), ctypes.c_double(sm_scale),
+            _ptr(k8), _ptr(v8), _ptr(ks), _ptr(vs)]
+    D = batch.head_dim
+    if rows is None:
+        O = np.full((batch.total_q, batch.num_q_heads, D), np.nan, dtype=np.float64)
+        LSE = np.full((batch.total_q, batch.num_q_heads), np.nan, dtype=np.float64)
+        rc = lib().oracle_attention_fp8(*args, ctypes.c_int(-1), ctypes.c_void_p(0), ctypes.c_void_p(0),
+                                        ctypes.c_void_p(0), _ptr(O), _ptr(LSE))
+    else:
+        req, head, row = (_i32(x) for x in rows)
+        S = req.shape[0]
+        O = np.zeros((S, D), dtype=np.float64)
+        LSE = np.zeros(S, dtype=np.float64)
+        rc = lib().oracle_attention_fp8(*args, ctypes.c_int(S), _ptr(req), _ptr(head), _ptr(row), _ptr(O), _ptr(LSE))
+    assert rc == 0
+    return O, LSE

@@ -29,6 +29,14 @@
 // V); star tree; an independently written brute force; torch fp64 softmax /
 // logsumexp on gathered K/V; page-permutation invariance; key-shift identity;
 // merge identity over arbitrary partitions; GQA special cases; append-then-gather round trip.
+//
+// fp8 KV-cache variant (a variant the survey of the paper's related directions lists; the paper
+// itself defines no fp8 cache, so format, scale granularity and rounding are this build's
+// reading - parity unpinned by the paper): K and V are stored as e4m3 bytes (1 sign, 4 exponent
+// bits of bias 7, 3 mantissa bits, no infinities, 0x7F / 0xFF = NaN) with one fp32 scale per
+// (page, kv head) for K and one for V; the attended value is decode(byte) * scale, exactly, in
+// fp64, and everything after that is the same definition as above.  Pins: the 256-entry decode
+// against a library conversion; scale = 1 on values representable in e4m3 equals the bf16 path.
 
 #include <cmath>
 #include <cstdint>
@@ -50,8 +58,24 @@ inline double widen(uint16_t b) {
   return static_cast<double>(f);
 }
 
+// e4m3 ("fn" flavour) byte -> fp64, exact.  exponent field 0: subnormal m/8 * 2^-6; else
+// (1 + m/8) * 2^(e-7); exponent 15 with mantissa 7 is NaN (there are no infinities).
+inline double decode_e4m3(uint8_t b) {
+  const int sign = b >> 7, e = (b >> 3) & 15, m = b & 7;
+  double v;
+  if (e == 15 && m == 7) v = std::numeric_limits<double>::quiet_NaN();
+  else if (e == 0) v = std::ldexp(static_cast<double>(m) / 8.0, -6);
+  else v = std::ldexp(1.0 + static_cast<double>(m) / 8.0, e - 7);
+  return sign ? -v : v;
+}
+
 struct Problem {
   int R, Hq, Hkv, D, B;
+  // fp8 variant: byte pools (same strides, in elements) and per-(page, kv head) scales; null = bf16
+  const uint8_t* k8 = nullptr;
+  const uint8_t* v8 = nullptr;
+  const float* k_scale = nullptr;
+  const float* v_scale = nullptr;
   const int32_t* q_len;
   const int32_t* kv_len;
   const int32_t* mask_kind;   // 0 causal, 1 tree
@@ -93,6 +117,15 @@ inline int64_t kv_offset(const Problem& p, int r, int g, int j) {
          static_cast<int64_t>(slot) * p.token_stride;
 }
 
+// Element d of the K (which = 0) or V (which = 1) row of cached token j of request r, kv head g.
+inline double kv_elem(const Problem& p, int which, int r, int g, int j, int d) {
+  const int64_t off = kv_offset(p, r, g, j) + d;
+  if (p.k8 == nullptr) return widen((which ? p.v_pool : p.k_pool)[off]);
+  const int64_t page = p.block_table[static_cast<int64_t>(r) * p.bt_stride + j / p.B];
+  const float sc = (which ? p.v_scale : p.k_scale)[page * p.Hkv + g];
+  return decode_e4m3((which ? p.v8 : p.k8)[off]) * static_cast<double>(sc);
+}
+
 // Steps 1-3 for one (request, q head, row).  Outputs: o[D], lse, sum of p,
 // and optionally the probabilities p[0..L).
 // `keep` (nullable, u8[L]) restricts the allowed set further (used to form the
@@ -123,9 +156,8 @@ void attend_row(const Problem& p, int r, int64_t q_start, int a, int i, double* 
   double mx = -std::numeric_limits<double>::infinity();
   for (int j = 0; j < L; ++j) {
     if (!m[j]) continue;
-    const uint16_t* krow = p.k_pool + kv_offset(p, r, g, j);
     double acc = 0.0;
-    for (int d = 0; d < D; ++d) acc += widen(qrow[d]) * widen(krow[d]);
+    for (int d = 0; d < D; ++d) acc += widen(qrow[d]) * kv_elem(p, 0, r, g, j, d);
     s[j] = p.sm_scale * acc;
     if (s[j] > mx) mx = s[j];
   }
@@ -139,8 +171,7 @@ void attend_row(const Problem& p, int r, int64_t q_start, int a, int i, double* 
     double pj = 0.0;
     if (m[j]) {
       pj = std::exp(s[j] - l);
-      const uint16_t* vrow = p.v_pool + kv_offset(p, r, g, j);
-      for (int d = 0; d < D; ++d) o[d] += pj * widen(vrow[d]);
+      for (int d = 0; d < D; ++d) o[d] += pj * kv_elem(p, 1, r, g, j, d);
       ps += pj;
     }
     if (probs) probs[j] = pj;
@@ -221,6 +252,42 @@ int oracle_attention_rows(PROBLEM_ARGS, int S, const int32_t* req, const int32_t
   for (int s = 0; s < S; ++s)
     attend_row(p, req[s], q_start[req[s]], head[s], row[s], O + static_cast<int64_t>(s) * D,
                LSE + s, nullptr, nullptr);
+  return 0;
+}
+
+// fp8 KV-cache variant of the two calls above: k_pool / v_pool of PROBLEM_ARGS are ignored (pass
+// null); k8 / v8 are the byte pools with the same element strides, k_scale / v_scale fp32
+// [pages, Hkv].  rows-mode when S >= 0 (req / head / row select the outputs), whole batch when S < 0.
+int oracle_attention_fp8(PROBLEM_ARGS, const uint8_t* k8, const uint8_t* v8, const float* k_scale,
+                         const float* v_scale, int S, const int32_t* req, const int32_t* head, const int32_t* row,
+                         double* O, double* LSE) {
+  Problem p = make_problem(PROBLEM_PASS);
+  if (Hkv <= 0 || Hq % Hkv != 0 || !k8 || !v8 || !k_scale || !v_scale) return -1;
+  p.k8 = k8; p.v8 = v8; p.k_scale = k_scale; p.v_scale = v_scale;
+  std::vector<int64_t> q_start(R + 1, 0);
+  for (int r = 0; r < R; ++r) q_start[r + 1] = q_start[r] + q_len[r];
+  if (S >= 0) {
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int s = 0; s < S; ++s)
+      attend_row(p, req[s], q_start[req[s]], head[s], row[s], O + static_cast<int64_t>(s) * D, LSE + s, nullptr,
+                 nullptr);
+    return 0;
+  }
+  for (int r = 0; r < R; ++r) {
+    const int64_t units = static_cast<int64_t>(q_len[r]) * Hq;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t u = 0; u < units; ++u) {
+      const int i = static_cast<int>(u / Hq), a = static_cast<int>(u % Hq);
+      const int64_t orow = (q_start[r] + i) * Hq + a;
+      attend_row(p, r, q_start[r], a, i, O + orow * D, LSE + orow, nullptr, nullptr);
+    }
+  }
+  return 0;
+}
+
+// The 256 decoded e4m3 values (for the table pin).
+int oracle_e4m3_table(double* out) {
+  for (int b = 0; b < 256; ++b) out[b] = decode_e4m3(static_cast<uint8_t>(b));
   return 0;
 }
 

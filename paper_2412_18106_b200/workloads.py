@@ -74,6 +74,8 @@ class Tensors:
     k_pool: torch.Tensor  # bf16 [P, Hkv, B, D]
     v_pool: torch.Tensor  # bf16 [P, Hkv, B, D]
     qkv: Optional[torch.Tensor] = None  # bf16 [T, Hq + 2 Hkv, D] when fused
+    k_scale: Optional[torch.Tensor] = None  # fp8 KV cache: fp32 [P, Hkv]; the pools are then uint8 e4m3 bytes
+    v_scale: Optional[torch.Tensor] = None
 
 
 def _pages_needed(q_len, kv_len, page_size):
@@ -363,6 +365,23 @@ def make_tensors(batch: Batch, seed: Optional[int] = None, fused_qkv: bool = Fal
             k_pool[unused] = tail_fill
             v_pool[unused] = -tail_fill
     return Tensors(q=q, k_pool=k_pool, v_pool=v_pool, qkv=qkv)
+
+
+def to_fp8_kv(tensors: Tensors, unit_scale: bool = False) -> Tensors:
+    """Inputs for the fp8 KV-cache variant: the K and V pools as e4m3 bytes with one fp32 scale
+    per (page, kv head), chosen so that the page's largest magnitude maps to 448 (or scale = 1
+    with `unit_scale`).  The cast is the library's (torch.float8_e4m3fn); what the attention
+    kernels and the oracle receive are the bytes and the scales."""
+    out = []
+    for pool in (tensors.k_pool, tensors.v_pool):
+        x = pool.float()
+        if unit_scale:
+            scale = torch.ones(x.shape[:2], dtype=torch.float32)
+        else:
+            scale = (x.abs().amax(dim=(2, 3)) / 448.0).clamp_min(2.0 ** -20)
+        q = (x / scale[:, :, None, None]).to(torch.float8_e4m3fn)
+        out.append((q.view(torch.uint8), scale.contiguous()))
+    return Tensors(q=tensors.q, k_pool=out[0][0], v_pool=out[1][0], qkv=tensors.qkv, k_scale=out[0][1], v_scale=out[1][1])
 
 
 def set_tile_onehot_v(batch: Batch, tensors: Tensors, tile: int = 128) -> None:

@@ -20,10 +20,10 @@ LSE_REL = 1e-3
 # ||O_ref||_2 + O_ROW_ABS.  Arithmetic behind it: P and O are each rounded once to bf16 (relative
 # error uniform in +-2^-9, rms 2^-9 / sqrt 3 = 1.1e-3 each), which gives about 1.6e-3 relative per
 # row; 2^-7 = 7.8e-3 leaves a factor of five.  LSE: fp32 arithmetic in the log2 domain, observed
-# error below 2e-6 of max(1, |ref|); the bound is ten times that.
+# error 3.5e-7 of max(1, |ref|) over the whole GPU suite; the bound is about ten times that.
 O_ROW_REL = 2.0 ** -7
 O_ROW_ABS = 1e-5
-LSE_REL_TIGHT = 2e-5
+LSE_REL_TIGHT = 5e-6
 
 # Largest values seen by check_against_oracle in this process (written out by conftest at exit).
 OBSERVED = {"o_max_abs": 0.0, "o_mean_abs": 0.0, "o_row_rel": 0.0, "lse_rel": 0.0, "checks": 0}
