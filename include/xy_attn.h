@@ -68,6 +68,12 @@ enum {
                            worker runs its own list */
 };
 
+/* Element type of the paged K/V cache. */
+enum {
+  XY_KV_BF16 = 0,     /* bf16 pools, xy_attn_run (the paper's cache) */
+  XY_KV_FP8_E4M3 = 1  /* e4m3 byte pools with fp32 scales per (page, kv head), xy_attn_run_fp8kv */
+};
+
 typedef struct {
   int32_t num_q_heads;       /* Hq */
   int32_t num_kv_heads;      /* Hkv, divides Hq; q head a reads kv head a / (Hq/Hkv) */
@@ -84,6 +90,7 @@ typedef struct {
   int32_t tile_tokens;       /* XY_PLAN_PAPER only: tileSize in tokens (0 = 128 / (Hq/Hkv)) */
   int32_t max_splits;        /* upper bound on KV splits of one tile unit (0 = 32, or up to 128 when so few
                               * streaming units exist that 32 splits each would leave workers idle) */
+  int32_t kv_dtype;          /* XY_KV_*: decides which run call the context serves (and the tile plan) */
   int64_t workspace_bytes;   /* split-KV workspace (fp32 partial O and LSE); 0 = 256 MiB */
 } xy_attn_config;
 
@@ -219,6 +226,28 @@ int xy_attn_run(xy_attn_ctx* ctx, const void* q, int64_t q_token_stride, const v
                 int64_t token_stride, const int32_t* block_table, int32_t block_table_stride,
                 const uint64_t* tree_mask, float sm_scale, void* o, int64_t o_token_stride,
                 float* lse, void* stream);
+
+/* Meta-Attention over an fp8 KV cache.  The paper's cache is bf16; an fp8 cache is a variant the
+ * related-work directions name, and nothing in the paper fixes its format, so this is the
+ * library's own definition: K and V are stored as e4m3 bytes (1 sign, 4 exponent bits of bias 7,
+ * 3 mantissa bits, no infinities, 0x7F / 0xFF = NaN: never store those) and the attended value
+ * is  decode(byte) * scale[page][kv_head]  with one fp32 scale per page and kv head, K and V
+ * separately.  Everything else - requests, masks, block tables, Q, O, LSE - is as in xy_attn_run,
+ * and the context must have been created with kv_dtype = XY_KV_FP8_E4M3 (xy_attn_run then
+ * returns XY_ERR_UNSUPPORTED, and so does this call on a bf16 context).
+ *   k_pool/v_pool  DEVICE uint8 [num_pages, Hkv, B, D]; strides in elements (= bytes), multiples
+ *                  of 16; D contiguous
+ *   k_scale/v_scale DEVICE fp32 [num_pages, Hkv], contiguous, finite and positive
+ * Requires page_size >= 16.  Widening e4m3 to f16 is exact; Q is used as f16 after a per-row
+ * power-of-two factor (exact for every element within 2^-14 of its row's largest); scores, the
+ * softmax and O accumulate in fp32; P is rounded to f16.  Dense tiles run on the warp-level MMA
+ * path in this variant.  xy_attn_append_kv and xy_attn_debug_gather do not serve fp8 contexts
+ * (quantising on append needs a scale policy that the caller owns). */
+int xy_attn_run_fp8kv(xy_attn_ctx* ctx, const void* q, int64_t q_token_stride, const void* k_pool,
+                      const void* v_pool, const float* k_scale, const float* v_scale, int64_t num_pages,
+                      int64_t page_stride, int64_t head_stride, int64_t token_stride,
+                      const int32_t* block_table, int32_t block_table_stride, const uint64_t* tree_mask,
+                      float sm_scale, void* o, int64_t o_token_stride, float* lse, void* stream);
 
 /* KV-cache append with fused QKV split (the step before attention: Sections 4.1.1 and 5.4).
  * For every planned request r and new token i the K and V head rows of the fused tensor

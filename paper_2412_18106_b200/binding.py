@@ -35,12 +35,15 @@ XY_KERNEL_MMA = 2
 XY_PLAN_BALANCED = 0
 XY_PLAN_PAPER = 1
 
+XY_KV_BF16 = 0
+XY_KV_FP8_E4M3 = 1
+
 
 class xy_attn_config(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in (
         "num_q_heads", "num_kv_heads", "head_dim", "page_size", "max_requests", "max_q_tokens",
         "max_pages_per_req", "max_tree_nodes", "device", "num_workers", "kernel", "plan_mode",
-        "tile_tokens", "max_splits")] + [("workspace_bytes", ctypes.c_int64)]
+        "tile_tokens", "max_splits", "kv_dtype")] + [("workspace_bytes", ctypes.c_int64)]
 
 
 class xy_attn_request(ctypes.Structure):
@@ -83,6 +86,7 @@ EXPORTS = (
     "xy_attn_append_kv", "xy_attn_worker_times", "xy_attn_get_queue", "xy_attn_plan_cache",
     "xy_attn_plan_shared", "xy_attn_shard_context", "xy_attn_merge_shards",
     "xy_attn_find_prefix_groups", "xy_attn_debug_check_block_table", "xy_attn_debug_inject",
+    "xy_attn_run_fp8kv",
 )
 
 _lib = None
@@ -105,6 +109,8 @@ def load() -> ctypes.CDLL:
     L.xy_attn_plan_shared.argtypes = [vp, vp, i32, vp, i32, vp, i32, vp, ctypes.POINTER(xy_attn_plan_info)]
     L.xy_attn_run.argtypes = [vp, vp, i64, vp, vp, i64, i64, i64, i64, vp, i32, vp, ctypes.c_float,
                               vp, i64, vp, vp]
+    L.xy_attn_run_fp8kv.argtypes = [vp, vp, i64, vp, vp, vp, vp, i64, i64, i64, i64, vp, i32, vp, ctypes.c_float,
+                                    vp, i64, vp, vp]
     L.xy_attn_merge.argtypes = [vp, vp, i32, i64, i32, vp, vp, vp]
     L.xy_attn_merge_shards.argtypes = [vp, vp, i32, i64, i32, vp, vp, vp]
     L.xy_attn_find_prefix_groups.argtypes = [vp, i32, vp, i32, i32, i32, i32, vp, i32, ctypes.POINTER(i32)]
@@ -156,11 +162,11 @@ class XYAttn:
                  max_requests: int = 256, max_q_tokens: int = 1 << 15, max_pages_per_req: int = 1024,
                  max_tree_nodes: int = 64, device: int = 0, num_workers: int = 0,
                  kernel: int = XY_KERNEL_AUTO, plan_mode: int = XY_PLAN_BALANCED, tile_tokens: int = 0,
-                 max_splits: int = 0, workspace_bytes: int = 0):
+                 max_splits: int = 0, workspace_bytes: int = 0, kv_dtype: int = XY_KV_BF16):
         self.lib = load()
         self.cfg = xy_attn_config(num_q_heads, num_kv_heads, head_dim, page_size, max_requests,
                                   max_q_tokens, max_pages_per_req, max_tree_nodes, device, num_workers,
-                                  kernel, plan_mode, tile_tokens, max_splits, workspace_bytes)
+                                  kernel, plan_mode, tile_tokens, max_splits, kv_dtype, workspace_bytes)
         self._ctx = ctypes.c_void_p(0)
         rc = self.lib.xy_attn_create(ctypes.byref(self.cfg), ctypes.byref(self._ctx))
         if rc != XY_OK:
@@ -248,6 +254,30 @@ class XYAttn:
         self._check(self.lib.xy_attn_run(
             self._ctx, q.data_ptr(), q.stride(0), k_pool.data_ptr(), v_pool.data_ptr(),
             k_pool.shape[0], k_pool.stride(0), k_pool.stride(1), k_pool.stride(2),
+            block_table.data_ptr(), block_table.stride(0), tm, float(sm_scale), o.data_ptr(),
+            o.stride(0), lse.data_ptr(), _stream_ptr(stream)))
+
+    # -- xy_attn_run_fp8kv
+    def run_fp8kv(self, q: torch.Tensor, k_pool: torch.Tensor, v_pool: torch.Tensor, k_scale: torch.Tensor,
+                  v_scale: torch.Tensor, block_table: torch.Tensor, sm_scale: float, o: torch.Tensor,
+                  lse: torch.Tensor, tree_mask: Optional[torch.Tensor] = None, stream=None) -> None:
+        """k_pool / v_pool uint8 (e4m3 bytes) [P, Hkv, B, D], k_scale / v_scale fp32 [P, Hkv]."""
+        for t in (q, k_pool, v_pool, k_scale, v_scale, block_table, o, lse):
+            if not t.is_cuda:
+                raise XYAttnError(XY_ERR_INVALID_ARG, "run_fp8kv needs CUDA tensors (there is no CPU path)")
+        assert q.dtype == torch.bfloat16 and k_pool.dtype == torch.uint8 and v_pool.dtype == torch.uint8
+        assert k_scale.dtype == torch.float32 and v_scale.dtype == torch.float32
+        assert k_scale.is_contiguous() and v_scale.is_contiguous() and k_scale.shape == (k_pool.shape[0], k_pool.shape[1])
+        assert v_scale.shape == k_scale.shape
+        assert o.dtype == torch.bfloat16 and lse.dtype == torch.float32 and block_table.dtype == torch.int32
+        assert q.stride(2) == 1 and q.stride(1) == self.cfg.head_dim
+        assert o.stride(2) == 1 and o.stride(1) == self.cfg.head_dim and lse.is_contiguous()
+        assert k_pool.stride() == v_pool.stride() and k_pool.stride(3) == 1
+        assert block_table.stride(1) == 1
+        tm = ctypes.c_void_p(tree_mask.data_ptr()) if tree_mask is not None else ctypes.c_void_p(0)
+        self._check(self.lib.xy_attn_run_fp8kv(
+            self._ctx, q.data_ptr(), q.stride(0), k_pool.data_ptr(), v_pool.data_ptr(), k_scale.data_ptr(),
+            v_scale.data_ptr(), k_pool.shape[0], k_pool.stride(0), k_pool.stride(1), k_pool.stride(2),
             block_table.data_ptr(), block_table.stride(0), tm, float(sm_scale), o.data_ptr(),
             o.stride(0), lse.data_ptr(), _stream_ptr(stream)))
 

@@ -106,6 +106,8 @@ int xy_attn_create(const xy_attn_config* cfg, xy_attn_ctx** out) {
     return XY_ERR_INVALID_ARG;
   if (cfg->kernel < XY_KERNEL_AUTO || cfg->kernel > XY_KERNEL_MMA) return XY_ERR_INVALID_ARG;
   if (cfg->plan_mode != XY_PLAN_BALANCED && cfg->plan_mode != XY_PLAN_PAPER) return XY_ERR_INVALID_ARG;
+  if (cfg->kv_dtype != XY_KV_BF16 && cfg->kv_dtype != XY_KV_FP8_E4M3) return XY_ERR_INVALID_ARG;
+  if (cfg->kv_dtype == XY_KV_FP8_E4M3 && cfg->page_size < 16) return XY_ERR_UNSUPPORTED;
 
   xy_attn_ctx* c = new (std::nothrow) xy_attn_ctx();
   if (c == nullptr) return XY_ERR_INVALID_ARG;
@@ -285,15 +287,23 @@ int xy_attn_debug_check_block_table(xy_attn_ctx* ctx, const int32_t* block_table
   return XY_OK;
 }
 
-int xy_attn_run(xy_attn_ctx* ctx, const void* q, int64_t q_token_stride, const void* k_pool,
-                const void* v_pool, int64_t num_pages, int64_t page_stride, int64_t head_stride,
-                int64_t token_stride, const int32_t* block_table, int32_t block_table_stride,
-                const uint64_t* tree_mask, float sm_scale, void* o, int64_t o_token_stride,
-                float* lse, void* stream) {
+}  // extern "C"
+
+namespace {
+
+// The body of xy_attn_run and xy_attn_run_fp8kv (k_scale / v_scale null: bf16 pools).
+int run_impl(xy_attn_ctx* ctx, const void* q, int64_t q_token_stride, const void* k_pool,
+             const void* v_pool, const float* k_scale, const float* v_scale, int64_t num_pages, int64_t page_stride,
+             int64_t head_stride, int64_t token_stride, const int32_t* block_table, int32_t block_table_stride,
+             const uint64_t* tree_mask, float sm_scale, void* o, int64_t o_token_stride,
+             float* lse, void* stream) {
   if (ctx == nullptr) return XY_ERR_INVALID_ARG;
   ctx->last_launches = 0;
   if (ctx->host_only) return set_err(ctx, XY_ERR_UNSUPPORTED, "host-only context cannot run");
   if (!ctx->planned) return set_err(ctx, XY_ERR_NOT_PLANNED, "xy_attn_run before xy_attn_plan");
+  const bool fp8 = k_scale != nullptr;
+  if (fp8 != (ctx->cfg.kv_dtype == XY_KV_FP8_E4M3))
+    return set_err(ctx, XY_ERR_UNSUPPORTED, "the context's kv_dtype does not match this run call");
   const PlanResult& p = ctx->plan;
   if (p.tasks.empty()) return XY_OK;
   const xy_attn_config& cfg = ctx->cfg;
@@ -305,9 +315,11 @@ int xy_attn_run(xy_attn_ctx* ctx, const void* q, int64_t q_token_stride, const v
   if (q_token_stride < static_cast<int64_t>(cfg.num_q_heads) * kHeadDim || q_token_stride % 8 != 0 ||
       o_token_stride < static_cast<int64_t>(cfg.num_q_heads) * kHeadDim || o_token_stride % 8 != 0)
     return set_err(ctx, XY_ERR_INVALID_ARG, "token stride of q / o too small or not a multiple of 8");
-  if (token_stride < kHeadDim || token_stride % 8 != 0 || head_stride % 8 != 0 || head_stride < 1 ||
-      page_stride % 8 != 0 || page_stride < 1 || num_pages < 1)
+  const int64_t sa = fp8 ? 16 : 8;  // strides must keep every row 16-byte aligned
+  if (token_stride < kHeadDim || token_stride % sa != 0 || head_stride % sa != 0 || head_stride < 1 ||
+      page_stride % sa != 0 || page_stride < 1 || num_pages < 1)
     return set_err(ctx, XY_ERR_INVALID_ARG, "bad K/V pool strides or num_pages");
+  if (fp8 && v_scale == nullptr) return set_err(ctx, XY_ERR_INVALID_ARG, "null scale pointer");
   if (block_table_stride < 1) return set_err(ctx, XY_ERR_INVALID_ARG, "bad block_table_stride");
   if (!(sm_scale > 0.f) || !(sm_scale < 1e30f))
     return set_err(ctx, XY_ERR_INVALID_ARG, "sm_scale must be positive and finite");
@@ -361,6 +373,9 @@ int xy_attn_run(xy_attn_ctx* ctx, const void* q, int64_t q_token_stride, const v
   // Task-Table (each worker walks its own list), as does the reference kernel.
   a.dynamic = (cfg.plan_mode == XY_PLAN_BALANCED && cfg.kernel != XY_KERNEL_REFERENCE) ? 1 : 0;
   a.debug_skip_fill = ctx->dbg_skip_fill;
+  a.k_scale = k_scale;
+  a.v_scale = v_scale;
+  a.kv_fp8 = fp8 ? 1 : 0;
   // Every run starts with a clean status word and queue head (one memset covers both): a run
   // after a device-side timeout is an ordinary run.  The sticky record (status[1]) is kept.
   XY_CUDA(ctx, cudaMemsetAsync(a.status, 0, 17 * sizeof(int32_t), s));
@@ -410,6 +425,30 @@ int xy_attn_run(xy_attn_ctx* ctx, const void* q, int64_t q_token_stride, const v
   return XY_OK;
 }
 
+}  // namespace
+
+extern "C" {
+
+int xy_attn_run(xy_attn_ctx* ctx, const void* q, int64_t q_token_stride, const void* k_pool,
+                const void* v_pool, int64_t num_pages, int64_t page_stride, int64_t head_stride,
+                int64_t token_stride, const int32_t* block_table, int32_t block_table_stride,
+                const uint64_t* tree_mask, float sm_scale, void* o, int64_t o_token_stride,
+                float* lse, void* stream) {
+  return run_impl(ctx, q, q_token_stride, k_pool, v_pool, nullptr, nullptr, num_pages, page_stride, head_stride,
+                  token_stride, block_table, block_table_stride, tree_mask, sm_scale, o, o_token_stride, lse, stream);
+}
+
+int xy_attn_run_fp8kv(xy_attn_ctx* ctx, const void* q, int64_t q_token_stride, const void* k_pool,
+                      const void* v_pool, const float* k_scale, const float* v_scale, int64_t num_pages,
+                      int64_t page_stride, int64_t head_stride, int64_t token_stride,
+                      const int32_t* block_table, int32_t block_table_stride, const uint64_t* tree_mask,
+                      float sm_scale, void* o, int64_t o_token_stride, float* lse, void* stream) {
+  if (ctx == nullptr) return XY_ERR_INVALID_ARG;
+  if (k_scale == nullptr || v_scale == nullptr) return set_err(ctx, XY_ERR_INVALID_ARG, "null scale pointer");
+  return run_impl(ctx, q, q_token_stride, k_pool, v_pool, k_scale, v_scale, num_pages, page_stride, head_stride,
+                  token_stride, block_table, block_table_stride, tree_mask, sm_scale, o, o_token_stride, lse, stream);
+}
+
 int xy_attn_set_timing(xy_attn_ctx* ctx, int32_t enable) {
   if (ctx == nullptr) return XY_ERR_INVALID_ARG;
   if (ctx->host_only) return set_err(ctx, XY_ERR_UNSUPPORTED, "host-only context");
@@ -445,6 +484,7 @@ int xy_attn_append_kv(xy_attn_ctx* ctx, const void* qkv, int64_t qkv_token_strid
                       const int32_t* block_table, int32_t block_table_stride, void* stream) {
   if (ctx == nullptr) return XY_ERR_INVALID_ARG;
   if (ctx->host_only) return set_err(ctx, XY_ERR_UNSUPPORTED, "host-only context cannot run");
+  if (ctx->cfg.kv_dtype != XY_KV_BF16) return set_err(ctx, XY_ERR_UNSUPPORTED, "append serves bf16 caches only");
   if (!ctx->planned) return set_err(ctx, XY_ERR_NOT_PLANNED, "xy_attn_append_kv before xy_attn_plan");
   const PlanResult& p = ctx->plan;
   if (p.total_q == 0) return XY_OK;
@@ -561,6 +601,7 @@ int xy_attn_debug_gather(xy_attn_ctx* ctx, int32_t req, int32_t kv_head, const v
                          int32_t block_table_stride, void* out_k, void* out_v, void* stream) {
   if (ctx == nullptr) return XY_ERR_INVALID_ARG;
   if (ctx->host_only) return set_err(ctx, XY_ERR_UNSUPPORTED, "host-only context cannot run");
+  if (ctx->cfg.kv_dtype != XY_KV_BF16) return set_err(ctx, XY_ERR_UNSUPPORTED, "gather serves bf16 caches only");
   if (!ctx->planned) return set_err(ctx, XY_ERR_NOT_PLANNED, "gather before plan");
   if (req < 0 || req >= static_cast<int32_t>(ctx->plan.reqs.size()) || kv_head < 0 ||
       kv_head >= ctx->cfg.num_kv_heads || !k_pool || !v_pool || !block_table || !out_k || !out_v)

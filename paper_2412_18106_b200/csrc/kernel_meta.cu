@@ -59,7 +59,9 @@ struct __align__(8) SmemBarriers {
 constexpr int kSmemQ = 2 * kTileBytes;
 constexpr int kSmemRing = kStages * kTileBytes;
 constexpr int kSmemMl = kConsumerWarps * 16 * 2 * 4;
-constexpr int kSmemTotal = 1024 /*align slack*/ + kSmemQ + kSmemRing + kSmemMl + sizeof(SmemBarriers) + 128 + 256;
+constexpr int kSmemFp8 = 1024;  // fp8 KV path: per-row Q factors [128] and a ring of per-tile page scales [8][16]
+constexpr int kScaleSlots = 8;
+constexpr int kSmemTotal = 1024 /*align slack*/ + kSmemQ + kSmemRing + kSmemMl + sizeof(SmemBarriers) + 128 + 256 + kSmemFp8;
 
 __device__ __forceinline__ uint32_t swz(uint32_t row, uint32_t chunk16 /*0..15*/) {
   return (chunk16 >> 3) * kHalfBytes + row * 128u + (((chunk16 & 7u) ^ (row & 7u)) << 4);
@@ -93,7 +95,20 @@ __device__ __forceinline__ bool visible(const RunArgs& a, const ReqInfo& rq, int
 // every 128-key tile).  Keeps m (log2 domain), l (thread-partial) and O in registers.
 // KEEPQ: Q fragments stay in registers for the whole task (streaming); otherwise they are
 // re-read from shared memory at every k-step to leave registers for the 128-key score tile.
-template <int NT, bool KEEPQ>
+// F16: operands are f16 (the fp8 KV-cache path: K / V widened exactly from e4m3, Q converted with a
+// power-of-two factor per row) and the scores carry per-row and per-page factors (FpScale).
+struct FpScale {
+  float q_lo, q_hi;        // 2^e of the two rows this thread holds: undoes the row's Q pre-scaling
+  const float* tile;       // shared memory: [0..7] K scale, [8..15] V scale of the tile's pages
+  int page_shift;
+};
+
+template <bool F16>
+__device__ __forceinline__ void mma16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  if constexpr (F16) mma_f16_16816(c, a, b0, b1); else mma_bf16_16816(c, a, b0, b1);
+}
+
+template <int NT, bool KEEPQ, bool F16 = false>
 struct WarpTile {
   float o[16][4];
   float m_lo, m_hi, l_lo, l_hi;
@@ -154,10 +169,10 @@ struct WarpTile {
       for (int ks = 0; ks < 8; ks += 2) {
         const uint32_t(&qa)[4] = KEEPQ ? qf[KEEPQ ? ks : 0] : qq[ks];
         const uint32_t(&qb)[4] = KEEPQ ? qf[KEEPQ ? ks + 1 : 0] : qq[ks + 1];
-        mma_bf16_16816(s[0], qa, kb[ks][0], kb[ks][1]);
-        mma_bf16_16816(s[1], qa, kb[ks][2], kb[ks][3]);
-        mma_bf16_16816(t[0], qb, kb[ks + 1][0], kb[ks + 1][1]);
-        mma_bf16_16816(t[1], qb, kb[ks + 1][2], kb[ks + 1][3]);
+        mma16816<F16>(s[0], qa, kb[ks][0], kb[ks][1]);
+        mma16816<F16>(s[1], qa, kb[ks][2], kb[ks][3]);
+        mma16816<F16>(t[0], qb, kb[ks + 1][0], kb[ks + 1][1]);
+        mma16816<F16>(t[1], qb, kb[ks + 1][2], kb[ks + 1][3]);
       }
 #pragma unroll
       for (int n = 0; n < 2; ++n)
@@ -183,22 +198,30 @@ struct WarpTile {
         const uint32_t key = koff + np * 16 + (lane & 7) + (mi >> 1) * 8;
         uint32_t b0, b1, b2, b3;
         ldmatrix_x4(k_smem + swz(key, ks * 2 + (mi & 1)), b0, b1, b2, b3);
-        mma_bf16_16816(s[2 * np], qa, b0, b1);
-        mma_bf16_16816(s[2 * np + 1], qa, b2, b3);
+        mma16816<F16>(s[2 * np], qa, b0, b1);
+        mma16816<F16>(s[2 * np + 1], qa, b2, b3);
       }
     }
   }
 
   // Mask + online softmax (Update rescale) on s; leaves P (bf16 A fragments) in p.
+  // koff: key offset of s[0] inside the 128-key tile (selects the page whose scales apply)
   __device__ __forceinline__ void softmax(const RunArgs& a, const ReqInfo& rq, float (&s)[NT][4],
                                           uint32_t (&p)[NT / 2][4], int col0, int i_lo, int i_hi,
-                                          bool need_mask, float scale_log2, int lane) {
+                                          bool need_mask, float scale_log2, int lane, const FpScale* fs = nullptr,
+                                          int koff = 0) {
     float mx_lo = -INFINITY, mx_hi = -INFINITY;
 #pragma unroll
     for (int n = 0; n < NT; ++n) {
+      float f_lo = scale_log2, f_hi = scale_log2;
+      if constexpr (F16) {
+        const float ks = fs->tile[(koff + n * 8) >> fs->page_shift];
+        f_lo = scale_log2 * fs->q_lo * ks;
+        f_hi = scale_log2 * fs->q_hi * ks;
+      }
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        float v = s[n][e] * scale_log2;
+        float v = s[n][e] * ((e < 2) ? f_lo : f_hi);
         if (need_mask) {
           const int col = col0 + n * 8 + 2 * (lane & 3) + (e & 1);
           if (!visible(a, rq, (e < 2) ? i_lo : i_hi, col)) v = -INFINITY;
@@ -241,8 +264,15 @@ struct WarpTile {
       sum_lo += p0 + p1;
       sum_hi += p2 + p3;
       // A fragment of k-step n/2: a0,a1 from the even n-tile, a2,a3 from the odd one
-      p[n >> 1][(n & 1) * 2 + 0] = pack_bf16(p0, p1);
-      p[n >> 1][(n & 1) * 2 + 1] = pack_bf16(p2, p3);
+      if constexpr (F16) {
+        // the V scale of the key's page rides on P (l keeps the unscaled sum)
+        const float vs = fs->tile[8 + ((koff + n * 8) >> fs->page_shift)];
+        p[n >> 1][(n & 1) * 2 + 0] = pack_f16(p0 * vs, p1 * vs);
+        p[n >> 1][(n & 1) * 2 + 1] = pack_f16(p2 * vs, p3 * vs);
+      } else {
+        p[n >> 1][(n & 1) * 2 + 0] = pack_bf16(p0, p1);
+        p[n >> 1][(n & 1) * 2 + 1] = pack_bf16(p2, p3);
+      }
     }
     l_lo += sum_lo;
     l_hi += sum_hi;
@@ -259,8 +289,8 @@ struct WarpTile {
         ldmatrix_x4_trans(v_smem + swz(key, dp * 2 + (mi >> 1)), vb[dp][0], vb[dp][1], vb[dp][2], vb[dp][3]);
 #pragma unroll
       for (int dp = 0; dp < 8; ++dp) {
-        mma_bf16_16816(o[2 * dp], p[0], vb[dp][0], vb[dp][1]);
-        mma_bf16_16816(o[2 * dp + 1], p[0], vb[dp][2], vb[dp][3]);
+        mma16816<F16>(o[2 * dp], p[0], vb[dp][0], vb[dp][1]);
+        mma16816<F16>(o[2 * dp + 1], p[0], vb[dp][2], vb[dp][3]);
       }
       return;
     }
@@ -271,8 +301,8 @@ struct WarpTile {
       for (int dp = 0; dp < 8; ++dp) {
         uint32_t b0, b1, b2, b3;
         ldmatrix_x4_trans(v_smem + swz(key, dp * 2 + (mi >> 1)), b0, b1, b2, b3);
-        mma_bf16_16816(o[2 * dp], p[kk], b0, b1);
-        mma_bf16_16816(o[2 * dp + 1], p[kk], b2, b3);
+        mma16816<F16>(o[2 * dp], p[kk], b0, b1);
+        mma16816<F16>(o[2 * dp + 1], p[kk], b2, b3);
       }
     }
   }
@@ -284,6 +314,73 @@ struct WarpTile {
     l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
   }
 };
+
+// ------------------------------------------------------------------------------------------
+// fp8 KV-cache path (a variant beside the paper's bf16 cache; Section 4.1.1's paged layout with
+// e4m3 bytes and one fp32 scale per page and kv head).  A 128-key tile arrives as 16 KiB of
+// bytes in the upper half of its 32 KiB stage (row = key, 128 B, 16-byte chunks XOR-swizzled by
+// row like every other tile); the warp that is going to read 16 of its rows first widens them in
+// place to the f16 tile layout (exact: every e4m3 value is an f16 value).  Two lanes share a row;
+// the upper-half destination of a row is the very line its bytes came from, hence the warp-wide
+// barrier between the loads and the stores.
+__device__ __forceinline__ void widen_rows16(uint32_t stage, int row0, int lane) {
+  const uint32_t row = row0 + (lane >> 1), half = lane & 1u, r7 = row & 7u;
+  const uint32_t src = stage + kHalfBytes + row * 128u;
+  uint4 in[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) in[q] = lds128(src + (((half * 4u + q) ^ r7) << 4));
+  // the partner lane's source chunks lie in the line this lane is about to overwrite (and vice versa)
+  asm volatile("" ::"r"(in[0].x), "r"(in[1].x), "r"(in[2].x), "r"(in[3].x), "r"(in[0].w), "r"(in[1].w), "r"(in[2].w),
+               "r"(in[3].w));
+  __syncwarp();
+  const uint32_t dst = stage + half * kHalfBytes + row * 128u;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const uint32_t w[4] = {in[q].x, in[q].y, in[q].z, in[q].w};
+    uint32_t h[8];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      h[2 * k] = e4m3x2_to_f16x2(static_cast<uint16_t>(w[k] & 0xFFFFu));
+      h[2 * k + 1] = e4m3x2_to_f16x2(static_cast<uint16_t>(w[k] >> 16));
+    }
+    sts128(dst + ((static_cast<uint32_t>(2 * q) ^ r7) << 4), make_uint4(h[0], h[1], h[2], h[3]));
+    sts128(dst + ((static_cast<uint32_t>(2 * q + 1) ^ r7) << 4), make_uint4(h[4], h[5], h[6], h[7]));
+  }
+  __syncwarp();
+}
+
+// Q rows of the tile in shared memory, bf16 -> f16 in place, each row multiplied by a power of two
+// that brings its largest element below 4 (exact in f16 for every element within 2^-14 of the
+// row's largest; bf16's exponent range does not fit f16 otherwise).  qmult[row] receives the
+// inverse factor, which the softmax folds into the score scale.  kLanesPerRow lanes share a row.
+template <int kLanesPerRow>
+__device__ __forceinline__ void q_rows_to_f16(uint32_t q_smem, int row0, float* qmult, int lane) {
+  constexpr int kChunks = 16 / kLanesPerRow;  // 16-byte chunks (8 elements) per lane
+  const uint32_t row = row0 + lane / kLanesPerRow, c0 = (lane % kLanesPerRow) * kChunks;
+  uint4 v[kChunks];
+  uint32_t emax = 0;
+#pragma unroll
+  for (int c = 0; c < kChunks; ++c) {
+    v[c] = lds128(q_smem + swz(row, c0 + c));
+    const uint32_t w[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) emax = max(emax, max(w[k] & 0x7F80u, (w[k] >> 16) & 0x7F80u));
+  }
+#pragma unroll
+  for (int o = 1; o < kLanesPerRow; o <<= 1) emax = max(emax, __shfl_xor_sync(0xffffffffu, emax, o));
+  uint32_t e = emax >> 7;                       // biased exponent of the row's largest element
+  e = e == 0 ? 127u : min(max(e, 2u), 253u);    // an all-zero row keeps factor 1
+  const float down = __uint_as_float((254u - e) << 23), up = __uint_as_float(e << 23);
+#pragma unroll
+  for (int c = 0; c < kChunks; ++c) {
+    uint32_t w[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+      w[k] = pack_f16(__uint_as_float(w[k] << 16) * down, __uint_as_float(w[k] & 0xFFFF0000u) * down);
+    sts128(q_smem + swz(row, c0 + c), make_uint4(w[0], w[1], w[2], w[3]));
+  }
+  if (lane % kLanesPerRow == 0) qmult[row] = up;
+}
 
 struct TaskView {
   xy_attn_task t;
@@ -345,18 +442,28 @@ __device__ __forceinline__ void report_timeout(const RunArgs& a) {
 // 128-key tile, keeps its own online-softmax state over those keys, and the eight partial
 // results are merged through shared memory when the task ends (the in-CTA Update stage of
 // Section 4.2.1).  pipe_state: ring stage | phase << 8 | dead << 16, returned updated.
+// kFp8: the stages hold e4m3 bytes; every warp widens its 16 keys before use, the Q rows in shared
+// memory are f16 (converted by the caller), qmult / scale_ring carry the row and page factors and
+// tile_seq counts the key tiles this worker has consumed (it selects the scale slot).
+template <bool kFp8>
 __device__ __forceinline__ uint32_t stream_task(const RunArgs& a, const TaskView& tv, uint32_t q_smem, uint32_t ring,
                                              SmemBarriers* bars, float* xch, float* ml, uint32_t pipe_state,
-                                             float scale_log2) {
+                                             float scale_log2, const float* qmult, const float* scale_ring,
+                                             uint32_t& tile_seq) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   Pipe pipe{static_cast<int>(pipe_state & 0xFFu), (pipe_state >> 8) & 1u};
   bool dead = (pipe_state >> 16) & 1u;
   const int h = tv.rq.kv_len;
   const bool tree = tv.rq.mask_kind == XY_MASK_TREE;
   const int koff = warp * 16;
-  WarpTile<2, false> w;
+  WarpTile<2, false, kFp8> w;
   w.init();
   w.load_q(q_smem, 0, lane);
+  FpScale fs{1.f, 1.f, scale_ring, a.page_shift};
+  if constexpr (kFp8) {
+    fs.q_lo = qmult[lane >> 2];
+    fs.q_hi = qmult[(lane >> 2) + 8];
+  }
   const int r_lo = min(lane >> 2, tv.rows - 1), r_hi = min((lane >> 2) + 8, tv.rows - 1);
   const int i_lo = tv.t.tok0 + r_lo / tv.G, i_hi = tv.t.tok0 + r_hi / tv.G;
   const int i_max = tv.t.tok0 + tv.t.ntok - 1;
@@ -384,14 +491,20 @@ __device__ __forceinline__ uint32_t stream_task(const RunArgs& a, const TaskView
       dead = true;
     }
     XY_PH(0)
+    if constexpr (kFp8) {
+      fs.tile = scale_ring + (tile_seq % kScaleSlots) * 16;
+      ++tile_seq;
+      if (work) widen_rows16(ring + pipe.stage * kTileBytes, koff, lane);
+    }
     if (work) w.qk(ring + pipe.stage * kTileBytes, koff, lane, s);
+    if constexpr (kFp8) fence_proxy_async_smem();  // the widened rows are overwritten by the next bulk copy
     __syncwarp();
     if (lane == 0) mbar_arrive(smem_u32(&bars->empty[pipe.stage]));
     pipe.advance();
     XY_PH(1)
     if (work) {
       const bool need_mask = kTail ? (tree ? (col0 + 16 > h) : (col0 + 16 > h + tv.t.tok0 + 1)) : false;
-      w.softmax(a, tv.rq, s, p, col0, i_lo, i_hi, need_mask, scale_log2, lane);
+      w.softmax(a, tv.rq, s, p, col0, i_lo, i_hi, need_mask, scale_log2, lane, &fs, koff);
     }
     XY_PH(2)
     if (!dead && !mbar_wait_block(smem_u32(&bars->full[pipe.stage]), pipe.phase, a.status)) {
@@ -399,7 +512,11 @@ __device__ __forceinline__ uint32_t stream_task(const RunArgs& a, const TaskView
       dead = true;
     }
     XY_PH(3)
+    if constexpr (kFp8) {
+      if (work) widen_rows16(ring + pipe.stage * kTileBytes, koff, lane);
+    }
     if (work) w.pv(ring + pipe.stage * kTileBytes, koff, lane, p);
+    if constexpr (kFp8) fence_proxy_async_smem();
     __syncwarp();
     if (lane == 0) mbar_arrive(smem_u32(&bars->empty[pipe.stage]));
     pipe.advance();
@@ -521,7 +638,7 @@ struct __align__(8) UmmaBarriers {
 static_assert(kStatusWaitLimit == kStatusWaitLimitWord, "one word, two names");
 static_assert(sizeof(UmmaBarriers) <= 128, "the shared-memory layout reserves 128 bytes for UmmaBarriers");
 
-template <bool kUmma>
+template <bool kUmma, bool kFp8>
 __global__ void __launch_bounds__(kThreads, 1)
 meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constant__ CUtensorMap k_map,
                       const __grid_constant__ CUtensorMap v_map) {
@@ -536,6 +653,9 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
   UmmaBarriers* ub = reinterpret_cast<UmmaBarriers*>(gen_base + kSmemQ + kSmemRing + kSmemMl + sizeof(SmemBarriers));
   TaskRing* tq = reinterpret_cast<TaskRing*>(gen_base + kSmemQ + kSmemRing + kSmemMl + sizeof(SmemBarriers) + 128);
   float* xch = reinterpret_cast<float*>(gen_base);  // streaming merge area, aliases the Q tiles
+  static_assert(!(kUmma && kFp8), "the fp8 KV path runs on the warp-level MMA paths");
+  float* qmult = reinterpret_cast<float*>(gen_base + kSmemQ + kSmemRing + kSmemMl + sizeof(SmemBarriers) + 128 + 256);
+  float* scale_ring = qmult + 128;  // [kScaleSlots][16]: K scales [0..7], V scales [8..15] of a tile's pages
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
@@ -617,7 +737,9 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
       const uint64_t pol_stream = make_l2_policy_evict_first(), pol_keep = make_l2_policy_evict_last();
       // Fill one stage (the K or the V tile) once its previous reader has released it.
       int n_fill = 0;
-      auto fill = [&](int op, bool by_umma, int kv_head, int kt, const int32_t* bt, int npages, int page0) {
+      uint32_t k_fills = 0;  // K tiles filled so far (fp8: selects the scale slot)
+      auto fill = [&](int op, bool by_umma, int kv_head, int kt, const int32_t* bt, int npages, int page0,
+                      float ks0, float vs0) {
         // Failure-path test hook (xy_attn_debug_inject): this worker leaves out one fill, so the
         // stage's `full` barrier never completes and the readers' bounded waits run out.
         if (n_fill++ == a.debug_skip_fill) {
@@ -645,9 +767,48 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
         last_umma = by_umma ? (last_umma | bit) : (last_umma & ~bit);
         tr(1 + op);
         const uint32_t full = smem_u32(&bars->full[pipe.stage]);
-        mbar_arrive_expect_tx(full, kTileBytes);
         const uint32_t dst = ring + pipe.stage * kTileBytes;
         const CUtensorMap* map = op == 0 ? &k_map : &v_map;
+        if constexpr (kFp8) {
+          // e4m3 bytes: one box per page (128 B per key) into the upper half of the stage; the K
+          // fill also leaves the K and V scales of the tile's pages in the tile's scale slot, before
+          // the arrive that the readers' wait synchronises with.
+          int pages[8];
+          pages[0] = page0;
+          if (ppt > 1) {
+#pragma unroll
+            for (int p = 0; p < 8; ++p)
+              if (p < ppt) pages[p] = __ldg(bt + min(kt * ppt + p, npages - 1));  // past the end: reload the last
+          }
+          if (op == 0) {
+            float* slot = scale_ring + (k_fills % kScaleSlots) * 16;
+            ++k_fills;
+            if (ppt == 1) {
+              slot[0] = ks0;
+              slot[8] = vs0;
+            } else {
+#pragma unroll
+              for (int p = 0; p < 8; ++p) {
+                if (p < ppt) {
+                  const int64_t si = static_cast<int64_t>(pages[p]) * a.num_kv_heads + kv_head;
+                  slot[p] = __ldg(a.k_scale + si);
+                  slot[8 + p] = __ldg(a.v_scale + si);
+                }
+              }
+            }
+          }
+          mbar_arrive_expect_tx(full, kHalfBytes);
+          if (ppt == 1) {
+            tma_load_4d_hint(dst + kHalfBytes, map, full, 0, 0, kv_head, page0, pol_stream);
+          } else {
+#pragma unroll
+            for (int p = 0; p < 8; ++p)
+              if (p < ppt) tma_load_4d(dst + kHalfBytes + p * page_bytes, map, full, 0, 0, kv_head, pages[p]);
+          }
+          pipe.advance();
+          return;
+        }
+        mbar_arrive_expect_tx(full, kTileBytes);
         if (ppt == 1) {
           // K/V of streaming tasks is read once: mark it evict-first in L2 so that it does not
           // push out the K/V that the q tiles of a prefill share through L2 (kept evict-last).
@@ -671,6 +832,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
       struct Tile {
         const int32_t* bt;
         int kv_head, kt, npages, page;
+        float ks, vs;  // fp8, one page per tile: that page's K and V scale
         bool by_umma, valid;
       };
       int f_ti = t_begin, f_kt = 0, f_hi = 0, f_head = 0, f_npages = 1;
@@ -704,6 +866,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
         x.bt = f_bt;
         x.kv_head = x.kt = x.page = 0;
         x.npages = 1;
+        x.ks = x.vs = 1.f;
         x.by_umma = false;
         while (!f_open || f_kt >= f_hi) {
           const int ti = grab();
@@ -728,14 +891,28 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
         ++f_kt;
         return x;
       };
+      // fp8, one page per tile: the page's scales are requested one step after its block-table
+      // entry (which they depend on) and used one step later still.
+      auto request_scales = [&](Tile& x) {
+        if constexpr (kFp8) {
+          if (ppt == 1 && x.valid) {
+            const int64_t si = static_cast<int64_t>(x.page) * a.num_kv_heads + x.kv_head;
+            x.ks = __ldg(a.k_scale + si);
+            x.vs = __ldg(a.v_scale + si);
+          }
+        }
+      };
       Tile q0 = next_tile(), q1 = next_tile(), q2 = next_tile();
+      request_scales(q0);
+      request_scales(q1);
       while (q0.valid && !dead) {
         const Tile cur = q0;
         q0 = q1;
         q1 = q2;
         q2 = next_tile();
-        fill(0, cur.by_umma, cur.kv_head, cur.kt, cur.bt, cur.npages, cur.page);
-        if (!dead) fill(1, cur.by_umma, cur.kv_head, cur.kt, cur.bt, cur.npages, cur.page);
+        request_scales(q1);
+        fill(0, cur.by_umma, cur.kv_head, cur.kt, cur.bt, cur.npages, cur.page, cur.ks, cur.vs);
+        if (!dead) fill(1, cur.by_umma, cur.kv_head, cur.kt, cur.bt, cur.npages, cur.page, cur.ks, cur.vs);
       }
       // No bulk copy of this CTA may still be in flight when it exits: the latest fill of every
       // stage has landed once its `full` phase completes (immediate on the normal path, where the
@@ -900,6 +1077,7 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
     Pipe pipe{0, 0};
     bool dead = false;
     uint32_t ph_s = 0, ph_o = 0;  // this warpgroup's s_full / o_done parities
+    uint32_t tile_seq = 0;        // key tiles consumed so far (fp8: selects the scale slot)
     Tracer tr;
     tr.init(a, warp >> 2, (threadIdx.x & 127) == 0);
     const int X = warp >> 2;       // sub-tile this warpgroup owns on the tcgen05 path
@@ -1223,15 +1401,27 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
         }
         cp_async_commit_wait_all();
         named_bar_sync(1, kConsumerThreads);
+        if constexpr (kFp8) {
+          // Q rows become f16 with a power-of-two factor per row (dense: each warp its own 16 rows;
+          // streaming: the 16 rows shared by all warps, two per warp)
+          if (stream) q_rows_to_f16<16>(q_smem, warp * 2, qmult, lane);
+          else q_rows_to_f16<2>(q_smem, warp * 16, qmult, lane);
+          named_bar_sync(1, kConsumerThreads);
+        }
       }
 
       if (!kUmma && !stream) {  // (with kUmma every dense task took the tcgen05 path above)
         // ---------------- dense: this warp owns rows x0 .. x0+15 -------------------------
         const int x0 = warp * 16;
         const bool active = x0 < tv.rows;
-        WarpTile<16, false> w;
+        WarpTile<16, false, kFp8> w;
         w.init();
         if (active) w.load_q(q_smem, x0, lane);
+        FpScale fs{1.f, 1.f, scale_ring, a.page_shift};
+        if constexpr (kFp8) {
+          fs.q_lo = qmult[x0 + (lane >> 2)];
+          fs.q_hi = qmult[x0 + (lane >> 2) + 8];
+        }
         const int r_lo = min(x0 + (lane >> 2), tv.rows - 1), r_hi = min(x0 + (lane >> 2) + 8, tv.rows - 1);
         const int i_lo = tv.t.tok0 + r_lo / G, i_hi = tv.t.tok0 + r_hi / G;
         const int i_min = tv.t.tok0 + min(x0, tv.rows - 1) / G;
@@ -1245,19 +1435,32 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
             report_timeout(a);
             dead = true;
           }
+          if constexpr (kFp8) {
+            // every warp widens 16 keys of the tile, all warps read all of it
+            fs.tile = scale_ring + (tile_seq % kScaleSlots) * 16;
+            ++tile_seq;
+            widen_rows16(ring + pipe.stage * kTileBytes, warp * 16, lane);
+            named_bar_sync(1, kConsumerThreads);
+          }
           if (work) w.qk(ring + pipe.stage * kTileBytes, 0, lane, s);
+          if constexpr (kFp8) fence_proxy_async_smem();
           __syncwarp();
           if (lane == 0) mbar_arrive(smem_u32(&bars->empty[pipe.stage]));
           pipe.advance();
           if (work) {
             const bool need_mask = tree ? (col0 + kKeyTile > h) : (col0 + kKeyTile > h + i_min + 1);
-            w.softmax(a, tv.rq, s, p, col0, i_lo, i_hi, need_mask, scale_log2, lane);
+            w.softmax(a, tv.rq, s, p, col0, i_lo, i_hi, need_mask, scale_log2, lane, &fs, 0);
           }
           if (!dead && !mbar_wait_block(smem_u32(&bars->full[pipe.stage]), pipe.phase, a.status)) {
             report_timeout(a);
             dead = true;
           }
+          if constexpr (kFp8) {
+            widen_rows16(ring + pipe.stage * kTileBytes, warp * 16, lane);
+            named_bar_sync(1, kConsumerThreads);
+          }
           if (work) w.pv(ring + pipe.stage * kTileBytes, 0, lane, p);
+          if constexpr (kFp8) fence_proxy_async_smem();
           __syncwarp();
           if (lane == 0) mbar_arrive(smem_u32(&bars->empty[pipe.stage]));
           pipe.advance();
@@ -1283,8 +1486,8 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
         named_bar_sync(1, kConsumerThreads);  // Q tile may be overwritten by the next task
       } else {
         // ---------------- streaming (see stream_task) ----
-        const uint32_t st = stream_task(a, tv, q_smem, ring, bars, xch, ml, pipe.stage | (pipe.phase << 8) |
-                                        (dead ? 1u << 16 : 0u), scale_log2);
+        const uint32_t st = stream_task<kFp8>(a, tv, q_smem, ring, bars, xch, ml, pipe.stage | (pipe.phase << 8) |
+                                              (dead ? 1u << 16 : 0u), scale_log2, qmult, scale_ring, tile_seq);
         pipe.stage = st & 0xFFu;
         pipe.phase = (st >> 8) & 1u;
         dead = (st >> 16) & 1u;
@@ -1329,16 +1532,18 @@ EncodeTiledFn encode_fn() {
 
 // 4-D map over a paged pool [pages, Hkv, B, D]: box = one page of one head, 64 elements wide.
 bool encode_pool_map(CUtensorMap* m, const void* pool, int64_t num_pages, int num_kv_heads, int page_size,
-                     int64_t page_stride, int64_t head_stride, int64_t token_stride) {
+                     int64_t page_stride, int64_t head_stride, int64_t token_stride, bool fp8) {
   EncodeTiledFn fn = encode_fn();
   if (fn == nullptr) return false;
+  // bf16: two boxes of 64 elements per row; e4m3 bytes: one box of 128 - 128 B per row either way
+  const cuuint64_t esz = fp8 ? 1 : 2;
   cuuint64_t dims[4] = {static_cast<cuuint64_t>(kHeadDim), static_cast<cuuint64_t>(page_size),
                         static_cast<cuuint64_t>(num_kv_heads), static_cast<cuuint64_t>(num_pages)};
-  cuuint64_t strides[3] = {static_cast<cuuint64_t>(token_stride) * 2, static_cast<cuuint64_t>(head_stride) * 2,
-                           static_cast<cuuint64_t>(page_stride) * 2};
-  cuuint32_t box[4] = {64, static_cast<cuuint32_t>(page_size), 1, 1};
+  cuuint64_t strides[3] = {static_cast<cuuint64_t>(token_stride) * esz, static_cast<cuuint64_t>(head_stride) * esz,
+                           static_cast<cuuint64_t>(page_stride) * esz};
+  cuuint32_t box[4] = {fp8 ? 128u : 64u, static_cast<cuuint32_t>(page_size), 1, 1};
   cuuint32_t estr[4] = {1, 1, 1, 1};
-  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(pool), dims, strides, box, estr,
+  CUresult r = fn(m, fp8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(pool), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
@@ -1349,24 +1554,28 @@ bool encode_pool_map(CUtensorMap* m, const void* pool, int64_t num_pages, int nu
 cudaError_t launch_meta(const RunArgs& a, int num_workers, int64_t num_pages, bool umma, MetaLaunchCache* cache,
                         cudaStream_t s) {
   static_assert(sizeof(CUtensorMap) == 128, "MetaLaunchCache holds a tensor map in 128 bytes");
-  auto kernel = umma ? meta_attention_kernel<true> : meta_attention_kernel<false>;
-  if (!cache->attr_set[umma ? 1 : 0]) {
+  const bool fp8 = a.kv_fp8 != 0;
+  if (fp8) umma = false;
+  auto kernel = fp8 ? meta_attention_kernel<false, true>
+                    : (umma ? meta_attention_kernel<true, false> : meta_attention_kernel<false, false>);
+  const int which = fp8 ? 2 : (umma ? 1 : 0);
+  if (!cache->attr_set[which]) {
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTotal);
     if (e != cudaSuccess) return e;
-    cache->attr_set[umma ? 1 : 0] = true;
+    cache->attr_set[which] = true;
   }
   CUtensorMap* k_map = reinterpret_cast<CUtensorMap*>(cache->maps[0]);
   CUtensorMap* v_map = reinterpret_cast<CUtensorMap*>(cache->maps[1]);
   const bool same = cache->valid && cache->k_pool == a.k_pool && cache->v_pool == a.v_pool &&
                     cache->num_pages == num_pages && cache->page_stride == a.page_stride &&
                     cache->head_stride == a.head_stride && cache->token_stride == a.token_stride &&
-                    cache->num_kv_heads == a.num_kv_heads && cache->page_size == a.page_size;
+                    cache->num_kv_heads == a.num_kv_heads && cache->page_size == a.page_size && cache->fp8 == fp8;
   if (!same) {
     cache->valid = false;
     if (!encode_pool_map(k_map, a.k_pool, num_pages, a.num_kv_heads, a.page_size, a.page_stride, a.head_stride,
-                         a.token_stride) ||
+                         a.token_stride, fp8) ||
         !encode_pool_map(v_map, a.v_pool, num_pages, a.num_kv_heads, a.page_size, a.page_stride, a.head_stride,
-                         a.token_stride))
+                         a.token_stride, fp8))
       return cudaErrorInvalidValue;
     cache->k_pool = a.k_pool;
     cache->v_pool = a.v_pool;
@@ -1376,6 +1585,7 @@ cudaError_t launch_meta(const RunArgs& a, int num_workers, int64_t num_pages, bo
     cache->token_stride = a.token_stride;
     cache->num_kv_heads = a.num_kv_heads;
     cache->page_size = a.page_size;
+    cache->fp8 = fp8;
     cache->valid = true;
   }
   MetaParams P{a};

@@ -2,6 +2,8 @@
 // block-table gather.  The reference kernel walks the same Task-Table as the fast
 // kernels and is kept for bisecting: one warp per packed row, one key at a time.
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_fp8.h>
 #include <cuda_runtime.h>
 
 #include "xy_kernels.h"
@@ -16,6 +18,24 @@ __device__ __forceinline__ float bf16_bits_to_float(uint16_t b) {
 
 __device__ __forceinline__ uint16_t float_to_bf16_bits(float f) {
   return __bfloat16_as_ushort(__float2bfloat16_rn(f));
+}
+
+// Four consecutive K or V elements of a cached token as fp32: bf16 pools, or (fp8 KV cache) e4m3
+// bytes times the page's scale.  `off` counts elements from the pool's base.
+__device__ __forceinline__ void load_kv4(const RunArgs& a, const uint16_t* pool, int64_t off, float scale, float (&out)[4]) {
+  if (a.kv_fp8) {
+    const uint32_t w = *reinterpret_cast<const uint32_t*>(reinterpret_cast<const uint8_t*>(pool) + off);
+    const __half2_raw lo = __nv_cvt_fp8x2_to_halfraw2(static_cast<__nv_fp8x2_storage_t>(w & 0xFFFFu), __NV_E4M3);
+    const __half2_raw hi = __nv_cvt_fp8x2_to_halfraw2(static_cast<__nv_fp8x2_storage_t>(w >> 16), __NV_E4M3);
+    const float2 f0 = __half22float2(__half2(lo)), f1 = __half22float2(__half2(hi));
+    out[0] = f0.x * scale;
+    out[1] = f0.y * scale;
+    out[2] = f1.x * scale;
+    out[3] = f1.y * scale;
+  } else {
+#pragma unroll
+    for (int d = 0; d < 4; ++d) out[d] = bf16_bits_to_float(pool[off + d]);
+  }
 }
 
 __device__ __forceinline__ float warp_sum(float v) {
@@ -57,18 +77,24 @@ __global__ void __launch_bounds__(128) ref_attention_kernel(RunArgs a) {
         const int64_t page = bt[j >> a.page_shift];
         const int64_t off = page * a.page_stride + static_cast<int64_t>(t.kv_head) * a.head_stride +
                             static_cast<int64_t>(j & (a.page_size - 1)) * a.token_stride + lane * 4;
-        const uint16_t* kp = a.k_pool + off;
-        const uint16_t* vp = a.v_pool + off;
+        float kf[4], vf[4];
+        float ksc = 1.f, vsc = 1.f;
+        if (a.kv_fp8) {
+          ksc = a.k_scale[page * a.num_kv_heads + t.kv_head];
+          vsc = a.v_scale[page * a.num_kv_heads + t.kv_head];
+        }
+        load_kv4(a, a.k_pool, off, ksc, kf);
+        load_kv4(a, a.v_pool, off, vsc, vf);
         float dot = 0.f;
 #pragma unroll
-        for (int d = 0; d < 4; ++d) dot += qv[d] * bf16_bits_to_float(kp[d]);
+        for (int d = 0; d < 4; ++d) dot += qv[d] * kf[d];
         const float s = warp_sum(dot) * a.sm_scale;
         const float m_new = fmaxf(m, s);
         const float alpha = __expf(m - m_new);  // m = -inf on the first key: alpha = 0
         const float p = __expf(s - m_new);
         l = l * alpha + p;
 #pragma unroll
-        for (int d = 0; d < 4; ++d) o[d] = o[d] * alpha + p * bf16_bits_to_float(vp[d]);
+        for (int d = 0; d < 4; ++d) o[d] = o[d] * alpha + p * vf[d];
         m = m_new;
       }
       const float inv = l > 0.f ? 1.f / l : 0.f;

@@ -237,6 +237,7 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
   out->shape.push_back(static_cast<int32_t>(std::min<int64_t>(partial_row_capacity, INT32_MAX)));
   out->shape.push_back(cfg.plan_mode * 4 + cfg.kernel);
   out->shape.push_back(cfg.max_splits);
+  out->shape.push_back(cfg.kv_dtype);
   for (const Unit& u : units) {
     out->shape.push_back(u.req);
     out->shape.push_back(u.kv_head);
@@ -253,7 +254,7 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
     out->shape_hash = hsh;
   }
   const int64_t flops_now = 4ll * kHeadDim * cfg.num_q_heads * pairs;
-  const int64_t kv_bytes_now = 2ll * kv_tokens * cfg.num_kv_heads * kHeadDim * 2;
+  const int64_t kv_bytes_now = 2ll * kv_tokens * cfg.num_kv_heads * kHeadDim * (cfg.kv_dtype == XY_KV_FP8_E4M3 ? 1 : 2);
   if (cache != nullptr) {
     ++cache->clock;
     for (PlanCache::Entry& e : cache->entries) {

@@ -72,7 +72,9 @@ struct PlanCache {
 };
 
 // 128-row sub-tiles one dense task may hold (the tcgen05 path ping-pongs two; the others one).
-inline int dense_subtiles(const xy_attn_config& cfg) { return cfg.kernel == XY_KERNEL_AUTO ? 2 : 1; }
+inline int dense_subtiles(const xy_attn_config& cfg) {
+  return cfg.kernel == XY_KERNEL_AUTO && cfg.kv_dtype == XY_KV_BF16 ? 2 : 1;
+}
 
 // Host-only planning.  Returns XY_OK or an error code and fills `err`.
 // `cache` (nullable): Task-Tables of earlier plans; a plan whose decomposition equals a cached one
@@ -111,6 +113,11 @@ struct RunArgs {
   const int32_t* queue;
   int32_t* queue_head;
   int32_t num_tasks, dynamic;
+  // fp8 KV cache: k_pool / v_pool hold e4m3 bytes (strides in bytes) and these are the fp32 scales
+  // [pages, Hkv] of K and V
+  const float* k_scale;
+  const float* v_scale;
+  int32_t kv_fp8;
   // test hook: the producer of every worker leaves out its debug_skip_fill-th stage fill (-1: none)
   int32_t debug_skip_fill;
 };

@@ -27,8 +27,8 @@ struct MetaLaunchCache {
   const void* v_pool = nullptr;
   int64_t num_pages = 0, page_stride = 0, head_stride = 0, token_stride = 0;
   int32_t num_kv_heads = 0, page_size = 0;
-  bool valid = false;
-  bool attr_set[2] = {false, false};
+  bool valid = false, fp8 = false;
+  bool attr_set[3] = {false, false, false};
 };
 
 cudaError_t launch_reference(const RunArgs& a, int num_workers, cudaStream_t s);

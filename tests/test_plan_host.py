@@ -24,7 +24,7 @@ def host_ctx(hq, hkv, page, **kw):
 
 def test_library_exports_every_declared_symbol():
     header = open(os.path.join(ROOT, "include", "xy_attn.h")).read()
-    declared = set(re.findall(r"\b(xy_attn_[a-z_]+)\s*\(", header))
+    declared = set(re.findall(r"\b(xy_attn_[a-z0-9_]+)\s*\(", header))
     assert declared == set(xb.EXPORTS)
     lib = ctypes.CDLL(xb.LIB_PATH)
     for name in declared:
@@ -35,7 +35,7 @@ def test_struct_sizes_match_header():
     assert ctypes.sizeof(xb.xy_attn_task) == 32
     assert ctypes.sizeof(xb.xy_attn_request) == 16
     assert ctypes.sizeof(xb.xy_attn_merge_unit) == 40
-    assert ctypes.sizeof(xb.xy_attn_config) == 14 * 4 + 8
+    assert ctypes.sizeof(xb.xy_attn_config) == 16 * 4 + 8   # 15 int32, padding, int64
 
 
 def test_create_rejects_bad_configs():
