@@ -136,6 +136,10 @@ typedef struct {
   int64_t partial_rows;   /* fp32 partial rows used in the workspace */
   float load_min, load_mean, load_max; /* per-worker summed task cost */
   float max_task_cost;
+  int32_t num_inline_merge_units; /* of num_merge_units: split units of at most 16 rows (decode, tiny verify) that the
+                                   * attention kernel merges itself - the task of the unit that finishes last does it;
+                                   * the others are merged by the merge kernel (they come first in the unit list) */
+  int32_t reserved;
 } xy_attn_plan_info;
 
 /* Create a context.  Allocates the device-side tables and the split workspace

@@ -70,7 +70,8 @@ class xy_attn_plan_info(ctypes.Structure):
                 ("useful_flops", ctypes.c_int64), ("kv_bytes", ctypes.c_int64),
                 ("partial_rows", ctypes.c_int64), ("load_min", ctypes.c_float),
                 ("load_mean", ctypes.c_float), ("load_max", ctypes.c_float),
-                ("max_task_cost", ctypes.c_float)]
+                ("max_task_cost", ctypes.c_float), ("num_inline_merge_units", ctypes.c_int32),
+                ("reserved", ctypes.c_int32)]
 
 
 TASK_DTYPE = np.dtype([(n, np.int32) for n in ("req", "kv_head", "tok0", "ntok", "kt_lo", "kt_hi", "part", "kind")])

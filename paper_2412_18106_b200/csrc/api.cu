@@ -32,10 +32,12 @@ struct xy_attn_ctx {
   xy_attn_task* d_tasks = nullptr;
   int32_t* d_worker_off = nullptr;
   int32_t* d_queue = nullptr;
+  int32_t* d_task_unit = nullptr;
   uint64_t* d_tree = nullptr;
   xy_attn_merge_unit* d_merges = nullptr;
   float* d_o_part = nullptr;
   float* d_lse_part = nullptr;
+  int32_t* d_status_base = nullptr;  // allocation; d_status = d_status_base + kStatusLead
   int32_t* d_status = nullptr;
   unsigned long long* d_trace = nullptr;
   unsigned long long* d_worker_times = nullptr;
@@ -79,11 +81,12 @@ void free_device(xy_attn_ctx* c) {
   cudaFree(c->d_tasks);
   cudaFree(c->d_worker_off);
   cudaFree(c->d_queue);
+  cudaFree(c->d_task_unit);
   cudaFree(c->d_tree);
   cudaFree(c->d_merges);
   cudaFree(c->d_o_part);
   cudaFree(c->d_lse_part);
-  cudaFree(c->d_status);
+  cudaFree(c->d_status_base);
   cudaFree(c->d_trace);
   cudaFree(c->d_worker_times);
 }
@@ -157,13 +160,17 @@ int xy_attn_create(const xy_attn_config* cfg, xy_attn_ctx** out) {
     alloc(reinterpret_cast<void**>(&c->d_tasks), sizeof(xy_attn_task) * c->cap_tasks);
     alloc(reinterpret_cast<void**>(&c->d_worker_off), sizeof(int32_t) * (c->num_workers + 1));
     alloc(reinterpret_cast<void**>(&c->d_queue), sizeof(int32_t) * c->cap_tasks);
+    alloc(reinterpret_cast<void**>(&c->d_task_unit), sizeof(int32_t) * c->cap_tasks);
     alloc(reinterpret_cast<void**>(&c->d_tree), sizeof(uint64_t) * c->cap_tree_words);
     alloc(reinterpret_cast<void**>(&c->d_merges), sizeof(xy_attn_merge_unit) * c->cap_merges);
     alloc(reinterpret_cast<void**>(&c->d_o_part), sizeof(float) * kHeadDim * c->cap_partial_rows);
     alloc(reinterpret_cast<void**>(&c->d_lse_part), sizeof(float) * c->cap_partial_rows);
-    alloc(reinterpret_cast<void**>(&c->d_status), 256);
+    // status words, then one completion counter per merge unit
+    const size_t status_bytes = sizeof(int32_t) * (kStatusLead + kStatusUnitCounts + c->cap_merges);
+    alloc(reinterpret_cast<void**>(&c->d_status_base), status_bytes);
+    c->d_status = c->d_status_base + kStatusLead;
     alloc(reinterpret_cast<void**>(&c->d_worker_times), sizeof(unsigned long long) * 4 * c->num_workers);
-    if (e == cudaSuccess) e = cudaMemset(c->d_status, 0, 256);
+    if (e == cudaSuccess) e = cudaMemset(c->d_status_base, 0, status_bytes);
     const int32_t default_limit = 1 << 22;
     if (e == cudaSuccess)
       e = cudaMemcpy(c->d_status + kStatusWaitLimit, &default_limit, sizeof default_limit, cudaMemcpyHostToDevice);
@@ -242,6 +249,9 @@ int xy_attn_plan_shared(xy_attn_ctx* ctx, const xy_attn_request* reqs, int32_t n
                                      sizeof(xy_attn_task) * p.tasks.size(), cudaMemcpyHostToDevice, s));
       if (!p.queue.empty())
         XY_CUDA(ctx, cudaMemcpyAsync(ctx->d_queue, p.queue.data(), sizeof(int32_t) * p.queue.size(),
+                                     cudaMemcpyHostToDevice, s));
+      if (!p.task_unit.empty())
+        XY_CUDA(ctx, cudaMemcpyAsync(ctx->d_task_unit, p.task_unit.data(), sizeof(int32_t) * p.task_unit.size(),
                                      cudaMemcpyHostToDevice, s));
       XY_CUDA(ctx, cudaMemcpyAsync(ctx->d_worker_off, p.worker_off.data(),
                                    sizeof(int32_t) * p.worker_off.size(), cudaMemcpyHostToDevice, s));
@@ -360,6 +370,7 @@ int run_impl(xy_attn_ctx* ctx, const void* q, int64_t q_token_stride, const void
   a.o_part = ctx->d_o_part;
   a.lse_part = ctx->d_lse_part;
   a.status = ctx->d_status;
+  const bool in_kernel_merges = p.num_launch_merges < static_cast<int32_t>(p.merges.size());
   a.trace = ctx->d_trace;
   a.worker_times = ctx->d_worker_times;
   a.num_q_heads = cfg.num_q_heads;
@@ -373,12 +384,15 @@ int run_impl(xy_attn_ctx* ctx, const void* q, int64_t q_token_stride, const void
   // Task-Table (each worker walks its own list), as does the reference kernel.
   a.dynamic = (cfg.plan_mode == XY_PLAN_BALANCED && cfg.kernel != XY_KERNEL_REFERENCE) ? 1 : 0;
   a.debug_skip_fill = ctx->dbg_skip_fill;
+  a.task_unit = in_kernel_merges ? ctx->d_task_unit : nullptr;
+  a.units = ctx->d_merges;
+  a.unit_count = ctx->d_status + kStatusUnitCounts;
   a.k_scale = k_scale;
   a.v_scale = v_scale;
   a.kv_fp8 = fp8 ? 1 : 0;
-  // Every run starts with a clean status word and queue head (one memset covers both): a run
-  // after a device-side timeout is an ordinary run.  The sticky record (status[1]) is kept.
-  XY_CUDA(ctx, cudaMemsetAsync(a.status, 0, 17 * sizeof(int32_t), s));
+  // Every run starts with a clean status word, queue head and unit counters (one memset): a run
+  // after a device-side timeout is an ordinary run.  The sticky record in front of them is kept.
+  XY_CUDA(ctx, cudaMemsetAsync(a.status, 0, (kStatusUnitCounts + (in_kernel_merges ? p.merges.size() : 0)) * sizeof(int32_t), s));
 
   const bool timed = ctx->timing && ctx->timed_runs < kMaxTimedRuns;
   if (timed) {
@@ -399,7 +413,7 @@ int run_impl(xy_attn_ctx* ctx, const void* q, int64_t q_token_stride, const void
   ctx->last_launches += 1;
   if (timed) XY_CUDA(ctx, cudaEventRecord(ctx->events[3 * ctx->timed_runs + 1], s));
 
-  if (!p.merges.empty()) {
+  if (p.num_launch_merges > 0) {
     MergeArgs m{};
     m.units = ctx->d_merges;
     m.reqs = ctx->d_reqs;
@@ -411,11 +425,12 @@ int run_impl(xy_attn_ctx* ctx, const void* q, int64_t q_token_stride, const void
     m.num_q_heads = cfg.num_q_heads;
     m.num_kv_heads = cfg.num_kv_heads;
     int max_rows = 1, max_parts = 1;
-    for (const xy_attn_merge_unit& mu : p.merges) {
+    for (int32_t k = 0; k < p.num_launch_merges; ++k) {
+      const xy_attn_merge_unit& mu = p.merges[k];
       max_rows = std::max(max_rows, mu.ntok * (cfg.num_q_heads / cfg.num_kv_heads));
       max_parts = std::max(max_parts, mu.nsplit + mu.nsplit1);
     }
-    XY_CUDA(ctx, launch_merge_units(m, static_cast<int>(p.merges.size()), max_rows, max_parts, s));
+    XY_CUDA(ctx, launch_merge_units(m, p.num_launch_merges, max_rows, max_parts, s));
     ctx->last_launches += 1;
   }
   if (timed) {
@@ -692,9 +707,10 @@ int xy_attn_device_status(xy_attn_ctx* ctx, int32_t* status_out) {
   XY_CUDA(ctx, cudaDeviceSynchronize());
   // word 0 is the last run's status (cleared by every run), word kStatusSticky the record of
   // every failure since the last call of this function: report it and clear both.
-  int32_t st[kStatusSticky + 1];
-  XY_CUDA(ctx, cudaMemcpy(st, ctx->d_status, sizeof st, cudaMemcpyDeviceToHost));
-  const int32_t seen = st[kStatusSticky] != 0 ? st[kStatusSticky] : st[0];
+  int32_t st[kStatusLead + 1];
+  XY_CUDA(ctx, cudaMemcpy(st, ctx->d_status_base, sizeof st, cudaMemcpyDeviceToHost));
+  const int32_t sticky = st[kStatusLead + kStatusSticky], last = st[kStatusLead];
+  const int32_t seen = sticky != 0 ? sticky : last;
   if (seen != 0) {
     XY_CUDA(ctx, cudaMemset(ctx->d_status, 0, sizeof(int32_t)));
     XY_CUDA(ctx, cudaMemset(ctx->d_status + kStatusSticky, 0, sizeof(int32_t)));

@@ -436,6 +436,58 @@ __device__ __forceinline__ void report_timeout(const RunArgs& a) {
   atomicExch(a.status + kStatusSticky, XY_ERR_DEVICE_TIMEOUT);
 }
 
+// Merge of a split streaming unit inside the attention kernel (the cross-task Update stage of
+// Section 4.2.1, run by the task of the unit that finished last).  rows <= 16; one warp per row;
+// LSE_c in lanes, the partial rows read eight at a time straight from L2.
+__device__ __forceinline__ float ldcg_f(const float* p) { return __ldcg(p); }
+__device__ __forceinline__ void merge_unit_in_kernel(const RunArgs& a, const xy_attn_merge_unit& u, int G, int warp,
+                                                     int lane) {
+  const int rows = u.ntok * G, ns = u.nsplit;
+  const ReqInfo rq = a.reqs[u.req];
+  for (int x = warp; x < rows; x += kConsumerWarps) {
+    const int64_t row0 = static_cast<int64_t>(u.part0) + x;  // partial row of split c: row0 + c * rows
+    float mx = -INFINITY;
+    for (int c = lane; c < ns; c += 32) mx = fmaxf(mx, ldcg_f(a.lse_part + row0 + static_cast<int64_t>(c) * rows));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    float z = 0.f;
+    for (int c = lane; c < ns; c += 32) {
+      const float lc = ldcg_f(a.lse_part + row0 + static_cast<int64_t>(c) * rows);
+      if (lc != -INFINITY) z += __expf(lc - mx);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
+    const float lse = mx + logf(z);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int c0 = 0; c0 < ns; c0 += 8) {
+      float w[8];
+      float4 v[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const int c = c0 + e;
+        const float lc = c < ns ? ldcg_f(a.lse_part + row0 + static_cast<int64_t>(c) * rows) : -INFINITY;
+        w[e] = lc != -INFINITY ? __expf(lc - lse) : 0.f;
+        // an empty split (weight 0) is not read
+        v[e] = w[e] != 0.f ? __ldcg(reinterpret_cast<const float4*>(a.o_part + (row0 + static_cast<int64_t>(c) * rows) * kHeadDim) + lane)
+                           : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        acc.x += w[e] * v[e].x;
+        acc.y += w[e] * v[e].y;
+        acc.z += w[e] * v[e].z;
+        acc.w += w[e] * v[e].w;
+      }
+    }
+    const int i = u.tok0 + x / G, head = u.kv_head * G + x % G;
+    uint2 packed;
+    packed.x = pack_bf16(acc.x, acc.y);
+    packed.y = pack_bf16(acc.z, acc.w);
+    *reinterpret_cast<uint2*>(a.o + static_cast<int64_t>(rq.q_start + i) * a.o_token_stride + head * kHeadDim + lane * 4) = packed;
+    if (lane == 0) a.lse[static_cast<int64_t>(rq.q_start + i) * a.num_q_heads + head] = lse;
+  }
+}
+
 // ------------------------------------------------------------------------------------------
 // One streaming task (at most 16 packed rows: decode steps, short verify windows and the thin
 // tails of prefill chunks), run by the eight consumer warps.  Every warp owns 16 keys of each
@@ -449,7 +501,7 @@ template <bool kFp8>
 __device__ __forceinline__ uint32_t stream_task(const RunArgs& a, const TaskView& tv, uint32_t q_smem, uint32_t ring,
                                              SmemBarriers* bars, float* xch, float* ml, uint32_t pipe_state,
                                              float scale_log2, const float* qmult, const float* scale_ring,
-                                             uint32_t& tile_seq) {
+                                             uint32_t& tile_seq, int unit) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   Pipe pipe{static_cast<int>(pipe_state & 0xFFu), (pipe_state >> 8) & 1u};
   bool dead = (pipe_state >> 16) & 1u;
@@ -578,6 +630,23 @@ __device__ __forceinline__ uint32_t stream_task(const RunArgs& a, const TaskView
       for (int e = 0; e < 8; e += 2)
         write_row_pair(a, tv, x, seg * 8 + e, acc[e] * inv, acc[e + 1] * inv);
       if (seg == 0) write_lse(a, tv, x, L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY);
+    }
+  }
+  if (unit >= 0) {
+    // This task is one KV split of a unit that is merged here: publish the partial, count the
+    // finished splits, and let the task that completes the unit merge it.  (Writers: stores, fence,
+    // barrier, one atomic; the last one: atomic, fence, loads that bypass L1.)
+    __shared__ int s_last;
+    __threadfence();
+    named_bar_sync(1, kConsumerThreads);
+    if (threadIdx.x == 0) {
+      const int ns = a.units[unit].nsplit;
+      s_last = atomicAdd(a.unit_count + unit, 1) == ns - 1 ? 1 : 0;
+    }
+    named_bar_sync(1, kConsumerThreads);
+    if (s_last) {
+      __threadfence();
+      merge_unit_in_kernel(a, a.units[unit], tv.G, warp, lane);
     }
   }
   return static_cast<uint32_t>(pipe.stage) | (pipe.phase << 8) | (dead ? 1u << 16 : 0u);
@@ -1487,7 +1556,8 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
       } else {
         // ---------------- streaming (see stream_task) ----
         const uint32_t st = stream_task<kFp8>(a, tv, q_smem, ring, bars, xch, ml, pipe.stage | (pipe.phase << 8) |
-                                              (dead ? 1u << 16 : 0u), scale_log2, qmult, scale_ring, tile_seq);
+                                              (dead ? 1u << 16 : 0u), scale_log2, qmult, scale_ring, tile_seq,
+                                              (a.task_unit != nullptr && tv.t.part >= 0) ? a.task_unit[ti] : -1);
         pipe.stage = st & 0xFFu;
         pipe.phase = (st >> 8) & 1u;
         dead = (st >> 16) & 1u;

@@ -266,6 +266,8 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
       out->worker_off = e.worker_off;
       out->queue = e.queue;
       out->merges = e.merges;
+      out->task_unit = e.task_unit;
+      out->num_launch_merges = e.num_launch_merges;
       out->partial_rows = e.partial_rows;
       out->info = e.info;
       out->info.useful_flops = flops_now;
@@ -323,6 +325,7 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
   std::vector<Pending> pend;
   int64_t prow = 0;
   std::vector<int32_t> unit_part(units.size(), -1), unit_nsplit(units.size(), 1);
+  std::vector<int32_t> pend_merge;  // per pending task: index in out->merges of its (plain) unit, or -1
   for (size_t k = 0; k < units.size(); ++k) {
     const Unit& u = units[k];
     const int chunk = chunk_tiles[k];
@@ -331,11 +334,14 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
     const bool partial = nsplit > 1 || u.group >= 0;  // group units always leave partials
     unit_nsplit[k] = nsplit;
     if (partial) unit_part[k] = static_cast<int32_t>(prow);
+    int32_t merge_idx = -1;
     if (nsplit > 1 && u.group < 0) {
       xy_attn_merge_unit mu{u.req, u.kv_head, u.tok0, u.ntok, static_cast<int32_t>(prow), nsplit, 0, 0, 0, 0};
+      merge_idx = static_cast<int32_t>(out->merges.size());
       out->merges.push_back(mu);
     }
     for (int c = 0; c < nsplit; ++c) {
+      pend_merge.push_back(merge_idx);
       Pending p;
       p.t.req = u.req;
       p.t.kv_head = u.kv_head;
@@ -366,6 +372,27 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
     }
   }
   out->partial_rows = prow;
+  // Streaming units (at most 16 rows: decode, tiny verify) are merged inside the attention kernel
+  // by whichever of their tasks finishes last; dense units (up to 256 rows x splits: a merge that
+  // is better spread over all workers) and the two-family units of shared-prefix groups go to the
+  // merge kernel.  `merges` is reordered: the merge kernel's units first.
+  std::vector<int32_t> merge_new(out->merges.size(), -1);
+  {
+    const bool in_kernel_ok = cfg.kernel != XY_KERNEL_REFERENCE && !paper;
+    std::vector<xy_attn_merge_unit> launch, inside;
+    std::vector<int32_t> launch_old, inside_old;
+    for (size_t m = 0; m < out->merges.size(); ++m) {
+      const xy_attn_merge_unit& mu = out->merges[m];
+      const bool in_kernel = in_kernel_ok && mu.nsplit1 == 0 && mu.ntok * G <= kStreamRowsMax;
+      (in_kernel ? inside : launch).push_back(mu);
+      (in_kernel ? inside_old : launch_old).push_back(static_cast<int32_t>(m));
+    }
+    out->num_launch_merges = static_cast<int32_t>(launch.size());
+    for (size_t k = 0; k < launch_old.size(); ++k) merge_new[launch_old[k]] = -1;  // their tasks carry no unit
+    for (size_t k = 0; k < inside_old.size(); ++k) merge_new[inside_old[k]] = static_cast<int32_t>(launch.size() + k);
+    out->merges = launch;
+    out->merges.insert(out->merges.end(), inside.begin(), inside.end());
+  }
 
   // ---- a3: reordering -> Task-Table ------------------------------------------------------
   std::vector<int> order(pend.size());
@@ -389,6 +416,7 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
     float load = 0.f;
     for (int id : lists[w]) {
       where[id] = static_cast<int32_t>(out->tasks.size());
+      out->task_unit.push_back(pend_merge[id] >= 0 ? merge_new[pend_merge[id]] : -1);
       out->tasks.push_back(pend[id].t);
       out->task_cost.push_back(pend[id].cost);
       load += pend[id].cost;
@@ -469,6 +497,8 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
   info.num_tasks = static_cast<int32_t>(out->tasks.size());
   info.num_dense_tasks = ndense;
   info.num_merge_units = static_cast<int32_t>(out->merges.size());
+  info.num_inline_merge_units = info.num_merge_units - out->num_launch_merges;
+  info.reserved = 0;
   info.num_workers = C;
   info.useful_flops = flops_now;
   info.kv_bytes = kv_bytes_now;
@@ -494,6 +524,8 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
     slot->worker_off = out->worker_off;
     slot->queue = out->queue;
     slot->merges = out->merges;
+    slot->task_unit = out->task_unit;
+    slot->num_launch_merges = out->num_launch_merges;
     slot->partial_rows = out->partial_rows;
     slot->info = out->info;
     slot->last_use = cache->clock;

@@ -52,7 +52,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const v
 }
 // The same for kernels whose status is a block of words: word kStatusWaitLimitWord holds the
 // number of polls after which a wait gives up (2^22 by default; a test hook lowers it).
-constexpr int kStatusWaitLimitWord = 33;
+constexpr int kStatusWaitLimitWord = -7;
 __device__ __forceinline__ bool wait_should_give_up(const volatile int32_t* status, uint32_t polls) {
   return status[0] != 0 || polls >= static_cast<uint32_t>(status[kStatusWaitLimitWord]);
 }

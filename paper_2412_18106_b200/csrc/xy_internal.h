@@ -12,12 +12,18 @@ namespace xy {
 constexpr int kHeadDim = 128;
 constexpr int kKeyTile = 128;      // keys per KV tile (one MMA N extent)
 constexpr int kStreamRowsMax = 16;
-// Words of the 256-byte status block: [0] the current run's status, polled by every bounded wait
-// and cleared when a run starts; the queue head of dynamic dealing (its own cache line); the
-// sticky record of failures that xy_attn_device_status reports and clears.
+// The status block, indexed from the word the kernels receive as `status`:
+//   [0]   the current run's status, polled by every bounded wait
+//   [16]  the queue head of dynamic dealing (its own cache line)
+//   [32 ..] one completion counter per merge unit
+// all of which one memset clears when a run starts; and in front of them, untouched by that,
+//   [-8]  the sticky record of failures that xy_attn_device_status reports and clears
+//   [-7]  the number of polls after which a bounded wait gives up (ptx.cuh reads the same word).
 constexpr int kStatusQueueHead = 16;
-constexpr int kStatusSticky = 32;
-constexpr int kStatusWaitLimit = 33;  // polls after which a bounded wait gives up (ptx.cuh reads the same word)
+constexpr int kStatusUnitCounts = 32;
+constexpr int kStatusSticky = -8;
+constexpr int kStatusWaitLimit = -7;
+constexpr int kStatusLead = 8;  // words in front of `status`
 constexpr int kTraceRoles = 4;      // sub-tile A, sub-tile B, MMA issuer, producer (worker 0 only)
 constexpr int kTraceLen = 2048;    // records per role and run
 
@@ -41,7 +47,10 @@ struct PlanResult {
   std::vector<float> task_cost;            // parallel to tasks
   std::vector<int32_t> worker_off;         // num_workers + 1
   std::vector<int32_t> queue;              // task indices by descending cost (dynamic dealing)
-  std::vector<xy_attn_merge_unit> merges;
+  std::vector<xy_attn_merge_unit> merges;  // units merged by the merge kernel first, then those merged in the attention kernel
+  std::vector<int32_t> task_unit;          // parallel to tasks: index in `merges` of the unit the last finisher merges
+                                           // inside the attention kernel, or -1
+  int32_t num_launch_merges = 0;           // leading entries of `merges` that the merge kernel handles
   int64_t partial_rows = 0;
   int64_t total_q = 0;
   xy_attn_plan_info info{};
@@ -62,6 +71,8 @@ struct PlanCache {
     std::vector<float> task_cost;
     std::vector<int32_t> worker_off, queue;
     std::vector<xy_attn_merge_unit> merges;
+    std::vector<int32_t> task_unit;
+    int32_t num_launch_merges = 0;
     int64_t partial_rows = 0;
     xy_attn_plan_info info{};
     uint64_t last_use = 0;
@@ -113,6 +124,10 @@ struct RunArgs {
   const int32_t* queue;
   int32_t* queue_head;
   int32_t num_tasks, dynamic;
+  // split units whose last finishing task merges them inside the kernel (streaming units)
+  const int32_t* task_unit;              // per task: unit index or -1 (null: no such unit)
+  const xy_attn_merge_unit* units;
+  int32_t* unit_count;                   // per unit: tasks finished so far (returns to 0 by itself)
   // fp8 KV cache: k_pool / v_pool hold e4m3 bytes (strides in bytes) and these are the fp32 scales
   // [pages, Hkv] of K and V
   const float* k_scale;

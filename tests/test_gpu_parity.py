@@ -68,7 +68,11 @@ def test_split_kv_long_decode_and_verify(kernel):
     assert info.num_merge_units > 0
     t = W.make_tensors(b)
     O, LSE = H.run_gpu(b, t, ctx=ctx)
-    assert ctx.last_launches() >= 2
+    # decode / tiny-verify units are merged inside the attention kernel (not by the SIMT kernel,
+    # which leaves every unit to the merge kernel); the merge kernel runs only for the others
+    inline = info.num_inline_merge_units
+    assert (inline > 0) == (kernel != xb.XY_KERNEL_REFERENCE)
+    assert ctx.last_launches() == (2 if info.num_merge_units > inline else 1)
     O_ref, LSE_ref = oracle.attention(b, t, H.SCALE)
     H.check_against_oracle(O, LSE, O_ref, LSE_ref, "split")
 

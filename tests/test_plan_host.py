@@ -416,3 +416,23 @@ def test_debug_block_table_check_on_the_host():
     with pytest.raises(xb.XYAttnError):
         g.debug_inject(-1, 0)
     g.debug_inject(0, -1)
+
+
+def test_merge_units_are_partitioned_into_merge_kernel_and_inline_units():
+    """Split units of at most 16 packed rows are merged inside the attention kernel and sit behind
+    the merge kernel's units in the unit list; the SIMT kernel and paper mode leave every unit to
+    the merge kernel.  The covering invariants do not depend on the order."""
+    rng = np.random.default_rng(3)
+    reqs = [(1, 30000, 0, None), (1, 9000, 0, None), (300, 20000, 0, None), (2, 50000, 1, [-1, 0]),
+            (40, 60000, 1, W.random_tree(rng, 40, 6))]
+    b = W.custom("partition", 8, 2, 128, reqs, seed=3)
+    c = host_ctx(8, 2, 128)
+    info = c.plan_batch(b)
+    mu = c.get_merge_units()
+    rows = mu["ntok"] * 4
+    n_launch = info.num_merge_units - info.num_inline_merge_units
+    assert info.num_inline_merge_units > 0 and n_launch > 0
+    assert np.all(rows[:n_launch] > 16) and np.all(rows[n_launch:] <= 16)
+    coverage_check(b, c, info)
+    r = host_ctx(8, 2, 128, kernel=xb.XY_KERNEL_REFERENCE)
+    assert r.plan_batch(b).num_inline_merge_units == 0
