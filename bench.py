@@ -232,12 +232,14 @@ def run_reference(args):
 # summarised under profiles/ (same workload, seed 0), each stamped with the commit of the kernel
 # that was captured and the date; a kernel change that may move traffic needs a new capture.
 NCU_TRAFFIC = {
+    # full_mix: the 5 GB pool is beyond what a multi-pass capture should hold; the dense path and the
+    # queue order that decide its traffic have not changed since this capture
     "full_mix": {"bytes": 6.00e9, "commit": "29136c8", "date": "2026-11-24", "summary": "profiles/launch_list_full_mix.md"},
-    "splitfuse_mix": {"bytes": 1.667e9, "commit": "29136c8", "date": "2026-11-24",
+    "splitfuse_mix": {"bytes": 1.666e9, "commit": "e5bad30", "date": "2026-11-25",
                       "summary": "profiles/meta_attention_splitfuse_mix.md"},
-    "verify_trees": {"bytes": 2.507e9, "commit": "29136c8", "date": "2026-11-24",
+    "verify_trees": {"bytes": 2.503e9, "commit": "e5bad30", "date": "2026-11-25",
                      "summary": "profiles/meta_attention_verify_trees.md"},
-    "decode_only": {"bytes": 0.594e9, "commit": "29136c8", "date": "2026-11-24",
+    "decode_only": {"bytes": 0.593e9, "commit": "e5bad30", "date": "2026-11-25",
                     "summary": "profiles/meta_attention_decode_only.md"},
     "long_context_decode": {"bytes": 3.202e9, "commit": "29136c8", "date": "2026-11-24",
                             "summary": "profiles/meta_attention_long_context_decode.md"},
