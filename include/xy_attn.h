@@ -50,9 +50,16 @@ enum { XY_MASK_CAUSAL = 0, XY_MASK_TREE = 1 };
 
 /* Which kernels xy_attn_run uses. */
 enum {
-  XY_KERNEL_AUTO = 0,      /* tcgen05 dense tiles + streaming decode tiles (the product path) */
+  XY_KERNEL_AUTO = 0,      /* the product path: tcgen05 dense tiles (prefill, verify; 256 packed rows per
+                              task) side by side with streaming tiles (decode) in one launch, tasks
+                              dealt from one mixed queue */
   XY_KERNEL_REFERENCE = 1, /* plain SIMT kernel for every tile: slow, kept for bisecting */
-  XY_KERNEL_MMA = 2        /* warp-level mma.sync tiles for every task (dense tasks too) */
+  XY_KERNEL_MMA = 2,       /* warp-level mma.sync tiles for every task (dense tasks too) */
+  XY_KERNEL_PAIR = 3       /* experimental: dense tiles on CTA pairs (tcgen05 cta_group::2, 512 packed
+                              rows per task), then the streaming tiles in a second launch.  Needs a
+                              bf16 cache, XY_PLAN_BALANCED and an even worker count (create fails
+                              otherwise); batches with shared-prefix groups run as XY_KERNEL_AUTO.
+                              Measured 8 - 20 % slower than XY_KERNEL_AUTO on the dense workloads. */
 };
 
 /* Task-Table construction (Section 3.3.1). */

@@ -31,6 +31,7 @@ XY_MASK_TREE = 1
 XY_KERNEL_AUTO = 0
 XY_KERNEL_REFERENCE = 1
 XY_KERNEL_MMA = 2
+XY_KERNEL_PAIR = 3
 
 XY_PLAN_BALANCED = 0
 XY_PLAN_PAPER = 1

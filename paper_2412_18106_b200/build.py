@@ -32,7 +32,9 @@ def _stale() -> bool:
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
-    deps = sources() + glob.glob(os.path.join(CSRC, "*.h")) + glob.glob(os.path.join(ROOT, "include", "*.h"))
+    deps = sources() + glob.glob(os.path.join(ROOT, "include", "*.h"))
+    for pat in ("*.h", "*.cuh", "*.inc"):
+        deps += glob.glob(os.path.join(CSRC, pat))
     return any(os.path.getmtime(d) > t for d in deps)
 
 
@@ -47,6 +49,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         obj = os.path.join(objdir, os.path.basename(src) + ".o")
         objs.append(obj)
         extra = ["-DXY_ENABLE_TRACE"] if os.environ.get("XY_BUILD_TRACE") == "1" else []
+        extra += os.environ.get("XY_NVCC_EXTRA", "").split()
         cmd = [nvcc] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + ["-x", "cu", "-c", src, "-o", obj]
         procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT)))
     failed = False

@@ -44,6 +44,7 @@ struct xy_attn_ctx {
   int last_launches = 0;
   MetaLaunchCache launch_cache;     // tensor maps of the last pools seen, kernel attributes set once
   int32_t dbg_skip_fill = -1;       // -1: none
+  bool pair = false;                // dense tasks run on CTA pairs (two launches per run: dense pairs, then streaming)
   bool debug_validate = false;      // XY_ATTN_DEBUG=1 at create: block tables are range-checked before launch
   std::vector<int32_t> dbg_bt;      // host copy of the block table for that check
   bool timing = false;
@@ -107,7 +108,9 @@ int xy_attn_create(const xy_attn_config* cfg, xy_attn_ctx** out) {
       cfg->max_tree_nodes < 0 || cfg->num_workers < 0 || cfg->max_splits < 0 ||
       cfg->workspace_bytes < 0 || cfg->tile_tokens < 0)
     return XY_ERR_INVALID_ARG;
-  if (cfg->kernel < XY_KERNEL_AUTO || cfg->kernel > XY_KERNEL_MMA) return XY_ERR_INVALID_ARG;
+  if (cfg->kernel < XY_KERNEL_AUTO || cfg->kernel > XY_KERNEL_PAIR) return XY_ERR_INVALID_ARG;
+  if (cfg->kernel == XY_KERNEL_PAIR && (cfg->kv_dtype != XY_KV_BF16 || cfg->plan_mode != XY_PLAN_BALANCED))
+    return XY_ERR_INVALID_ARG;
   if (cfg->plan_mode != XY_PLAN_BALANCED && cfg->plan_mode != XY_PLAN_PAPER) return XY_ERR_INVALID_ARG;
   if (cfg->kv_dtype != XY_KV_BF16 && cfg->kv_dtype != XY_KV_FP8_E4M3) return XY_ERR_INVALID_ARG;
   if (cfg->kv_dtype == XY_KV_FP8_E4M3 && cfg->page_size < 16) return XY_ERR_UNSUPPORTED;
@@ -137,6 +140,11 @@ int xy_attn_create(const xy_attn_config* cfg, xy_attn_ctx** out) {
     c->num_workers = 148;
   }
 
+  c->pair = cfg->kernel == XY_KERNEL_PAIR;
+  if (c->pair && (c->num_workers < 2 || c->num_workers % 2 != 0)) {
+    delete c;
+    return XY_ERR_INVALID_ARG;
+  }
   const int G = cfg->num_q_heads / cfg->num_kv_heads;
   const int sub_tok = 128 / G > 0 ? 128 / G : 1;
   const int tile_tok = cfg->plan_mode == XY_PLAN_PAPER
@@ -217,7 +225,7 @@ int xy_attn_plan_shared(xy_attn_ctx* ctx, const xy_attn_request* reqs, int32_t n
   std::string err;
   int rc = build_plan(ctx->cfg, ctx->num_workers, ctx->cap_partial_rows, reqs, num_reqs,
                       tree_parents, num_parents, &ctx->plan, &err, ctx->cache.capacity > 0 ? &ctx->cache : nullptr,
-                      groups, num_groups);
+                      groups, num_groups, ctx->pair && num_groups == 0);
   if (rc != XY_OK) {
     ctx->plan = PlanResult();
     return set_err(ctx, rc, err);
@@ -406,8 +414,26 @@ int run_impl(xy_attn_ctx* ctx, const void* q, int64_t q_token_stride, const void
 
   if (cfg.kernel == XY_KERNEL_REFERENCE) {
     XY_CUDA(ctx, launch_reference(a, ctx->num_workers, s));
+  } else if (p.queue_dense >= 0 && !fp8) {
+    // pair plan: the dense tasks on CTA pairs, then the streaming tasks on single CTAs
+    RunArgs d = a;
+    d.num_tasks = p.queue_dense;
+    if (d.num_tasks > 0) {
+      XY_CUDA(ctx, launch_pair_dense(d, ctx->num_workers, num_pages, &ctx->launch_cache, s));
+      ctx->last_launches += 1;
+    }
+    RunArgs st = a;
+    st.queue = a.queue + p.queue_dense;
+    st.num_tasks = a.num_tasks - p.queue_dense;
+    st.queue_head = a.queue_head + 1;  // its own head word, cleared by the same memset
+    if (st.num_tasks > 0) {
+      XY_CUDA(ctx, launch_meta(st, ctx->num_workers, num_pages, false, &ctx->launch_cache, s));
+      ctx->last_launches += 1;
+    }
+    ctx->last_launches -= 1;  // counted once more below
   } else {
-    XY_CUDA(ctx, launch_meta(a, ctx->num_workers, num_pages, cfg.kernel == XY_KERNEL_AUTO && p.info.num_dense_tasks > 0,
+    XY_CUDA(ctx, launch_meta(a, ctx->num_workers, num_pages,
+                             (cfg.kernel == XY_KERNEL_AUTO || cfg.kernel == XY_KERNEL_PAIR) && p.info.num_dense_tasks > 0,
                              &ctx->launch_cache, s));
   }
   ctx->last_launches += 1;

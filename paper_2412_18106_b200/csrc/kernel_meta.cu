@@ -1583,6 +1583,8 @@ meta_attention_kernel(const __grid_constant__ MetaParams P, const __grid_constan
   }
 }
 
+#include "kernel_pair.inc"
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
@@ -1601,8 +1603,9 @@ EncodeTiledFn encode_fn() {
 }
 
 // 4-D map over a paged pool [pages, Hkv, B, D]: box = one page of one head, 64 elements wide.
+// box_tokens: tokens per box (0: a whole page)
 bool encode_pool_map(CUtensorMap* m, const void* pool, int64_t num_pages, int num_kv_heads, int page_size,
-                     int64_t page_stride, int64_t head_stride, int64_t token_stride, bool fp8) {
+                     int64_t page_stride, int64_t head_stride, int64_t token_stride, bool fp8, int box_tokens = 0) {
   EncodeTiledFn fn = encode_fn();
   if (fn == nullptr) return false;
   // bf16: two boxes of 64 elements per row; e4m3 bytes: one box of 128 - 128 B per row either way
@@ -1611,7 +1614,7 @@ bool encode_pool_map(CUtensorMap* m, const void* pool, int64_t num_pages, int nu
                         static_cast<cuuint64_t>(num_kv_heads), static_cast<cuuint64_t>(num_pages)};
   cuuint64_t strides[3] = {static_cast<cuuint64_t>(token_stride) * esz, static_cast<cuuint64_t>(head_stride) * esz,
                            static_cast<cuuint64_t>(page_stride) * esz};
-  cuuint32_t box[4] = {fp8 ? 128u : 64u, static_cast<cuuint32_t>(page_size), 1, 1};
+  cuuint32_t box[4] = {fp8 ? 128u : 64u, static_cast<cuuint32_t>(box_tokens > 0 ? box_tokens : page_size), 1, 1};
   cuuint32_t estr[4] = {1, 1, 1, 1};
   CUresult r = fn(m, fp8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(pool), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -1660,6 +1663,45 @@ cudaError_t launch_meta(const RunArgs& a, int num_workers, int64_t num_pages, bo
   }
   MetaParams P{a};
   kernel<<<num_workers, kThreads, kSmemTotal, s>>>(P, *k_map, *v_map);
+  return cudaGetLastError();
+}
+
+// Dense tasks on CTA pairs: `a.queue` / `a.num_tasks` / `a.queue_head` describe the dense part of the
+// plan's queue.  num_workers CTAs (even) = num_workers / 2 pairs.
+cudaError_t launch_pair_dense(const RunArgs& a, int num_workers, int64_t num_pages, MetaLaunchCache* cache,
+                              cudaStream_t s) {
+  if (num_workers < 2) return cudaErrorInvalidValue;
+  if (!cache->attr_set[3]) {
+    cudaError_t e = cudaFuncSetAttribute(pair_dense_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTotal);
+    if (e != cudaSuccess) return e;
+    cache->attr_set[3] = true;
+  }
+  CUtensorMap* k_map = reinterpret_cast<CUtensorMap*>(cache->pair_maps[0]);
+  CUtensorMap* v_map = reinterpret_cast<CUtensorMap*>(cache->pair_maps[1]);
+  const bool same = cache->pair_valid && cache->pk_pool == a.k_pool && cache->pv_pool == a.v_pool &&
+                    cache->p_num_pages == num_pages && cache->p_page_stride == a.page_stride &&
+                    cache->p_head_stride == a.head_stride && cache->p_token_stride == a.token_stride &&
+                    cache->p_num_kv_heads == a.num_kv_heads && cache->p_page_size == a.page_size;
+  if (!same) {
+    cache->pair_valid = false;
+    // K: boxes of at most 64 tokens (a CTA stages 64 keys of a tile); V: whole pages, 64 columns
+    if (!encode_pool_map(k_map, a.k_pool, num_pages, a.num_kv_heads, a.page_size, a.page_stride, a.head_stride,
+                         a.token_stride, false, a.page_size < 64 ? a.page_size : 64) ||
+        !encode_pool_map(v_map, a.v_pool, num_pages, a.num_kv_heads, a.page_size, a.page_stride, a.head_stride,
+                         a.token_stride, false))
+      return cudaErrorInvalidValue;
+    cache->pk_pool = a.k_pool;
+    cache->pv_pool = a.v_pool;
+    cache->p_num_pages = num_pages;
+    cache->p_page_stride = a.page_stride;
+    cache->p_head_stride = a.head_stride;
+    cache->p_token_stride = a.token_stride;
+    cache->p_num_kv_heads = a.num_kv_heads;
+    cache->p_page_size = a.page_size;
+    cache->pair_valid = true;
+  }
+  MetaParams P{a};
+  pair_dense_kernel<<<num_workers & ~1, kThreads, kSmemTotal, s>>>(P, *k_map, *v_map);
   return cudaGetLastError();
 }
 

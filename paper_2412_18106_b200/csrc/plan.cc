@@ -28,6 +28,7 @@ namespace {
 // task boundary costs ~3 us (Q load, pipeline refill, epilogue).
 constexpr float kDenseVisitUs = 2.30f;
 constexpr float kStreamVisitUs = 1.00f;
+constexpr float kPairVisitUs = 1.35f;
 constexpr float kTaskFixedUs = 3.0f;
 constexpr int kMinChunkTiles = 4;
 // A task may cost at most this fraction of the mean per-worker load before its KV range is
@@ -55,7 +56,7 @@ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_capacity,
                const xy_attn_request* reqs, int32_t num_reqs, const int32_t* tree_parents,
                int32_t num_parents, PlanResult* out, std::string* err, PlanCache* cache,
-               const xy_attn_prefix_group* groups, int32_t num_groups) {
+               const xy_attn_prefix_group* groups, int32_t num_groups, bool pair) {
   *out = PlanResult();
   char buf[256];
   auto fail = [&](int code, const char* msg) {
@@ -185,7 +186,7 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
   // ---- a2: decomposition ----------------------------------------------------------------
   const bool paper = cfg.plan_mode == XY_PLAN_PAPER;
   const int sub_tok = std::max(1, 128 / G);  // tokens of one 128-row sub-tile
-  const int subtiles = dense_subtiles(cfg);
+  const int subtiles = pair ? 4 : dense_subtiles(cfg);  // a CTA pair holds two sub-tiles of 256 rows
   const int dense_tok = paper ? (cfg.tile_tokens > 0 ? cfg.tile_tokens : sub_tok) : subtiles * sub_tok;
   if (paper && cfg.kernel != XY_KERNEL_REFERENCE && dense_tok * G > 128 * subtiles)
     return fail(XY_ERR_UNSUPPORTED, "paper-mode tile_tokens x (Hq/Hkv) exceeds the rows one task may hold");
@@ -221,7 +222,8 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
         if (u.kind == 1) {
           u.visit_cost = kStreamVisitUs;
         } else {
-          u.visit_cost = kDenseVisitUs * static_cast<float>(std::max(1, ceil_div(rows, 256)));
+          // a pair advances one key tile of a 512-row unit per kPairVisitUs, which keeps two workers busy
+          u.visit_cost = pair ? 2.f * kPairVisitUs : kDenseVisitUs * static_cast<float>(std::max(1, ceil_div(rows, 256)));
         }
         u.paper_load = static_cast<float>(rows) * static_cast<float>(visible);
         units.push_back(u);
@@ -238,6 +240,7 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
   out->shape.push_back(cfg.plan_mode * 4 + cfg.kernel);
   out->shape.push_back(cfg.max_splits);
   out->shape.push_back(cfg.kv_dtype);
+  out->shape.push_back(pair ? 1 : 0);
   for (const Unit& u : units) {
     out->shape.push_back(u.req);
     out->shape.push_back(u.kv_head);
@@ -265,6 +268,7 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
       out->task_cost = e.task_cost;
       out->worker_off = e.worker_off;
       out->queue = e.queue;
+      out->queue_dense = e.queue_dense;
       out->merges = e.merges;
       out->task_unit = e.task_unit;
       out->num_launch_merges = e.num_launch_merges;
@@ -288,9 +292,16 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
     max_splits = 32;
     if (n_stream > 0) max_splits = std::max(32, std::min(128, ceil_div(num_workers, n_stream)));
   }
-  double total_cost = 0.0;
-  for (const Unit& u : units) total_cost += kTaskFixedUs + u.visit_cost * (u.nkt - u.kt0);
+  double total_cost = 0.0, total_kind[2] = {0.0, 0.0};
+  for (const Unit& u : units) {
+    const double c = kTaskFixedUs + u.visit_cost * (u.nkt - u.kt0);
+    total_cost += c;
+    total_kind[u.kind == 1 ? 1 : 0] += c;
+  }
   float cap = static_cast<float>(total_cost / std::max(1, num_workers) * kTaskCapFraction);
+  // pair plans run the two kinds one after the other: each kind is capped against its own mean load
+  float cap_kind[2] = {static_cast<float>(total_kind[0] / std::max(1, num_workers) * kTaskCapFraction),
+                       static_cast<float>(total_kind[1] / std::max(1, num_workers) * kTaskCapFraction)};
   const float dense_factor = kDenseCapFactor;
   std::vector<int> chunk_tiles(units.size(), 0);
   for (int attempt = 0; attempt < 64; ++attempt) {
@@ -300,8 +311,10 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
       int nsplit = 1;
       if (!paper) {
         const int nt = u.nkt - u.kt0;
-        const float cost = u.visit_cost * nt;
-        const float cap_u = u.kind == 1 ? cap : cap * dense_factor;
+        // (a pair task occupies two workers: its duration is half its cost)
+        const float cost = pair && u.kind == 0 ? 0.5f * u.visit_cost * nt : u.visit_cost * nt;
+        const float cap_u = pair ? (u.kind == 1 ? cap_kind[1] : cap_kind[0] * dense_factor)
+                                 : (u.kind == 1 ? cap : cap * dense_factor);
         nsplit = static_cast<int>(std::ceil(cost / std::max(cap_u, 1e-3f)));
         nsplit = std::min(nsplit, max_splits);
         nsplit = std::min(nsplit, std::max(1, nt / kMinChunkTiles));
@@ -315,6 +328,8 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
     }
     if (prow <= partial_row_capacity) break;
     cap *= 1.5f;  // fewer splits until the partials fit the workspace
+    cap_kind[0] *= 1.5f;
+    cap_kind[1] *= 1.5f;
     if (attempt == 63) return fail(XY_ERR_CAPACITY, "split-KV workspace too small");
   }
 
@@ -475,9 +490,11 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
       d.swap(regrouped);
     }
     size_t next[2] = {0, 0};
+    if (pair) out->queue_dense = static_cast<int32_t>(by_kind[0].size());
     for (size_t pos = 0; pos < order.size(); ++pos) {
       int kd;
-      if (next[0] >= by_kind[0].size()) kd = 1;
+      if (pair) kd = next[0] < by_kind[0].size() ? 0 : 1;  // two launches: all dense tasks, then all streaming tasks
+      else if (next[0] >= by_kind[0].size()) kd = 1;
       else if (next[1] >= by_kind[1].size()) kd = 0;
       else {
         // A task must start while at least its own length of work per worker remains, or it
@@ -523,6 +540,7 @@ int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_c
     slot->task_cost = out->task_cost;
     slot->worker_off = out->worker_off;
     slot->queue = out->queue;
+    slot->queue_dense = out->queue_dense;
     slot->merges = out->merges;
     slot->task_unit = out->task_unit;
     slot->num_launch_merges = out->num_launch_merges;

@@ -47,6 +47,8 @@ struct PlanResult {
   std::vector<float> task_cost;            // parallel to tasks
   std::vector<int32_t> worker_off;         // num_workers + 1
   std::vector<int32_t> queue;              // task indices by descending cost (dynamic dealing)
+  int32_t queue_dense = -1;                // pair plans: the first queue_dense entries are the dense tasks (for the
+                                           // CTA-pair launch), the rest the streaming tasks; -1: one mixed queue
   std::vector<xy_attn_merge_unit> merges;  // units merged by the merge kernel first, then those merged in the attention kernel
   std::vector<int32_t> task_unit;          // parallel to tasks: index in `merges` of the unit the last finisher merges
                                            // inside the attention kernel, or -1
@@ -70,6 +72,7 @@ struct PlanCache {
     std::vector<xy_attn_task> tasks;
     std::vector<float> task_cost;
     std::vector<int32_t> worker_off, queue;
+    int32_t queue_dense = -1;
     std::vector<xy_attn_merge_unit> merges;
     std::vector<int32_t> task_unit;
     int32_t num_launch_merges = 0;
@@ -84,17 +87,19 @@ struct PlanCache {
 
 // 128-row sub-tiles one dense task may hold (the tcgen05 path ping-pongs two; the others one).
 inline int dense_subtiles(const xy_attn_config& cfg) {
-  return cfg.kernel == XY_KERNEL_AUTO && cfg.kv_dtype == XY_KV_BF16 ? 2 : 1;
+  return (cfg.kernel == XY_KERNEL_AUTO || cfg.kernel == XY_KERNEL_PAIR) && cfg.kv_dtype == XY_KV_BF16 ? 2 : 1;
 }
 
 // Host-only planning.  Returns XY_OK or an error code and fills `err`.
+// `pair`: plan for the CTA-pair dense kernel: dense units of up to 512 packed rows, the dense and
+// the streaming tasks in separate parts of the queue (they run in two launches).
 // `cache` (nullable): Task-Tables of earlier plans; a plan whose decomposition equals a cached one
 // takes its Task-Table from there and only rebuilds the Token-Table and the tree masks.
 // `groups` (nullable): shared-prefix decode groups, see xy_attn_plan_shared.
 int build_plan(const xy_attn_config& cfg, int num_workers, int64_t partial_row_capacity,
                const xy_attn_request* reqs, int32_t num_reqs, const int32_t* tree_parents,
                int32_t num_parents, PlanResult* out, std::string* err, PlanCache* cache = nullptr,
-               const xy_attn_prefix_group* groups = nullptr, int32_t num_groups = 0);
+               const xy_attn_prefix_group* groups = nullptr, int32_t num_groups = 0, bool pair = false);
 
 // Arguments every attention kernel takes.
 struct RunArgs {

@@ -28,12 +28,20 @@ struct MetaLaunchCache {
   int64_t num_pages = 0, page_stride = 0, head_stride = 0, token_stride = 0;
   int32_t num_kv_heads = 0, page_size = 0;
   bool valid = false, fp8 = false;
-  bool attr_set[3] = {false, false, false};
+  bool attr_set[4] = {false, false, false, false};
+  // the CTA-pair kernel's maps (K in boxes of at most 64 tokens)
+  alignas(64) unsigned char pair_maps[2][128];
+  const void* pk_pool = nullptr;
+  const void* pv_pool = nullptr;
+  int64_t p_num_pages = 0, p_page_stride = 0, p_head_stride = 0, p_token_stride = 0;
+  int32_t p_num_kv_heads = 0, p_page_size = 0;
+  bool pair_valid = false;
 };
 
 cudaError_t launch_reference(const RunArgs& a, int num_workers, cudaStream_t s);
 cudaError_t launch_meta(const RunArgs& a, int num_workers, int64_t num_pages, bool umma, MetaLaunchCache* cache,
                         cudaStream_t s);
+cudaError_t launch_pair_dense(const RunArgs& a, int num_workers, int64_t num_pages, MetaLaunchCache* cache, cudaStream_t s);
 cudaError_t launch_merge_units(const MergeArgs& a, int num_units, int max_rows, int max_parts, cudaStream_t s);
 cudaError_t launch_merge_plain(const float* o_part, const float* lse_part, int num_splits,
                                int64_t rows, uint16_t* o, float* lse, cudaStream_t s);

@@ -436,3 +436,27 @@ def test_merge_units_are_partitioned_into_merge_kernel_and_inline_units():
     coverage_check(b, c, info)
     r = host_ctx(8, 2, 128, kernel=xb.XY_KERNEL_REFERENCE)
     assert r.plan_batch(b).num_inline_merge_units == 0
+
+
+@pytest.mark.parametrize("name", ["splitfuse_mix", "verify_trees", "full_mix"])
+def test_pair_plans_put_dense_tasks_of_up_to_512_rows_first(name):
+    """XY_KERNEL_PAIR plans for the CTA-pair dense kernel: dense tasks hold up to 512 packed rows
+    (two 256-row sub-tiles, each split over two CTAs) and come first in the queue, siblings
+    together; the streaming tasks follow in descending order of length.  XY_KERNEL_AUTO keeps
+    256-row tasks in one mixed queue.  Coverage holds for both."""
+    b = W.CONFIGS[name]()
+    G = b.num_q_heads // b.num_kv_heads
+    for kernel, max_rows in ((xb.XY_KERNEL_PAIR, 512), (xb.XY_KERNEL_AUTO, 256)):
+        c = host_ctx(b.num_q_heads, b.num_kv_heads, b.page_size, kernel=kernel)
+        info = c.plan_batch(b)
+        coverage_check(b, c, info)
+        tasks, queue = c.get_tasks(), c.get_queue()
+        dense = tasks[tasks["kind"] == 0]
+        assert int((dense["ntok"] * G).max()) <= max_rows
+        if kernel == xb.XY_KERNEL_PAIR:
+            assert int((dense["ntok"] * G).max()) > 256
+            kinds = tasks["kind"][queue]
+            nd = int((kinds == 0).sum())
+            assert np.all(kinds[:nd] == 0) and np.all(kinds[nd:] == 1)
+            ntiles = (tasks["kt_hi"] - tasks["kt_lo"])[queue]
+            assert np.all(np.diff(ntiles[nd:]) <= 0)
