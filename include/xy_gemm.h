@@ -38,6 +38,22 @@ extern "C" {
 int xy_gemm_run(const void* a, int64_t lda, const void* w, int64_t ldw, void* c, int64_t ldc, int32_t M,
                 int32_t N, int32_t K, int32_t tile_n, void* stream);
 
+/* The same with DEVICE scratch memory, which lets the last, partial wave of tiles be split along K
+ * over every SM when K is long (K >= 8192 and a last wave of at most 0.6 of the SMs; measured
+ * rule): each SM multiplies a run of K chunks of one or two of those tiles and leaves fp32 partial
+ * sums in the scratch; a second, small kernel on the same stream adds a tile's partial sums in a
+ * fixed order (bit-reproducible) and stores the tile.  No thread waits for another CTA.
+ *   workspace        DEVICE, 16-byte aligned, at least xy_gemm_workspace_bytes() bytes (a smaller
+ *                    one, or NULL, gives xy_gemm_run's behaviour); contents do not matter.  Calls
+ *                    that may run at the same time need scratch of their own.
+ * Errors as xy_gemm_run. */
+int xy_gemm_run_ws(const void* a, int64_t lda, const void* w, int64_t ldw, void* c, int64_t ldc, int32_t M,
+                   int32_t N, int32_t K, int32_t tile_n, void* workspace, int64_t workspace_bytes, void* stream);
+
+/* Bytes of scratch xy_gemm_run_ws can use on the current device (2 slots of a 128 x 256 fp32 tile
+ * per SM: 38.8 MB with 148 SMs), or -1 if the device cannot be queried. */
+int64_t xy_gemm_workspace_bytes(void);
+
 /* Status of the device-side waits of the GEMM kernels on the current device since the last call of
  * this function: 0, or XY_ERR_DEVICE_TIMEOUT if a bounded wait inside a kernel gave up (the
  * kernel then returns early and its output is invalid).  Synchronises the device. */

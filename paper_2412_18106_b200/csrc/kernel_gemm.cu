@@ -45,7 +45,43 @@ struct GemmParams {
   int64_t ldc;
   int32_t M, N, K;
   int32_t m_tiles, n_tiles;
+  // Work split.  Tiles [0, wave_tiles) are computed whole, tile blockIdx.x + i * gridDim.x by CTA
+  // blockIdx.x (wave_tiles is a multiple of the grid size).  The K chunks of the remaining sk_tiles
+  // tiles form one line of sk_tiles * k_chunks units, of which CTA b takes units [b * upc, (b + 1) * upc):
+  // at most two segments, each part of one tile (upc <= k_chunks).
+  int32_t wave_tiles, sk_tiles, upc;
+  float* ws;     // partial sums: slot 2 b + s of CTA b's segment s, [kTileN / 4][128] float4
+  int32_t grid;  // CTAs of the GEMM kernel (the fix-up kernel derives the segments from it)
 };
+
+// One piece of work of a CTA: K chunks [kc_lo, kc_hi) of a tile; slot < 0: the whole tile.
+struct GemmItem {
+  int tile, kc_lo, kc_hi, slot;
+};
+__device__ __forceinline__ bool gemm_item(const GemmParams& P, int k_chunks, int idx, GemmItem& it) {
+  const int G = static_cast<int>(gridDim.x), b = static_cast<int>(blockIdx.x);
+  if (b + idx * G < P.wave_tiles) {
+    it.tile = b + idx * G;
+    it.kc_lo = 0;
+    it.kc_hi = k_chunks;
+    it.slot = -1;
+    return true;
+  }
+  if (P.sk_tiles == 0) return false;
+  const int s = idx - P.wave_tiles / G;  // with split tiles, wave_tiles is a multiple of the grid size
+  if (s < 0 || s > 1) return false;
+  const int u0 = b * P.upc, u1 = min(u0 + P.upc, P.sk_tiles * k_chunks);
+  if (u0 >= u1) return false;
+  const int first = u0 / k_chunks;
+  const int lo = s == 0 ? u0 : (first + 1) * k_chunks;
+  const int hi = s == 0 ? min(u1, (first + 1) * k_chunks) : u1;
+  if (lo >= hi) return false;
+  it.tile = P.wave_tiles + first + s;
+  it.kc_lo = lo - (first + s) * k_chunks;
+  it.kc_hi = hi - (first + s) * k_chunks;
+  it.slot = (it.kc_lo == 0 && it.kc_hi == k_chunks) ? -1 : 2 * b + s;
+  return true;
+}
 
 struct __align__(8) GemmBarriers {
   uint64_t full[8], empty[8];
@@ -92,9 +128,11 @@ smooth_gemm_kernel(const GemmParams P, const __grid_constant__ CUtensorMap a_map
     prefetch_tensormap(&w_map);
     uint32_t pos = 0;
     bool dead = false;
-    for (int t = blockIdx.x; t < num_tiles && !dead; t += gridDim.x) {
+    GemmItem it;
+    for (int idx = 0; !dead && gemm_item(P, k_chunks, idx, it); ++idx) {
+      const int t = it.tile;
       const int m0 = (t % P.m_tiles) * kTileM, n0 = (t / P.m_tiles) * kTileN;
-      for (int kc = 0; kc < k_chunks; ++kc, ++pos) {
+      for (int kc = it.kc_lo; kc < it.kc_hi; ++kc, ++pos) {
         const uint32_t s = pos % Cfg::kStages, use = pos / Cfg::kStages;
         if (use > 0 && !mbar_wait(smem_u32(&bars->empty[s]), (use - 1) & 1u, status)) {
           atomicExch(&g_gemm_status, XY_ERR_DEVICE_TIMEOUT);
@@ -117,7 +155,8 @@ smooth_gemm_kernel(const GemmParams P, const __grid_constant__ CUtensorMap a_map
                                 ((static_cast<uint32_t>(kTileM) >> 4) << 24);
     uint32_t pos = 0, local = 0;
     bool dead = false;
-    for (int t = blockIdx.x; t < num_tiles && !dead; t += gridDim.x, ++local) {
+    GemmItem it;
+    for (int idx = 0; !dead && gemm_item(P, k_chunks, idx, it); ++idx, ++local) {
       const uint32_t buf = local & 1u, use = local >> 1;
       if (use > 0 && !mbar_wait(smem_u32(&bars->acc_empty[buf]), (use - 1) & 1u, status)) {
         atomicExch(&g_gemm_status, XY_ERR_DEVICE_TIMEOUT);
@@ -125,7 +164,7 @@ smooth_gemm_kernel(const GemmParams P, const __grid_constant__ CUtensorMap a_map
       }
       tc_fence_after();
       const uint32_t d_tmem = tmem + buf * kTileN;
-      for (int kc = 0; kc < k_chunks; ++kc, ++pos) {
+      for (int kc = it.kc_lo; kc < it.kc_hi; ++kc, ++pos) {
         const uint32_t s = pos % Cfg::kStages;
         if (!mbar_wait(smem_u32(&bars->full[s]), (pos / Cfg::kStages) & 1u, status)) {
           atomicExch(&g_gemm_status, XY_ERR_DEVICE_TIMEOUT);
@@ -137,7 +176,8 @@ smooth_gemm_kernel(const GemmParams P, const __grid_constant__ CUtensorMap a_map
         const uint32_t w_lo = (((base + s * Cfg::kStageBytes + kABytes) >> 4) & 0x3FFFu) | (1u << 16);
 #pragma unroll
         for (int k16 = 0; k16 < 4; ++k16)
-          umma_ss64(d_tmem, kDescHi | (a_lo + k16 * 2), kDescHi | (w_lo + k16 * 2), kIdesc, (kc | k16) ? 1u : 0u);
+          umma_ss64(d_tmem, kDescHi | (a_lo + k16 * 2), kDescHi | (w_lo + k16 * 2), kIdesc,
+                    (kc > it.kc_lo || k16) ? 1u : 0u);
         umma_commit(smem_u32(&bars->empty[s]));  // the stage is free once these MMAs have read it
       }
       if (!dead) umma_commit(smem_u32(&bars->acc_full[buf]));
@@ -147,35 +187,60 @@ smooth_gemm_kernel(const GemmParams P, const __grid_constant__ CUtensorMap a_map
     const int q = warp & 3;  // tensor-memory lanes 32 q .. 32 q + 31 belong to this warp
     const int row_in_tile = q * 32 + lane;
     uint32_t local = 0;
-    for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++local) {
+    GemmItem it;
+    for (int idx = 0; gemm_item(P, k_chunks, idx, it); ++idx, ++local) {
       const uint32_t buf = local & 1u;
       if (!mbar_wait(smem_u32(&bars->acc_full[buf]), (local >> 1) & 1u, status)) {
         atomicExch(&g_gemm_status, XY_ERR_DEVICE_TIMEOUT);
         break;
       }
       tc_fence_after();
+      const int t = it.tile;
       const int m0 = (t % P.m_tiles) * kTileM, n0 = (t / P.m_tiles) * kTileN;
       const int row = m0 + row_in_tile;
       const uint32_t t_acc = tmem + (static_cast<uint32_t>(q * 32) << 16) + buf * kTileN;
       uint16_t* crow = P.c + static_cast<int64_t>(row) * P.ldc + n0;
+      if (it.slot < 0) {
+#pragma unroll 2
+        for (int c0 = 0; c0 < kTileN; c0 += 32) {
+          uint32_t v[32];
+          tmem_ld_32x32b_x32(t_acc + c0, v);
+          tmem_wait_ld();
+          if (row < P.M) {  // selective write: virtual padding rows are never stored
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+              if (n0 + c0 + g * 8 < P.N) {
+                uint4 o;
+                o.x = pack_bf16(__uint_as_float(v[g * 8 + 0]), __uint_as_float(v[g * 8 + 1]));
+                o.y = pack_bf16(__uint_as_float(v[g * 8 + 2]), __uint_as_float(v[g * 8 + 3]));
+                o.z = pack_bf16(__uint_as_float(v[g * 8 + 4]), __uint_as_float(v[g * 8 + 5]));
+                o.w = pack_bf16(__uint_as_float(v[g * 8 + 6]), __uint_as_float(v[g * 8 + 7]));
+                *reinterpret_cast<uint4*>(crow + c0 + g * 8) = o;
+              }
+            }
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bars->acc_empty[buf]));
+        continue;
+      }
+      // A segment of a split tile: leave the fp32 partial sums in this segment's slot (column
+      // group by column group, 128 consecutive rows each: coalesced).  gemm_fixup_kernel, launched
+      // behind this kernel, adds a tile's segments in the order of the CTAs and stores the tile.
+      // (Letting the segment that arrives last add them was measured first: one CTA then reads
+      // every partial sum of its tile with 32 - 64 KiB in flight, 20 - 40 us for a 128 x 256 tile.)
+      float4* slot = reinterpret_cast<float4*>(P.ws) + static_cast<int64_t>(it.slot) * (kTileN / 4) * kTileM;
 #pragma unroll 2
       for (int c0 = 0; c0 < kTileN; c0 += 32) {
         uint32_t v[32];
         tmem_ld_32x32b_x32(t_acc + c0, v);
         tmem_wait_ld();
-        if (row < P.M) {  // selective write: virtual padding rows are never stored
 #pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            if (n0 + c0 + g * 8 < P.N) {
-              uint4 o;
-              o.x = pack_bf16(__uint_as_float(v[g * 8 + 0]), __uint_as_float(v[g * 8 + 1]));
-              o.y = pack_bf16(__uint_as_float(v[g * 8 + 2]), __uint_as_float(v[g * 8 + 3]));
-              o.z = pack_bf16(__uint_as_float(v[g * 8 + 4]), __uint_as_float(v[g * 8 + 5]));
-              o.w = pack_bf16(__uint_as_float(v[g * 8 + 6]), __uint_as_float(v[g * 8 + 7]));
-              *reinterpret_cast<uint4*>(crow + c0 + g * 8) = o;
-            }
-          }
-        }
+        for (int g = 0; g < 8; ++g)
+          slot[(c0 / 4 + g) * kTileM + row_in_tile] =
+              make_float4(__uint_as_float(v[4 * g]), __uint_as_float(v[4 * g + 1]), __uint_as_float(v[4 * g + 2]),
+                          __uint_as_float(v[4 * g + 3]));
       }
       tc_fence_before();
       __syncwarp();
@@ -190,6 +255,53 @@ smooth_gemm_kernel(const GemmParams P, const __grid_constant__ CUtensorMap a_map
   }
 }
 
+
+// Adds the partial sums of the split tiles and stores them.  Grid: (column blocks of 32, split
+// tiles); 128 threads = the tile's rows.  The segments of tile sk belong to the consecutive CTAs
+// whose unit ranges meet [sk * k_chunks, (sk + 1) * k_chunks); a tile with one segment was stored
+// whole by the GEMM kernel.  Every load of a thread is independent of the others (up to 8 per
+// segment in flight), and the sum runs in the order of the CTAs: bit-reproducible.
+template <int kTileN>
+__global__ void __launch_bounds__(128) gemm_fixup_kernel(const GemmParams P) {
+  const int sk = blockIdx.y, k_chunks = (P.K + kChunkK - 1) / kChunkK;
+  const int b_first = (sk * k_chunks) / P.upc, b_last = ((sk + 1) * k_chunks - 1) / P.upc;
+  if (b_first == b_last) return;
+  const int t = P.wave_tiles + sk;
+  const int m0 = (t % P.m_tiles) * kTileM, n0 = (t / P.m_tiles) * kTileN;
+  const int row_in_tile = threadIdx.x, row = m0 + row_in_tile;
+  const int c0 = blockIdx.x * 32;
+  float4 acc[8];
+#pragma unroll
+  for (int g = 0; g < 8; ++g) acc[g] = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int bb = b_first; bb <= b_last; ++bb) {
+    const int seg = sk - (bb * P.upc) / k_chunks;  // 0 or 1: which of that CTA's segments is this tile
+    const float4* src = reinterpret_cast<const float4*>(P.ws) +
+                        static_cast<int64_t>(2 * bb + seg) * (kTileN / 4) * kTileM + row_in_tile;
+    float4 x[8];
+#pragma unroll
+    for (int g = 0; g < 8; ++g) x[g] = __ldcg(src + (c0 / 4 + g) * kTileM);
+#pragma unroll
+    for (int g = 0; g < 8; ++g) {
+      acc[g].x += x[g].x;
+      acc[g].y += x[g].y;
+      acc[g].z += x[g].z;
+      acc[g].w += x[g].w;
+    }
+  }
+  if (row >= P.M) return;
+  uint16_t* crow = P.c + static_cast<int64_t>(row) * P.ldc + n0;
+#pragma unroll
+  for (int g = 0; g < 4; ++g) {
+    if (n0 + c0 + g * 8 < P.N) {
+      uint4 o;
+      o.x = pack_bf16(acc[2 * g].x, acc[2 * g].y);
+      o.y = pack_bf16(acc[2 * g].z, acc[2 * g].w);
+      o.z = pack_bf16(acc[2 * g + 1].x, acc[2 * g + 1].y);
+      o.w = pack_bf16(acc[2 * g + 1].z, acc[2 * g + 1].w);
+      *reinterpret_cast<uint4*>(crow + c0 + g * 8) = o;
+    }
+  }
+}
 
 // ------------------------------------------------------------------------------------------
 // Split-K variant for small token counts (few tiles).  A whole-K tile is one serial
@@ -399,9 +511,15 @@ bool encode_matrix_map(CUtensorMap* m, const void* ptr, int64_t rows, int64_t K,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Bytes of scratch the split of the last, partial wave of tiles needs: two partial-sum slots of a
+// 128 x kTileN fp32 tile per CTA.
+constexpr int64_t gemm_workspace_bytes(int tile_n, int num_sms) {
+  return static_cast<int64_t>(num_sms) * 2 * kTileM * tile_n * 4;
+}
+
 template <int kTileN>
 cudaError_t launch_gemm(const void* a, int64_t lda, const void* w, int64_t ldw, void* c, int64_t ldc, int M, int N,
-                        int K, int num_sms, cudaStream_t s) {
+                        int K, int num_sms, void* workspace, int64_t workspace_bytes, cudaStream_t s) {
   using Cfg = GemmCfg<kTileN>;
   auto kernel = smooth_gemm_kernel<kTileN>;
   static bool attr_set[64] = {false};  // per device: the opt-in to large dynamic shared memory
@@ -424,8 +542,33 @@ cudaError_t launch_gemm(const void* a, int64_t lda, const void* w, int64_t ldw, 
   P.K = K;
   P.m_tiles = (M + kTileM - 1) / kTileM;
   P.n_tiles = (N + kTileN - 1) / kTileN;
-  const int tiles = P.m_tiles * P.n_tiles;
-  kernel<<<tiles < num_sms ? tiles : num_sms, kGemmThreads, Cfg::kSmem, s>>>(P, a_map, w_map);
+  const int tiles = P.m_tiles * P.n_tiles, k_chunks = (K + kChunkK - 1) / kChunkK;
+  int grid = tiles < num_sms ? tiles : num_sms;
+  P.wave_tiles = tiles;
+  P.sk_tiles = 0;
+  P.upc = k_chunks;
+  P.ws = nullptr;
+  // With scratch memory, the tiles of the last, partial wave are split along K over every SM when
+  // the chain of K chunks is long: a tile is a serial chain on one SM, so a last wave of few
+  // tiles otherwise costs a whole tile time.  Measured on the Linear shapes at M = 4096: Down
+  // (K = 14336, 512 tiles = 3.46 waves) 401 -> 358 us; with K = 4096 the split tail and its fix-up
+  // cost what the shorter wave saves (QKV 155 -> 158 us: full waves there run at the L2's pace,
+  // 28 us per wave against 22 us of MMAs, and a thin last wave is already cheaper than a full
+  // one), so chains under 128 chunks are left whole.  With fewer tiles than SMs (M <= 512) the
+  // split was level with whole tiles (QKV M = 256: 26.3 against 25.3 us) and is not used.
+  const int rest = tiles % num_sms;
+  if (kTileN >= 32 && workspace != nullptr && workspace_bytes >= gemm_workspace_bytes(kTileN, num_sms) &&
+      tiles > num_sms && rest > 0 && k_chunks >= 128 && rest * 5 <= num_sms * 3) {
+    const int units = rest * k_chunks;
+    P.wave_tiles = tiles - rest;
+    P.sk_tiles = rest;
+    P.upc = (units + grid - 1) / grid;
+    P.ws = static_cast<float*>(workspace);
+  }
+  P.grid = grid;
+  kernel<<<grid, kGemmThreads, Cfg::kSmem, s>>>(P, a_map, w_map);
+  if (P.sk_tiles > 0)
+    gemm_fixup_kernel<kTileN><<<dim3(kTileN / 32, P.sk_tiles), 128, 0, s>>>(P);
   return cudaGetLastError();
 }
 
@@ -474,8 +617,24 @@ cudaError_t launch_gemm_splitk(const void* a, int64_t lda, const void* w, int64_
 }  // namespace
 }  // namespace xy
 
+extern "C" int64_t xy_gemm_workspace_bytes(void) {
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+    return -1;
+  return xy::gemm_workspace_bytes(256, sms);
+}
+
 extern "C" int xy_gemm_run(const void* a, int64_t lda, const void* w, int64_t ldw, void* c, int64_t ldc, int32_t M,
                            int32_t N, int32_t K, int32_t tile_n, void* stream) {
+  return xy_gemm_run_ws(a, lda, w, ldw, c, ldc, M, N, K, tile_n, nullptr, 0, stream);
+}
+
+extern "C" int xy_gemm_run_ws(const void* a, int64_t lda, const void* w, int64_t ldw, void* c, int64_t ldc, int32_t M,
+                              int32_t N, int32_t K, int32_t tile_n, void* workspace, int64_t workspace_bytes,
+                              void* stream) {
+  if (workspace != nullptr && ((reinterpret_cast<uintptr_t>(workspace) & 15) || workspace_bytes < 0))
+    return XY_ERR_INVALID_ARG;
   if (M < 0 || N < 8 || K < 8 || (N % 8) || (K % 8) || (lda % 8) || (ldw % 8) || (ldc % 8) || lda < K || ldw < K ||
       ldc < N)
     return XY_ERR_INVALID_ARG;
@@ -519,10 +678,10 @@ extern "C" int xy_gemm_run(const void* a, int64_t lda, const void* w, int64_t ld
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   cudaError_t e;
   switch (tile_n) {
-    case 256: e = xy::launch_gemm<256>(a, lda, w, ldw, c, ldc, M, N, K, sms, s); break;
-    case 128: e = xy::launch_gemm<128>(a, lda, w, ldw, c, ldc, M, N, K, sms, s); break;
-    case 64: e = xy::launch_gemm<64>(a, lda, w, ldw, c, ldc, M, N, K, sms, s); break;
-    default: e = xy::launch_gemm<32>(a, lda, w, ldw, c, ldc, M, N, K, sms, s); break;
+    case 256: e = xy::launch_gemm<256>(a, lda, w, ldw, c, ldc, M, N, K, sms, workspace, workspace_bytes, s); break;
+    case 128: e = xy::launch_gemm<128>(a, lda, w, ldw, c, ldc, M, N, K, sms, workspace, workspace_bytes, s); break;
+    case 64: e = xy::launch_gemm<64>(a, lda, w, ldw, c, ldc, M, N, K, sms, workspace, workspace_bytes, s); break;
+    default: e = xy::launch_gemm<32>(a, lda, w, ldw, c, ldc, M, N, K, sms, workspace, workspace_bytes, s); break;
   }
   return e == cudaSuccess ? XY_OK : XY_ERR_CUDA;
 }

@@ -8,7 +8,7 @@ import torch
 
 from . import binding as xb
 
-GEMM_EXPORTS = ("xy_gemm_run", "xy_gemm_device_status")
+GEMM_EXPORTS = ("xy_gemm_run", "xy_gemm_run_ws", "xy_gemm_workspace_bytes", "xy_gemm_device_status")
 
 _ready = False
 
@@ -20,14 +20,29 @@ def _lib():
         vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
         L.xy_gemm_run.argtypes = [vp, i64, vp, i64, vp, i64, i32, i32, i32, i32, vp]
         L.xy_gemm_run.restype = ctypes.c_int
+        L.xy_gemm_run_ws.argtypes = [vp, i64, vp, i64, vp, i64, i32, i32, i32, i32, vp, i64, vp]
+        L.xy_gemm_run_ws.restype = ctypes.c_int
+        L.xy_gemm_workspace_bytes.argtypes = []
+        L.xy_gemm_workspace_bytes.restype = i64
         L.xy_gemm_device_status.argtypes = [ctypes.POINTER(i32)]
         L.xy_gemm_device_status.restype = ctypes.c_int
         _ready = True
     return L
 
 
-def xy_gemm_run(a: torch.Tensor, w: torch.Tensor, c: torch.Tensor, tile_n: int = 0, stream=None) -> None:
-    """c[M, N] = a[M, K] w[N, K]^T (bf16 CUDA tensors, last dimension contiguous; rows may be strided)."""
+def xy_gemm_workspace(device) -> torch.Tensor:
+    """Zero-filled scratch of xy_gemm_workspace_bytes() bytes for xy_gemm_run(..., workspace=...)."""
+    with torch.cuda.device(device):
+        n = int(_lib().xy_gemm_workspace_bytes())
+    if n < 0:
+        raise xb.XYAttnError(xb.XY_ERR_CUDA, "xy_gemm_workspace_bytes failed")
+    return torch.zeros(n, dtype=torch.uint8, device=device)
+
+
+def xy_gemm_run(a: torch.Tensor, w: torch.Tensor, c: torch.Tensor, tile_n: int = 0, stream=None,
+                workspace: Optional[torch.Tensor] = None) -> None:
+    """c[M, N] = a[M, K] w[N, K]^T (bf16 CUDA tensors, last dimension contiguous; rows may be strided).
+    With `workspace` (from xy_gemm_workspace) the call goes through xy_gemm_run_ws."""
     for t in (a, w, c):
         if t.dtype != torch.bfloat16 or not t.is_cuda or t.dim() != 2 or (t.numel() and t.stride(1) != 1):
             raise ValueError("xy_gemm_run takes 2-D bf16 CUDA tensors with a contiguous last dimension")
@@ -36,9 +51,15 @@ def xy_gemm_run(a: torch.Tensor, w: torch.Tensor, c: torch.Tensor, tile_n: int =
     if w.shape[1] != K or tuple(c.shape) != (M, N):
         raise ValueError("shape mismatch")
     lda = a.stride(0) if M > 1 else max(K, a.stride(0))
-    rc = _lib().xy_gemm_run(a.data_ptr(), lda, w.data_ptr(), w.stride(0), c.data_ptr(),
-                            c.stride(0) if M > 1 else max(N, c.stride(0)), M, N, K, int(tile_n),
-                            xb._stream_ptr(stream))
+    ldc = c.stride(0) if M > 1 else max(N, c.stride(0))
+    if workspace is None:
+        rc = _lib().xy_gemm_run(a.data_ptr(), lda, w.data_ptr(), w.stride(0), c.data_ptr(), ldc, M, N, K,
+                                int(tile_n), xb._stream_ptr(stream))
+    else:
+        if workspace.dtype != torch.uint8 or not workspace.is_cuda or not workspace.is_contiguous():
+            raise ValueError("workspace must be a contiguous uint8 CUDA tensor")
+        rc = _lib().xy_gemm_run_ws(a.data_ptr(), lda, w.data_ptr(), w.stride(0), c.data_ptr(), ldc, M, N, K,
+                                   int(tile_n), workspace.data_ptr(), workspace.numel(), xb._stream_ptr(stream))
     if rc != 0:
         raise xb.XYAttnError(rc, "xy_gemm_run failed")
 

@@ -90,3 +90,35 @@ def test_small_token_counts_take_the_split_k_path(M, N, K):
     must match the oracle like the single-CTA product does (ragged N, K not a multiple of the
     split, rows past M untouched)."""
     check(M, N, K, 0, seed=M + N)
+
+
+@pytest.mark.parametrize("shape", [(600, 4000, 8264, 128), (640, 7936, 8200, 256), (1100, 4096, 8192, 0)])
+def test_last_wave_split_along_k_with_scratch_matches_oracle_and_repeats_bitwise(shape):
+    """More tiles than SMs, a thin last wave and a long K: with scratch memory the last wave's
+    tiles are split along K over all SMs and a fix-up kernel adds the partial sums.  Ragged M, N
+    and K included; the result must match the oracle, repeat bit for bit, and stay inside
+    [0, M) x [0, N)."""
+    M, N, K, tile_n = shape
+    g = torch.Generator().manual_seed(K)
+    a = torch.randn((M, K), generator=g).to(torch.bfloat16)
+    w = torch.randn((N, K), generator=g).to(torch.bfloat16)
+    ws = xg.xy_gemm_workspace(torch.device("cuda:0"))
+    ws.fill_(0xFF)  # contents of the scratch must not matter
+    c_buf = torch.full((M + 1, N + 8), float("nan"), dtype=torch.bfloat16, device="cuda")
+    c = c_buf[:M, :N]
+    xg.xy_gemm_run(a.cuda(), w.cuda(), c, tile_n=tile_n, workspace=ws)
+    c2 = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+    xg.xy_gemm_run(a.cuda(), w.cuda(), c2, tile_n=tile_n, workspace=ws)
+    assert xg.xy_gemm_device_status() == 0
+    assert torch.equal(c, c2)
+    got = c.float().cpu().numpy().astype(np.float64)
+    ref = G.linear(a, w)
+    tol = 2.0 ** -8 * np.abs(ref) + 2.0 ** -14 * np.sqrt(K)
+    bad = np.abs(got - ref) > tol
+    assert not bad.any(), (shape, float(np.abs(got - ref).max()), int(bad.sum()))
+    rest = c_buf.float().cpu().numpy()
+    assert np.isnan(rest[M:, :]).all() and np.isnan(rest[:M, N:]).all()
+    # without scratch the same call computes whole tiles: same result within the tolerance
+    c3 = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+    xg.xy_gemm_run(a.cuda(), w.cuda(), c3, tile_n=tile_n)
+    assert not (np.abs(c3.float().cpu().numpy().astype(np.float64) - ref) > tol).any()
