@@ -22,18 +22,24 @@
 extern "C" {
 #endif
 
+/* tile_n flag: compute 256 x tile_n tiles on pairs of CTAs (tcgen05 cta_group::2; tile_n 128 or 256). */
+#define XY_GEMM_PAIR 0x1000
+
 /* Asynchronous on `stream` (a cudaStream_t, may be 0); allocates nothing; no host sync.
  *   a  DEVICE bf16, row m at a + m*lda (elements), K contiguous; lda >= K
  *   w  DEVICE bf16, row n at w + n*ldw, K contiguous (the layout of a Linear weight); ldw >= K
  *   c  DEVICE bf16, row m at c + m*ldc, N contiguous; ldc >= N; written for m < M, n < N only
  *   M >= 0 (0: nothing to do), N >= 8, K >= 8; N, K, lda, ldw, ldc multiples of 8; the three base
  *   pointers 16-byte aligned
- *   tile_n  columns per tile: 32, 64, 128, 256, or 0 to let the library choose: 256 when the
- *           128 x 256 tiles give every SM a tile, else 128; and for M <= 512 with few tiles a
- *           split of K over a thread-block cluster (2..8 CTAs per 128 x 128 tile, partial sums
- *           added through distributed shared memory), which puts the idle SMs to work
+ *   tile_n  columns per tile: 32, 64, 128, 256 (128-row tiles on single CTAs), XY_GEMM_PAIR | 128
+ *           or XY_GEMM_PAIR | 256 (256-row tiles on CTA pairs), or 0 to let the library choose:
+ *           256 x 256 pair tiles when M > 128 pads to a multiple of 256 with at most 15 % waste
+ *           and those tiles number at least a quarter of the SMs; else, for M <= 512 with few
+ *           tiles, a split of K over a thread-block cluster (2..8 CTAs per 128 x 128 tile, partial
+ *           sums added through distributed shared memory), which puts the idle SMs to work; else
+ *           128 x 256 tiles when they give half of the SMs a tile, else 128 x 128
  * Returns XY_OK, XY_ERR_INVALID_ARG (null pointer, bad size or alignment), XY_ERR_UNSUPPORTED
- * (tile_n not in {0, 32, 64, 128, 256}) or XY_ERR_CUDA.  Calls on one stream are ordered; the caller
+ * (tile_n not one of the values above) or XY_ERR_CUDA.  Calls on one stream are ordered; the caller
  * owns all buffers. */
 int xy_gemm_run(const void* a, int64_t lda, const void* w, int64_t ldw, void* c, int64_t ldc, int32_t M,
                 int32_t N, int32_t K, int32_t tile_n, void* stream);

@@ -256,6 +256,176 @@ smooth_gemm_kernel(const GemmParams P, const __grid_constant__ CUtensorMap a_map
 }
 
 
+// ------------------------------------------------------------------------------------------
+// CTA-pair variant for large problems: a cluster of two CTAs computes a 256 x kTileN tile with
+// tcgen05.mma.cta_group::2 (M = 256).  CTA r holds rows [128 r, 128 r + 128) of the tile's A and of
+// its accumulator and stages rows [kTileN / 2 * r, + kTileN / 2) of W: per 64-element K chunk a CTA
+// loads 16 KiB of A and kTileN * 64 bytes of W for 256 x kTileN x 64 multiply-adds of the pair,
+// two thirds of the single-CTA kernel's operand bytes per flop (what the full waves of the
+// single-CTA kernel are bound by: 28 us per wave against 22 us of MMAs), and an MMA of the pair
+// costs 64 cycles per 128 columns against 81.  Every CTA issues its own copies (no multicast);
+// their bytes are counted on the leader's barrier; completions (tcgen05.commit) arrive in both
+// CTAs; the peer's epilogue warps return an accumulator with a remote arrive.
+template <int kTileN>
+struct PairGemmCfg {
+  static constexpr int kWBytes = (kTileN / 2) * kChunkK * 2;
+  static constexpr int kStageBytes = kABytes + kWBytes;
+  static constexpr int kStages = kTileN == 256 ? 6 : 8;
+  static constexpr int kSmem = 1024 + kStages * kStageBytes + 256;
+  static constexpr uint32_t kTmemCols = 2 * kTileN;
+};
+
+template <int kTileN>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
+smooth_gemm_pair_kernel(const GemmParams P, const __grid_constant__ CUtensorMap a_map,
+                        const __grid_constant__ CUtensorMap w_map) {
+  using Cfg = PairGemmCfg<kTileN>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  GemmBarriers* bars =
+      reinterpret_cast<GemmBarriers*>(smem_raw + (base - smem_u32(smem_raw)) + Cfg::kStages * Cfg::kStageBytes);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const bool leader = rank == 0;
+  const volatile int32_t* status = &g_gemm_status;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < Cfg::kStages; ++s) {
+      mbar_init(smem_u32(&bars->full[s]), 1);   // leader: one arming arrive, bytes of both CTAs
+      mbar_init(smem_u32(&bars->empty[s]), 1);  // each CTA: one commit
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&bars->acc_full[b]), 1);   // each CTA: one commit
+      mbar_init(smem_u32(&bars->acc_empty[b]), 8);  // leader: four epilogue warps of each CTA
+    }
+    fence_mbar_init();
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(smem_u32(&bars->tmem_base), Cfg::kTmemCols);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();  // the peer's barriers exist before anything arrives on them
+  tc_fence_after();
+  const uint32_t tmem = bars->tmem_base;
+  const int num_tiles = P.m_tiles * P.n_tiles;  // m_tiles counts 256-row tiles here
+  const int k_chunks = (P.K + kChunkK - 1) / kChunkK;
+  const int cluster = static_cast<int>(blockIdx.x >> 1), clusters = static_cast<int>(gridDim.x >> 1);
+  auto wait_cluster = [&](uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < (1u << 22); ++i) {
+      if (mbar_try_wait_cluster(bar, parity)) return true;
+      if ((i & 4095u) == 4095u && status[0] != 0) return false;
+    }
+    return false;
+  };
+
+  if (warp == 0 && lane == 0) {
+    // ---------------------------------------------------------------- producer (both CTAs)
+    prefetch_tensormap(&a_map);
+    prefetch_tensormap(&w_map);
+    const uint32_t full_leader = cluster_map(smem_u32(&bars->full[0]), 0);
+    uint32_t pos = 0;
+    bool dead = false;
+    for (int t = cluster; t < num_tiles && !dead; t += clusters) {
+      const int m0 = (t % P.m_tiles) * 256 + 128 * static_cast<int>(rank);
+      const int n0 = (t / P.m_tiles) * kTileN + (kTileN / 2) * static_cast<int>(rank);
+      for (int kc = 0; kc < k_chunks; ++kc, ++pos) {
+        const uint32_t s = pos % Cfg::kStages, use = pos / Cfg::kStages;
+        if (use > 0 && !wait_cluster(smem_u32(&bars->empty[s]), (use - 1) & 1u)) {
+          atomicExch(&g_gemm_status, XY_ERR_DEVICE_TIMEOUT);
+          dead = true;
+          break;
+        }
+        if (leader) mbar_arrive_expect_tx(smem_u32(&bars->full[s]), 2 * Cfg::kStageBytes);
+        const uint32_t dst = base + s * Cfg::kStageBytes, bar = full_leader + s * 8u;
+        tma_load_2d_pair(dst, &a_map, bar, kc * kChunkK, m0);           // rows past M arrive as zeros
+        tma_load_2d_pair(dst + kABytes, &w_map, bar, kc * kChunkK, n0);  // rows past N likewise
+      }
+    }
+  } else if (warp == 1 && lane == 0 && leader) {
+    // ---------------------------------------------------------------- MMA issuer (leader)
+    constexpr uint64_t kDescHi = static_cast<uint64_t>((1024u >> 4) | (1u << 14) | (2u << 29)) << 32;
+    constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((static_cast<uint32_t>(kTileN) >> 3) << 17) |
+                                ((256u >> 4) << 24);
+    uint32_t pos = 0, local = 0;
+    bool dead = false;
+    for (int t = cluster; t < num_tiles && !dead; t += clusters, ++local) {
+      const uint32_t buf = local & 1u, use = local >> 1;
+      if (use > 0 && !wait_cluster(smem_u32(&bars->acc_empty[buf]), (use - 1) & 1u)) {
+        atomicExch(&g_gemm_status, XY_ERR_DEVICE_TIMEOUT);
+        break;
+      }
+      tc_fence_after();
+      const uint32_t d_tmem = tmem + buf * kTileN;
+      for (int kc = 0; kc < k_chunks; ++kc, ++pos) {
+        const uint32_t s = pos % Cfg::kStages;
+        if (!wait_cluster(smem_u32(&bars->full[s]), (pos / Cfg::kStages) & 1u)) {
+          atomicExch(&g_gemm_status, XY_ERR_DEVICE_TIMEOUT);
+          dead = true;
+          break;
+        }
+        tc_fence_after();
+        const uint32_t a_lo = (((base + s * Cfg::kStageBytes) >> 4) & 0x3FFFu) | (1u << 16);
+        const uint32_t w_lo = (((base + s * Cfg::kStageBytes + kABytes) >> 4) & 0x3FFFu) | (1u << 16);
+#pragma unroll
+        for (int k16 = 0; k16 < 4; ++k16)
+          umma2_ss64(d_tmem, kDescHi | (a_lo + k16 * 2), kDescHi | (w_lo + k16 * 2), kIdesc, (kc | k16) ? 1u : 0u);
+        umma2_commit_both(smem_u32(&bars->empty[s]));  // the stage is free in both CTAs
+      }
+      if (!dead) umma2_commit_both(smem_u32(&bars->acc_full[buf]));
+    }
+  } else if (warp >= 2) {
+    // ---------------------------------------------------------------- epilogue (both CTAs)
+    const int q = warp & 3;
+    const int row_in_tile = q * 32 + lane;
+    const uint32_t acc_empty_leader = cluster_map(smem_u32(&bars->acc_empty[0]), 0);
+    uint32_t local = 0;
+    for (int t = cluster; t < num_tiles; t += clusters, ++local) {
+      const uint32_t buf = local & 1u;
+      if (!wait_cluster(smem_u32(&bars->acc_full[buf]), (local >> 1) & 1u)) {
+        atomicExch(&g_gemm_status, XY_ERR_DEVICE_TIMEOUT);
+        break;
+      }
+      tc_fence_after();
+      const int m0 = (t % P.m_tiles) * 256 + 128 * static_cast<int>(rank), n0 = (t / P.m_tiles) * kTileN;
+      const int row = m0 + row_in_tile;
+      const uint32_t t_acc = tmem + (static_cast<uint32_t>(q * 32) << 16) + buf * kTileN;
+      uint16_t* crow = P.c + static_cast<int64_t>(row) * P.ldc + n0;
+#pragma unroll 2
+      for (int c0 = 0; c0 < kTileN; c0 += 32) {
+        uint32_t v[32];
+        tmem_ld_32x32b_x32(t_acc + c0, v);
+        tmem_wait_ld();
+        if (row < P.M) {
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            if (n0 + c0 + g * 8 < P.N) {
+              uint4 o;
+              o.x = pack_bf16(__uint_as_float(v[g * 8 + 0]), __uint_as_float(v[g * 8 + 1]));
+              o.y = pack_bf16(__uint_as_float(v[g * 8 + 2]), __uint_as_float(v[g * 8 + 3]));
+              o.z = pack_bf16(__uint_as_float(v[g * 8 + 4]), __uint_as_float(v[g * 8 + 5]));
+              o.w = pack_bf16(__uint_as_float(v[g * 8 + 6]), __uint_as_float(v[g * 8 + 7]));
+              *reinterpret_cast<uint4*>(crow + c0 + g * 8) = o;
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) {
+        if (leader) mbar_arrive(smem_u32(&bars->acc_empty[buf])); else mbar_arrive_remote(acc_empty_leader + buf * 8u);
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();  // neither CTA leaves while the other may still touch its memory
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem, Cfg::kTmemCols);
+  }
+}
+
 // Adds the partial sums of the split tiles and stores them.  Grid: (column blocks of 32, split
 // tiles); 128 threads = the tile's rows.  The segments of tile sk belong to the consecutive CTAs
 // whose unit ranges meet [sk * k_chunks, (sk + 1) * k_chunks); a tile with one segment was stored
@@ -573,6 +743,37 @@ cudaError_t launch_gemm(const void* a, int64_t lda, const void* w, int64_t ldw, 
 }
 
 
+template <int kTileN>
+cudaError_t launch_gemm_pair(const void* a, int64_t lda, const void* w, int64_t ldw, void* c, int64_t ldc, int M, int N,
+                             int K, int num_sms, cudaStream_t s) {
+  using Cfg = PairGemmCfg<kTileN>;
+  auto kernel = smooth_gemm_pair_kernel<kTileN>;
+  static bool attr_set[64] = {false};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmem);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64) attr_set[dev] = true;
+  }
+  CUtensorMap a_map, w_map;
+  if (!encode_matrix_map(&a_map, a, M, K, lda, kTileM) || !encode_matrix_map(&w_map, w, N, K, ldw, kTileN / 2))
+    return cudaErrorInvalidValue;
+  GemmParams P = {};
+  P.c = static_cast<uint16_t*>(c);
+  P.ldc = ldc;
+  P.M = M;
+  P.N = N;
+  P.K = K;
+  P.m_tiles = (M + 255) / 256;
+  P.n_tiles = (N + kTileN - 1) / kTileN;
+  const int tiles = P.m_tiles * P.n_tiles, clusters = num_sms / 2;
+  const int grid = 2 * (tiles < clusters ? tiles : clusters);
+  kernel<<<grid, kGemmThreads, Cfg::kSmem, s>>>(P, a_map, w_map);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_gemm_splitk(const void* a, int64_t lda, const void* w, int64_t ldw, void* c, int64_t ldc, int M,
                                int N, int K, int splits, cudaStream_t s) {
   using Cfg = GemmCfg<128>;
@@ -638,6 +839,11 @@ extern "C" int xy_gemm_run_ws(const void* a, int64_t lda, const void* w, int64_t
   if (M < 0 || N < 8 || K < 8 || (N % 8) || (K % 8) || (lda % 8) || (ldw % 8) || (ldc % 8) || lda < K || ldw < K ||
       ldc < N)
     return XY_ERR_INVALID_ARG;
+  bool pair = (tile_n & XY_GEMM_PAIR) != 0;
+  if (pair) {
+    tile_n &= ~XY_GEMM_PAIR;
+    if (tile_n != 128 && tile_n != 256) return XY_ERR_UNSUPPORTED;
+  }
   if (tile_n != 0 && tile_n != 32 && tile_n != 64 && tile_n != 128 && tile_n != 256) return XY_ERR_UNSUPPORTED;
   if (M == 0) return XY_OK;
   if (!a || !w || !c || (reinterpret_cast<uintptr_t>(a) & 15) || (reinterpret_cast<uintptr_t>(w) & 15) ||
@@ -651,6 +857,25 @@ extern "C" int xy_gemm_run_ws(const void* a, int64_t lda, const void* w, int64_t
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
       return XY_ERR_CUDA;
     if (dev >= 0 && dev < 64) sm_count[dev] = sms;
+  }
+  if (tile_n == 0 && !pair && sms >= 2 && M > 128) {
+    // 256 x 256 tiles on CTA pairs when the padding of M to 256 rows stays under 15 % and the tiles
+    // give at least half of the pairs work: measured best or level with the best from 1024 tokens
+    // on (at 4096 tokens QKV 155 -> 143 us, OProj 105 -> 96, GateUp 667 -> 609, Down 369 -> 339), and
+    // at 256 tokens for GateUp only (112 tiles: 67 -> 61 us; the shapes with 16 - 24 tiles stay with
+    // 128-column tiles or the cluster split of K).
+    const int mp = (M + 255) / 256, np = (N + 255) / 256;
+    if ((mp * 256 - M) * 100 <= 15 * mp * 256 && mp * np * 4 >= sms) {
+      pair = true;
+      tile_n = 256;
+    }
+  }
+  if (pair) {
+    if (sms < 2) return XY_ERR_UNSUPPORTED;
+    const cudaError_t e =
+        tile_n == 256 ? xy::launch_gemm_pair<256>(a, lda, w, ldw, c, ldc, M, N, K, sms, static_cast<cudaStream_t>(stream))
+                      : xy::launch_gemm_pair<128>(a, lda, w, ldw, c, ldc, M, N, K, sms, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? XY_OK : XY_ERR_CUDA;
   }
   if (tile_n == 0 && M <= 512) {
     // Few tiles and one long serial chain over K per tile: split K over a cluster when that puts
@@ -669,11 +894,12 @@ extern "C" int xy_gemm_run_ws(const void* a, int64_t lda, const void* w, int64_t
     }
   }
   if (tile_n == 0) {
-    // 128 x 256 tiles read the least of A and W per flop; they are used when they give every SM
-    // a tile.  Below that 128 x 128 (measured: narrower tiles are not faster for small M, where
-    // the time is launch and pipeline-fill latency).
+    // 128 x 256 tiles read the least of A and W per flop; they are used when they give at least
+    // half of the SMs a tile (measured: OProj at 1024 tokens, 128 such tiles, 28 us against 44 us
+    // with 128 x 128; GateUp at 16 tokens 44 against 49 us).  Below that 128 x 128 (narrower tiles
+    // are not faster for small M, where the time is launch and pipeline-fill latency).
     const int64_t tiles256 = static_cast<int64_t>((M + 127) / 128) * ((N + 255) / 256);
-    tile_n = tiles256 >= sms ? 256 : 128;
+    tile_n = tiles256 * 2 >= sms ? 256 : 128;
   }
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   cudaError_t e;

@@ -10,6 +10,8 @@ from . import binding as xb
 
 GEMM_EXPORTS = ("xy_gemm_run", "xy_gemm_run_ws", "xy_gemm_workspace_bytes", "xy_gemm_device_status")
 
+XY_GEMM_PAIR = 0x1000  # tile_n flag: 256-row tiles on CTA pairs
+
 _ready = False
 
 

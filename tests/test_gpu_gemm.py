@@ -122,3 +122,23 @@ def test_last_wave_split_along_k_with_scratch_matches_oracle_and_repeats_bitwise
     c3 = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
     xg.xy_gemm_run(a.cuda(), w.cuda(), c3, tile_n=tile_n)
     assert not (np.abs(c3.float().cpu().numpy().astype(np.float64) - ref) > tol).any()
+
+
+PAIR = xg.XY_GEMM_PAIR
+
+
+@pytest.mark.parametrize("tile_n", [PAIR | 128, PAIR | 256])
+@pytest.mark.parametrize("M", [1, 129, 255, 256, 257, 600])
+def test_cta_pair_tiles_any_token_count_matches_oracle(M, tile_n):
+    check(M, 392, 328, tile_n, seed=M)  # N and K end in partial tiles / chunks; rows of the peer CTA may all be padding
+
+
+@pytest.mark.parametrize("tile_n", [PAIR | 128, PAIR | 256])
+def test_cta_pair_tiles_several_tiles_per_pair_and_strided_rows(tile_n):
+    check(1000, 5000, 1024, tile_n, seed=4)          # 4 x 20 (or 40) tiles over 74 pairs: two accumulators in use
+    check(300, 520, 72, tile_n, seed=8, lda=80, ldc=528)
+
+
+def test_library_choice_covers_pair_tiles():
+    check(1024, 4096, 512, 0, seed=11)   # picks 256 x 256 pair tiles
+    check(520, 28672, 128, 0, seed=12)   # 520 rows pad to 768: stays on single-CTA tiles
