@@ -28,7 +28,6 @@ constexpr int kTileM = 128;
 constexpr int kChunkK = 64;  // elements per K chunk = one 128-byte swizzle row
 constexpr int kGemmThreads = 192;
 constexpr int kABytes = kTileM * kChunkK * 2;  // 16 KiB
-
 __device__ int32_t g_gemm_status;
 
 template <int kTileN>
