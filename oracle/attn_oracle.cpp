@@ -30,7 +30,7 @@
 // logsumexp on gathered K/V; page-permutation invariance; key-shift identity;
 // merge identity over arbitrary partitions; GQA special cases; append-then-gather round trip.
 //
-// fp8 KV-cache variant (a variant the survey of the paper's related directions lists; the paper
+// fp8 KV-cache variant (an extension beside the paper's method: the paper
 // itself defines no fp8 cache, so format, scale granularity and rounding are this build's
 // reading - parity unpinned by the paper): K and V are stored as e4m3 bytes (1 sign, 4 exponent
 // bits of bias 7, 3 mantissa bits, no infinities, 0x7F / 0xFF = NaN) with one fp32 scale per
