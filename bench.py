@@ -248,7 +248,7 @@ NCU_TRAFFIC = {
 
 def ncu_traffic(name):
     e = NCU_TRAFFIC.get(name)
-    return (e["bytes"], "ncu capture of commit %s, %s (%s)" % (e["commit"], e["date"], e["summary"])) if e else (None, None)
+    return (e["bytes"], "ncu, commit %s, %s (%s)" % (e["commit"], e["date"], e["summary"])) if e else (None, None)
 
 
 def workload_config(name, batch):
@@ -432,9 +432,9 @@ def measure_gemm(dev, peaks, steps=20):
     """SmoothGEMM (Section 5) on the Linear shapes of the benchmark model (hidden 4096, 32 + 2 x 8
     heads of 128, MLP 14336) for token counts from a decode batch to a full chunk.  Device-timed
     back-to-back launches (the smallest cases are bound by launch latency, not by the kernel).
-    Fractions: flops against the measured burst bf16 peak (each kernel is timed alone), bytes
-    (A + W + C once) against the measured copy bandwidth; the larger of the two is the roofline.
-    The library GEMM (torch.matmul) is timed beside it for context."""
+    `frac`: the roofline time (flops at the measured burst bf16 peak, each kernel being timed alone, or
+    the bytes of A + W + C once at the measured copy bandwidth, whichever is longer) over the
+    measured time.  `lib_us`: the library GEMM (torch.matmul) timed beside it, for context."""
     import torch
 
     from paper_2412_18106_b200 import gemm as xg
@@ -462,8 +462,8 @@ def measure_gemm(dev, peaks, steps=20):
             ms_lib = timed(lambda: torch.matmul(a, w.T, out=c))
             flops, byts = 2.0 * M * N * K, 2.0 * (M * K + N * K + M * N)
             t_roof = max(flops / (peaks["bf16_tflops"] * 1e12), byts / (peaks["hbm_gbs"] * 1e9))
-            out["%s_M%d" % (name, M)] = {"ms": ms, "tflops": flops / ms / 1e9, "gbs": byts / ms / 1e6,
-                                         "roofline_frac_measured": t_roof / (ms * 1e-3), "library_ms": ms_lib}
+            out["%s_M%d" % (name, M)] = {"us": round(ms * 1e3, 1), "tflops": round(flops / ms / 1e9, 1),
+                                         "frac": round(t_roof / (ms * 1e-3), 3), "lib_us": round(ms_lib * 1e3, 1)}
     assert xg.xy_gemm_device_status() == 0
     return out
 
@@ -547,7 +547,7 @@ def measure_fp8_decode(dev, peaks, steps=200):
     k_ms = attn_ms / runs
     return {"kernel_ms": k_ms, "merge_ms": merge_ms / runs, "kv_bytes_fp8": int(info.kv_bytes), "algorithmic_bytes": alg,
             "gbs": alg / (k_ms * 1e-3) / 1e9, "bound": "hbm", "roofline_frac_measured": alg / (peaks["hbm_gbs"] * 1e9) / (k_ms * 1e-3),
-            "note": "widening e4m3 to f16 runs on the conversion unit (16 results per clock and SM): that, not HBM, bounds this path"}
+            "note": "bound by the e4m3 -> f16 conversion unit (16 results / clk / SM), not by HBM"}
 
 
 def measure_long_decode(kernel, dev, peaks, steps=20):
@@ -823,10 +823,9 @@ def main():
         e2e = {"value": job_flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": n_e2e,
                "host_clock_ms_per_step": e2e_host_ms, "bit_identical_to_resident_run": e2e_same,
-               "includes": "per step: host plan + H2D(fused QKV of the new tokens, block table, task tables) + "
-                           "KV-cache append + run + D2H(O, LSE); steps software-pipelined over three streams "
-                           "(copies of neighbouring steps overlap the kernels); the cached history is "
-                           "device-resident state; CUDA events around all steps, the last one after a device synchronize"}
+               "includes": "per step: host plan, H2D (fused QKV of the new tokens, block table, task tables), "
+                           "KV append, run, D2H (O, LSE); steps pipelined over three streams; cached history "
+                           "device-resident; CUDA events around all steps"}
 
     if world > 1:  # every collective is behind us: all ranks leave the group together
         dist.barrier()
