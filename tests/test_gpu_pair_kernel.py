@@ -81,3 +81,34 @@ def test_pair_kernel_wait_that_runs_out_reports_and_context_stays_usable():
     O, LSE = H.run_gpu(b, t, ctx=ctx)
     O_ref, LSE_ref = oracle.attention(b, t, H.SCALE)
     H.check_against_oracle(O, LSE, O_ref, LSE_ref, "pair after a timed-out run")
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_pair_kernel_random_batches_match_oracle_and_repeat_bitwise(seed):
+    """Random head ratios, page sizes, even worker counts and request mixes on the pair kernel."""
+    rng = np.random.default_rng(100 + seed)
+    hkv = int(rng.choice([1, 2, 4]))
+    G = int(rng.choice([1, 2, 4, 7, 8, 16]))
+    page = int(rng.choice([16, 32, 64, 128]))
+    reqs = []
+    for _ in range(int(rng.integers(1, 20))):
+        kind = rng.random()
+        kv = int(rng.integers(0, 1500)) if rng.random() < 0.8 else int(rng.integers(1500, 6000))
+        if kind < 0.3:
+            reqs.append((1, max(kv, 1), 0, None))
+        elif kind < 0.7:
+            reqs.append((int(rng.integers(2, 300)), kv, 0, None))
+        else:
+            n = int(rng.integers(2, 48))
+            reqs.append((n, kv, 1, W.random_tree(rng, n, int(rng.integers(1, 9)))))
+    workers = int(rng.choice([2, 6, 30, 148]))
+    b = W.custom("pair_fuzz%d" % seed, hkv * G, hkv, page, reqs, seed=seed)
+    t = W.make_tensors(b)
+    ctx = H.make_ctx(b, kernel=xb.XY_KERNEL_PAIR, num_workers=workers, max_tree_nodes=64)
+    ctx.plan_batch(b)
+    O_ref, LSE_ref = oracle.attention(b, t, H.SCALE)
+    O1, L1 = H.run_gpu(b, t, ctx=ctx)
+    H.check_against_oracle(O1, L1, O_ref, LSE_ref, "pair fuzz %d" % seed)
+    O2, L2 = H.run_gpu(b, t, ctx=ctx)
+    assert np.array_equal(O1, O2) and np.array_equal(L1, L2)
+    ctx.close()
