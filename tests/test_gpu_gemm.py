@@ -142,3 +142,17 @@ def test_cta_pair_tiles_several_tiles_per_pair_and_strided_rows(tile_n):
 def test_library_choice_covers_pair_tiles():
     check(1024, 4096, 512, 0, seed=11)   # picks 256 x 256 pair tiles
     check(520, 28672, 128, 0, seed=12)   # 520 rows pad to 768: stays on single-CTA tiles
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_random_shapes_and_tile_choices(seed):
+    """Random M, N, K (multiples of 8 for N and K), random row strides and every tile choice,
+    pair tiles included."""
+    rng = np.random.default_rng(seed)
+    M = int(rng.integers(1, 700))
+    N = 8 * int(rng.integers(1, 90))
+    K = 8 * int(rng.integers(1, 90))
+    tile_n = int(rng.choice([0, 32, 64, 128, 256, PAIR | 128, PAIR | 256]))
+    lda = K + 8 * int(rng.integers(0, 3))
+    ldc = N + 8 * int(rng.integers(0, 3))
+    check(M, N, K, tile_n, seed=100 + seed, lda=lda, ldc=ldc)
