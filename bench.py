@@ -419,13 +419,31 @@ def measure_stream(kernel, dev, peaks, chunks=48, budget=4096, reserved=512, ses
     hits, misses = ctx.plan_cache()
     ctx.close()
     sch.close()
+    # Where the Task-Table cache does earn hits: 64 steps of a pure decode phase (every request one
+    # token further each step; a step misses only when some request enters a new 128-key tile).
+    # Host-only context: the planner alone is timed.
+    hctx = xb.XYAttn(64, 8, 128, device=-1, num_workers=148, max_requests=256)
+    hctx.plan_cache(64)
+    kv0 = np.random.default_rng(1).integers(512, 8192, size=64)
+    t_hit, t_miss = [], []
+    for step in range(64):
+        h_before = hctx.plan_cache()[0]
+        t0 = time.perf_counter()
+        hctx.plan([1] * 64, list(kv0 + step), [0] * 64, [-1] * 64)
+        dt = time.perf_counter() - t0
+        (t_hit if hctx.plan_cache()[0] > h_before else t_miss).append(dt)
+    dh, dm = hctx.plan_cache()
+    hctx.close()
+    decode_phase = {"requests": 64, "steps": 64, "hits": dh, "misses": dm,
+                    "plan_us_hit": 1e6 * float(np.median(t_hit)) if t_hit else None,
+                    "plan_us_miss": 1e6 * float(np.median(t_miss)) if t_miss else None}
     n = max(1, done)
     return {"chunks": done, "budget_tokens": budget, "reserved_dv_tokens": reserved, "sessions": sessions,
             "tokens": tokens, "sched_us_per_chunk": 1e6 * t_sched / n, "plan_us_per_chunk": 1e6 * t_plan / n,
             "attn_ms_per_chunk": (attn_ms + merge_ms) / n, "wall_ms_per_chunk": wall_ms / n,
             "tflops_attention": flops / ((attn_ms + merge_ms) * 1e-3) / 1e12,
             "kv_gbs_attention": kvb / ((attn_ms + merge_ms) * 1e-3) / 1e9,
-            "task_table_cache": {"hits": hits, "misses": misses}}
+            "task_table_cache": {"hits": hits, "misses": misses, "decode_phase": decode_phase}}
 
 
 def measure_gemm(dev, peaks, steps=20):
